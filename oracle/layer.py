@@ -1,0 +1,121 @@
+"""One drafter backbone block around the all-boundary attention (test infrastructure).
+
+PARITY UNPINNED (structure): the paper names the backbone blocks only as "attention, MLP, and their
+normalizations" (Sec. 3.1, trainable/frozen split) and fixes no layer equations.  The block below is
+this build's reading -- the pre-norm block of the Qwen3 family the drafters are trained for:
+
+    xn  = bf16( rmsnorm(x) * g1 )
+    qkv = bf16( xn W_qkv^T )                      rows split as [Hq*D | Hkv*D | Hkv*D]
+    q,k = bf16( rmsnorm_over_D(.) * gain )        per head, when QK-norm is on
+    q,k = bf16( rope(., position) )               rotate-half, when RoPE is on
+    a   = bf16( all-boundary attention )          the mask slots' own k, v are the block keys/values;
+                                                  context and spine K/V are inputs (already projected)
+    h1  = fp32( x + a W_o^T )
+    hn  = bf16( rmsnorm(h1) * g2 )
+    act = bf16( silu(hn W_gate^T) * (hn W_up^T) )
+    y   = fp32( h1 + act W_down^T )
+
+The bf16 roundings are part of the definition ("bf16 inputs, fp32 accumulate" for every product); the
+sums themselves are taken in float64 here.  Positions: spine row s of request n sits at L_n + s; the
+unknown bonus of boundary j would sit at L_n + j + 1; mask slot i of boundary j therefore sits at
+L_n + j + 2 + i.  The individual pieces (rmsnorm, silu, rope, matmul) are pinned by closed forms in
+the tests; the composition is pinned by nothing but this text.
+"""
+from __future__ import annotations
+
+import math
+from typing import Optional
+
+import numpy as np
+
+from .attention import bf16_bits_to_f64, round_to_bf16, softmax_attention
+
+
+def _r16(x):
+    """Round to bf16, keep as float64 values."""
+    return round_to_bf16(x).astype(np.float64)
+
+
+def rmsnorm(x: np.ndarray, gain: Optional[np.ndarray], eps: float) -> np.ndarray:
+    """x / sqrt(mean(x^2) + eps) * gain over the last axis (float64)."""
+    ms = (x * x).mean(axis=-1, keepdims=True)
+    y = x / np.sqrt(ms + eps)
+    return y if gain is None else y * gain
+
+
+def silu(x: np.ndarray) -> np.ndarray:
+    return x / (1.0 + np.exp(-x))
+
+
+def rope(x: np.ndarray, pos: np.ndarray, theta: float) -> np.ndarray:
+    """Rotate-half rotary embedding.  x [..., R, D] with one position per row R (pos [R]).
+    Pair (d, d + D/2) is rotated by angle pos * theta^(-2d/D)."""
+    D = x.shape[-1]
+    half = D // 2
+    inv = theta ** (-2.0 * np.arange(half) / D)
+    ang = pos[:, None].astype(np.float64) * inv[None, :]
+    c, s = np.cos(ang), np.sin(ang)
+    x1, x2 = x[..., :half], x[..., half:]
+    return np.concatenate([x1 * c - x2 * s, x2 * c + x1 * s], axis=-1)
+
+
+class LayerOracle:
+    """Holds the decoded weights so that several boundaries can be evaluated without re-decoding."""
+
+    def __init__(self, lin, attn_in, prefix_base: int = 1, scale: Optional[float] = None):
+        sh = attn_in.shape
+        self.sh, self.lsh, self.ain = sh, lin.shape, attn_in
+        self.prefix_base = prefix_base
+        self.scale = scale if scale else 1.0 / math.sqrt(sh.head_dim)
+        self.x = lin.x
+        self.w_qkv = bf16_bits_to_f64(lin.w_qkv)
+        self.w_o = bf16_bits_to_f64(lin.w_o)
+        self.w_gu = bf16_bits_to_f64(lin.w_gate_up)
+        self.w_down = bf16_bits_to_f64(lin.w_down)
+        self.g1 = bf16_bits_to_f64(lin.rms1_w)
+        self.g2 = bf16_bits_to_f64(lin.rms2_w)
+        self.gq = bf16_bits_to_f64(lin.qnorm_w) if self.lsh.qk_norm else None
+        self.gk = bf16_bits_to_f64(lin.knorm_w) if self.lsh.qk_norm else None
+
+    def qkv_rows(self, n: int, j: int):
+        """q [Bq][Hq][D], k [Bq][Hkv][D], v [Bq][Hkv][D] of boundary j's mask slots (bf16 values, float64)."""
+        sh, L = self.sh, self.lsh
+        Hq, Hkv, D, Bq = sh.n_q_heads, sh.n_kv_heads, sh.head_dim, sh.block
+        x = bf16_bits_to_f64(self.x[n, j])                                   # [Bq][hidden]
+        xn = _r16(rmsnorm(x, self.g1, L.rms_eps))
+        qkv = _r16(xn @ self.w_qkv.T)
+        q = qkv[:, : Hq * D].reshape(Bq, Hq, D)
+        k = qkv[:, Hq * D:(Hq + Hkv) * D].reshape(Bq, Hkv, D)
+        v = qkv[:, (Hq + Hkv) * D:].reshape(Bq, Hkv, D)
+        if L.qk_norm:
+            q = _r16(rmsnorm(q, self.gq, L.rms_eps))
+            k = _r16(rmsnorm(k, self.gk, L.rms_eps))
+        if L.use_rope:
+            pos = sh.ctx_lens[n] + j + 2 + np.arange(Bq)
+            q = _r16(rope(q.transpose(1, 0, 2), pos, L.rope_theta)).transpose(1, 0, 2)
+            k = _r16(rope(k.transpose(1, 0, 2), pos, L.rope_theta)).transpose(1, 0, 2)
+        return x, q, k, v
+
+    def boundary(self, n: int, j: int):
+        """Forward of boundary j of request n.  Returns dict with y [Bq][hidden] (fp32 values) and the
+        intermediates q, k, v, a, h1."""
+        sh, L, A = self.sh, self.lsh, self.ain
+        Hq, Hkv, D, Bq = sh.n_q_heads, sh.n_kv_heads, sh.head_dim, sh.block
+        G = Hq // Hkv
+        x, q, k, v = self.qkv_rows(n, j)
+        lo, hi = int(A.ctx_offsets[n]), int(A.ctx_offsets[n + 1])
+        n_anchor = max(0, min(j + self.prefix_base, sh.spine))
+        a = np.zeros((Bq, Hq, D))
+        for g in range(Hkv):
+            keys = np.concatenate([bf16_bits_to_f64(A.k_ctx[lo:hi, g]), bf16_bits_to_f64(A.k_spine[n, :n_anchor, g]), k[:, g]])
+            vals = np.concatenate([bf16_bits_to_f64(A.v_ctx[lo:hi, g]), bf16_bits_to_f64(A.v_spine[n, :n_anchor, g]), v[:, g]])
+            for h in range(g * G, (g + 1) * G):
+                a[:, h], _ = softmax_attention(q[:, h], keys, vals, self.scale)
+        a = _r16(a).reshape(Bq, Hq * D)
+        h1 = (x + a @ self.w_o.T).astype(np.float32).astype(np.float64)
+        hn = _r16(rmsnorm(h1, self.g2, L.rms_eps))
+        gu = hn @ self.w_gu.T
+        I = L.intermediate
+        act = _r16(silu(gu[:, :I]) * gu[:, I:])
+        y = (h1 + act @ self.w_down.T).astype(np.float32)
+        return dict(y=y, q=q, k=k, v=v, a=a, h1=h1.astype(np.float32))

@@ -1,0 +1,118 @@
+"""Pins for oracle/layer.py pieces (closed forms, library routines) and the input generators (CPU only).
+The block STRUCTURE is this build's reading of the paper ("attention, MLP, and their normalizations")
+and stays unpinned by the paper; the library-composed check below only guards against slips."""
+import math
+
+import numpy as np
+import torch
+import torch.nn.functional as F
+
+import workloads as W
+from oracle import attention as OA
+from oracle import layer as OL
+
+
+def test_rmsnorm_closed_form_and_library():
+    x = np.full((2, 8), 3.0)
+    g = np.arange(1, 9, dtype=np.float64)
+    assert np.allclose(OL.rmsnorm(x, g, 1e-6), 3.0 / math.sqrt(9.0 + 1e-6) * g)
+    r = np.random.default_rng(0).standard_normal((5, 64))
+    ref = F.rms_norm(torch.from_numpy(r), (64,), torch.from_numpy(np.ones(64)), 1e-6).numpy()
+    assert np.allclose(OL.rmsnorm(r, None, 1e-6), ref, atol=1e-14)
+
+
+def test_silu():
+    x = np.linspace(-6, 6, 25)
+    assert OL.silu(np.zeros(1))[0] == 0
+    assert np.allclose(OL.silu(x), F.silu(torch.from_numpy(x)).numpy(), atol=1e-15)
+
+
+def test_rope_properties():
+    rng = np.random.default_rng(1)
+    x = rng.standard_normal((3, 4, 16))
+    pos = np.array([0, 5, 1000, 40000])
+    y = OL.rope(x, pos, 1e6)
+    assert np.allclose(y[:, 0], x[:, 0])                                         # position 0: identity
+    assert np.allclose((y * y).sum(-1), (x * x).sum(-1))                           # a rotation
+    # D = 2 is a plain planar rotation by the position (frequency 1)
+    v = np.array([[[1.0, 0.0]]])
+    r = OL.rope(v, np.array([math.pi / 2]), 1e6)
+    assert np.allclose(r[0, 0], [0.0, 1.0], atol=1e-15)
+    # scores depend on the position difference only
+    q, k = rng.standard_normal((1, 1, 16)), rng.standard_normal((1, 1, 16))
+    s1 = (OL.rope(q, np.array([17]), 1e4) * OL.rope(k, np.array([11]), 1e4)).sum()
+    s2 = (OL.rope(q, np.array([1017]), 1e4) * OL.rope(k, np.array([1011]), 1e4)).sum()
+    assert abs(s1 - s2) < 1e-9
+    # pair (d, d + D/2) turns with frequency theta^(-2d/D)
+    e = np.zeros((1, 1, 8)); e[0, 0, 1] = 1
+    r = OL.rope(e, np.array([3]), 100.0)
+    ang = 3 * 100.0 ** (-2 / 8)
+    assert np.allclose(r[0, 0, [1, 5]], [math.cos(ang), math.sin(ang)])
+
+
+def _small():
+    a = W.AttnShape((19, 7), 4, 2, 16, 3, 2)
+    l = W.LayerShape(64, 96)
+    return W.make_attn_inputs(a, 5), W.make_layer_inputs(l, a, 5)
+
+
+def test_layer_identity_when_projections_vanish():
+    ain, lin = _small()
+    lin.w_o[:] = 0
+    lin.w_down[:] = 0
+    orc = OL.LayerOracle(lin, ain)
+    y = orc.boundary(1, 2)["y"]
+    assert np.array_equal(y, OA.bf16_bits_to_f64(lin.x[1, 2]).astype(np.float32))
+
+
+def test_layer_against_library_composition():
+    """Same block assembled from torch library routines in float64 without the bf16 roundings."""
+    ain, lin = _small()
+    orc = OL.LayerOracle(lin, ain)
+    sh = ain.shape
+    Hq, Hkv, D, Bq = 4, 2, 16, 2
+    d = lambda b: torch.from_numpy(OA.bf16_bits_to_f64(b))
+    for (n, j) in [(0, 0), (1, 2)]:
+        got = orc.boundary(n, j)
+        x = d(lin.x[n, j])
+        xn = F.rms_norm(x, (64,), d(lin.rms1_w), 1e-6)
+        qkv = F.linear(xn, d(lin.w_qkv))
+        q = qkv[:, :64].reshape(Bq, Hq, D); k = qkv[:, 64:96].reshape(Bq, Hkv, D); v = qkv[:, 96:].reshape(Bq, Hkv, D)
+        q = F.rms_norm(q, (D,), d(lin.qnorm_w), 1e-6); k = F.rms_norm(k, (D,), d(lin.knorm_w), 1e-6)
+        pos = torch.tensor([sh.ctx_lens[n] + j + 2 + i for i in range(Bq)], dtype=torch.float64)
+        inv = 1e6 ** (-torch.arange(0, D, 2, dtype=torch.float64) / D)
+        ang = pos[:, None] * inv[None]
+        cos, sin = torch.cat([ang.cos(), ang.cos()], -1)[:, None], torch.cat([ang.sin(), ang.sin()], -1)[:, None]
+        rot = lambda t: torch.cat([-t[..., D // 2:], t[..., :D // 2]], -1)
+        q = q * cos + rot(q) * sin; k = k * cos + rot(k) * sin
+        lo, hi = int(ain.ctx_offsets[n]), int(ain.ctx_offsets[n + 1])
+        K = torch.cat([d(ain.k_ctx[lo:hi]), d(ain.k_spine[n, :j + 1]), k], 0)
+        V = torch.cat([d(ain.v_ctx[lo:hi]), d(ain.v_spine[n, :j + 1]), v], 0)
+        a = F.scaled_dot_product_attention(q.permute(1, 0, 2)[None], K.permute(1, 0, 2)[None], V.permute(1, 0, 2)[None],
+                                           enable_gqa=True)[0].permute(1, 0, 2).reshape(Bq, Hq * D)
+        h1 = x + F.linear(a, d(lin.w_o))
+        hn = F.rms_norm(h1, (64,), d(lin.rms2_w), 1e-6)
+        gu = F.linear(hn, d(lin.w_gate_up))
+        y = h1 + F.linear(F.silu(gu[:, :96]) * gu[:, 96:], d(lin.w_down))
+        assert np.abs(y.numpy() - got["y"]).max() < 2e-2          # only the bf16 rounding points differ
+        assert np.abs(a.numpy() - got["a"]).max() < 2e-2
+
+
+def test_generators_are_seeded_and_shaped():
+    w3 = W.workload(3)
+    assert w3.attn.batch == 16 and all(512 <= L <= 4096 for L in w3.attn.ctx_lens)
+    assert W.workload(3).attn.ctx_lens == w3.attn.ctx_lens
+    w1 = W.workload(1)
+    a = W.make_attn_inputs(w1.attn, w1.seed)
+    b = W.make_attn_inputs(w1.attn, w1.seed)
+    assert np.array_equal(a.q, b.q) and a.q.shape == (1, 5, 4, 4, 64) and a.k_ctx.shape == (128, 2, 64)
+    assert a.k_spine.shape == (1, 5, 2, 64) and a.k_blk.shape == (1, 5, 4, 2, 64)
+    x = W.bf16_bits_to_f32(a.k_ctx).astype(np.float64)
+    assert abs(x.mean()) < 0.05 and abs(x.std() - 1) < 0.05
+    v = W.make_verify_inputs(w1.verify, w1.seed)
+    assert v.target.shape == (1, 5, 1000) and v.draft_tokens.shape == (1, 4)
+    sv = W.VerifyShape(3, 4, 64, 2, 8, "sampling", 0.0, 3.0)
+    s = W.make_verify_inputs(sv, 9)
+    assert np.allclose(s.target.sum(-1), 1, atol=1e-5) and np.allclose(s.draft_probs.sum(-1), 1, atol=1e-5)
+    m = s.uniforms.astype(np.float64) * 2 ** 24
+    assert np.array_equal(m, np.round(m)) and m.max() < 2 ** 24 and m.min() >= 0
