@@ -1,0 +1,173 @@
+/* dpara.h -- C ABI of the B200 (sm_100a) all-boundary draft step.
+ *
+ * The method (paper Alg. 1): while the target model verifies the draft block t_{0:d}, the drafter
+ * backbone precomputes, in one pass, draft representations for EVERY acceptance boundary r = 0..d
+ * (Alg. 1 line 1, Sec. 3.2, Fig. 4); when verification returns the accepted length r and the bonus
+ * token b (Alg. 1 line 2, Sec. 2.1), branch r is selected (Alg. 1 line 3) and handed to the
+ * autoregressive head.  This library implements those two calls:
+ *
+ *   dpara_draft_all_boundaries  -- Alg. 1 line 1 for one backbone block: the tree-masked attention
+ *                                  of Fig. 4 for all boundaries at once (optionally wrapped in the
+ *                                  block's projections, norms and MLP).
+ *   dpara_verify_select         -- Alg. 1 lines 2-3 after the target forward: accepted length, bonus
+ *                                  token (greedy, or the rejection rule of App. C) and the gather of
+ *                                  the selected branch's representation.
+ *
+ * Conventions
+ *   - Every pointer is a DEVICE pointer unless its name starts with host_.  The caller owns every
+ *     buffer; the library allocates nothing and keeps no state between calls.
+ *   - Calls enqueue kernels on `stream` (a cudaStream_t passed as void*) and return without
+ *     synchronising.  Outputs are valid once the stream has reached the end of the call's work.
+ *   - The return code reports host-detectable errors; on any error nothing has been launched.
+ *     Conditions only the device can see (a draft token outside the vocabulary, a bounded wait that
+ *     expired) OR a bit into *status_word (may be NULL) and the kernels still finish with defined
+ *     outputs.
+ *   - bf16 tensors are row-major with the last index contiguous and must be 16-byte aligned.
+ *   - J = n_boundaries = d + 1.  Boundary j reads spine rows [0, min(j + prefix_base, n_spine)).
+ */
+#ifndef DPARA_H_
+#define DPARA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  DPARA_OK = 0,
+  DPARA_ERR_INVALID_ARG = -1, /* null pointer, non-positive size, misaligned buffer, bad range */
+  DPARA_ERR_UNSUPPORTED = -2, /* shape outside what the kernels are built for (see each call) */
+  DPARA_ERR_WORKSPACE = -3,   /* workspace missing or smaller than *_workspace_bytes() */
+  DPARA_ERR_CUDA = -4,        /* a CUDA runtime/driver call failed (launch, tensor-map encode) */
+  DPARA_ERR_TIMEOUT = -5      /* reserved for device-side bounded waits, reported via status_word */
+} dpara_status;
+
+/* bits OR-ed into *status_word by kernels */
+#define DPARA_STATUS_BAD_TOKEN 1u /* a draft token outside [0, vocab): rejected at that position */
+#define DPARA_STATUS_TIMEOUT 2u   /* a bounded device-side wait gave up; outputs of that tile are undefined */
+
+typedef enum { DPARA_BF16 = 0, DPARA_F32 = 1 } dpara_dtype;
+
+/* Shapes of one draft call (Sec. 3.2: d+1 boundaries, each a block of mask slots). */
+typedef struct {
+  int32_t batch;        /* b requests */
+  int32_t n_boundaries; /* J = d + 1 */
+  int32_t block;        /* Bq mask slots (query rows) per boundary */
+  int32_t n_q_heads;    /* Hq */
+  int32_t n_kv_heads;   /* Hkv; Hq % Hkv == 0; query head h reads KV head h / (Hq/Hkv) */
+  int32_t head_dim;     /* D: 64 or 128 */
+  int32_t prefix_base;  /* anchors visible to boundary j = j + prefix_base; paper (k = r + 1): 1 */
+  int32_t n_spine;      /* S spine rows stored per request (normally J) */
+  int32_t boundary_lo;  /* boundaries computed: [boundary_lo, boundary_hi); all = [0, J);        */
+  int32_t boundary_hi;  /* a conventional single-anchor-set draft step = [j, j + 1)               */
+  float softmax_scale;  /* 0 selects 1/sqrt(D) */
+} dpara_shape;
+
+/* Tensors of the attention (Fig. 4).  Context keys/values are the drafter-side projection of the
+ * cached target features C (Alg. 1 Require); spine keys/values belong to the feature-less draft block
+ * t_{0:d}; block keys/values belong to the mask slots themselves (branches attend bidirectionally
+ * within their own block).  In full-layer mode q, k_blk, v_blk and out may be NULL: they are
+ * produced inside the call. */
+typedef struct {
+  const void *q;                   /* [b][J][Bq][Hq][D] bf16 */
+  const void *k_ctx, *v_ctx;       /* [sum_n L_n][Hkv][D] bf16; request n owns rows ctx_offsets[n]..ctx_offsets[n+1) */
+  const int64_t *ctx_offsets;      /* [b+1] device copy */
+  const int64_t *host_ctx_offsets; /* [b+1] HOST copy of the same values (needed to size the grid) */
+  const void *k_spine, *v_spine;   /* [b][S][Hkv][D] bf16 */
+  const void *k_blk, *v_blk;       /* [b][J][Bq][Hkv][D] bf16; both NULL: slots read no block keys */
+  void *out;                       /* [b][J][Bq][Hq][D], dtype out_dtype; rows of boundaries outside [lo,hi) untouched */
+  int32_t out_dtype;               /* dpara_dtype */
+  float *out_lse;                  /* optional [b][J][Bq][Hq]: natural-log sum-exp of the scaled scores (NULL ok) */
+} dpara_attn_io;
+
+/* Full-layer mode (one pre-norm backbone block; the paper names only "attention, MLP, and their
+ * normalizations", Sec. 3.1 -- the equations are this library's reading, stated with the call). */
+typedef struct {
+  const void *x;                                   /* [b][J][Bq][hidden] bf16 hidden states of the mask slots */
+  const void *w_qkv;                               /* [(Hq + 2 Hkv) D][hidden] bf16, rows = [q | k | v] */
+  const void *w_o;                                 /* [hidden][Hq D] bf16 */
+  const void *w_gate_up;                           /* [2 inter][hidden] bf16, rows [0,inter) gate, [inter,2 inter) up */
+  const void *w_down;                              /* [hidden][inter] bf16 */
+  const void *rms1_w, *rms2_w;                     /* [hidden] bf16 gains; NULL = ones */
+  const void *qnorm_w, *knorm_w;                   /* [D] bf16 gains of the per-head q/k RMS norm; both NULL = no QK-norm */
+  float rms_eps;
+  float rope_theta;
+  int32_t use_rope;                                /* slot i of boundary j of request n sits at position L_n + j + 2 + i */
+  int32_t hidden, intermediate;
+  float *y_f32;                                    /* [b][J][Bq][hidden] fp32 output (required) */
+  void *y_bf16;                                    /* optional bf16 copy of y (NULL ok) */
+} dpara_layer_io;
+
+/* Bytes of scratch dpara_draft_all_boundaries needs for these shapes (0 is possible).
+ * host_ctx_offsets: [b+1] host array.  full_layer != 0: include the block's intermediates
+ * (hidden/intermediate are taken from `layer`, which may be NULL when full_layer == 0). */
+size_t dpara_draft_workspace_bytes(const dpara_shape *shape, const int64_t *host_ctx_offsets,
+                                   const dpara_layer_io *layer, int full_layer);
+
+/* Alg. 1 line 1 / Sec. 3.2 / Fig. 4.  For every request n, boundary j in [lo,hi), slot i, head h:
+ *   out = softmax(scale * q K^T) V over the keys  context[0..L_n)  ++  spine[0..min(j+prefix_base,S))
+ *   ++  block j (all Bq slots; omitted when k_blk == NULL),  fp32 accumulation, bf16 inputs.
+ * A row with no visible key gives out = 0 and lse = -inf.
+ * layer == NULL: attention only, on io->q / io->k_blk / io->v_blk.
+ * layer != NULL: xn = bf16(rmsnorm(x) g1); [q|k|v] = bf16(xn Wqkv^T); per-head RMS norm and rotary
+ *   embedding (rotate-half) on q, k, each rounded to bf16; the slots' own k, v are the block
+ *   keys/values; a = bf16(attention); h1 = x + a Wo^T (fp32); hn = bf16(rmsnorm(h1) g2);
+ *   act = bf16(silu(hn Wg^T) * (hn Wu^T)); y = h1 + act Wd^T (fp32).
+ * workspace: device scratch of at least dpara_draft_workspace_bytes(); contents need not be
+ *   initialised and are garbage afterwards; two calls in flight must not share it.
+ * Errors: INVALID_ARG (null/misaligned/ranges, ctx_offsets not non-decreasing), UNSUPPORTED
+ *   (head_dim not 64/128, Hq % Hkv != 0, Hq/Hkv > 16, block > 64, n_spine > 64), WORKSPACE, CUDA. */
+dpara_status dpara_draft_all_boundaries(const dpara_shape *shape, const dpara_attn_io *io,
+                                        const dpara_layer_io *layer, void *workspace,
+                                        size_t workspace_bytes, int32_t *status_word, void *stream);
+
+/* Verification-side tensors (Sec. 2.1; App. C for mode 1).  Row i of `target` is the target's
+ * prediction for the token after t_0..t_i, so draft t_{i+1} is judged by row i and the bonus comes
+ * from row r. */
+typedef struct {
+  int32_t batch;               /* b */
+  int32_t n_boundaries;        /* J = d + 1 target rows per request */
+  int32_t vocab;               /* V */
+  int32_t block;               /* Bq rows per representation */
+  int32_t hidden;              /* elements per representation row */
+  int32_t mode;                /* 0 greedy on logits, 1 rejection sampling on probabilities */
+  const float *target;         /* [b][J][V] fp32: logits (mode 0) or probabilities (mode 1) */
+  const float *draft_probs;    /* [b][J-1][V] fp32, mode 1 only: row i is the drafter distribution t_{i+1} was drawn from */
+  const int32_t *draft_tokens; /* [b][J-1] = t_1..t_d */
+  const float *uniforms;       /* [b][J] fp32, mode 1 only; each = m * 2^-24, m integer in [0, 2^24):
+                                  u[i] tests draft t_{i+1}; u[J-1] draws the bonus */
+  const void *reps;            /* [b][J][Bq][hidden] bf16 (e.g. `out`/`y_bf16` of the draft call); NULL: no gather */
+  int32_t *accept_len;         /* [b] r */
+  int32_t *bonus;              /* [b] b */
+  int32_t *gather_idx;         /* [b] index of the selected branch (= r) */
+  int32_t *out_tokens;         /* optional [b][J]: t_1..t_r, bonus, then -1 */
+  void *selected;              /* [b][Bq][hidden] bf16 = reps[n][r] (required when reps != NULL) */
+} dpara_verify_io;
+
+/* Bytes of scratch dpara_verify_select needs; only the sizes and mode of `io` are read. 0 on bad sizes. */
+size_t dpara_verify_workspace_bytes(const dpara_verify_io *io);
+
+/* Alg. 1 lines 2-3.  mode 0: a_i = lowest index of the maximum of row i (-0 == +0, NaN below every
+ * number); r = number of leading drafts with t_i == a_{i-1}; bonus = a_r.
+ * mode 1: draft t_i accepted iff fl32(u[i-1] * q_{i-1}(t_i)) < p_{i-1}(t_i), scan stops at the first
+ * rejection; bonus drawn by inverse CDF in vocabulary order from integer weights
+ * trunc(max(fl32(p_r - q_r), 0) * 2^32) (r < d) or trunc(p_d * 2^32) (r = d) with threshold
+ * (m * W) >> 24; empty residual falls back to p_r, then to the lowest-index maximum of p_r.
+ * A draft token outside [0, V) is rejected and sets DPARA_STATUS_BAD_TOKEN.
+ * selected[n] = reps[n][r] copied bit for bit.
+ * workspace: at least dpara_verify_workspace_bytes(); need not be initialised.
+ * Errors: INVALID_ARG, UNSUPPORTED (J > 64), WORKSPACE, CUDA. */
+dpara_status dpara_verify_select(const dpara_verify_io *io, void *workspace, size_t workspace_bytes,
+                                 int32_t *status_word, void *stream);
+
+const char *dpara_status_string(dpara_status s);
+
+/* Library/ABI version: major * 1000 + minor. */
+int32_t dpara_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DPARA_H_ */

@@ -1,0 +1,193 @@
+"""Python binding of libdpara.so (B200 / sm_100a all-boundary draft step).
+
+Argument marshalling only: every step of the path runs in the CUDA kernels behind the C ABI declared
+in include/dpara.h.  PyTorch supplies device memory and streams.  There is no CPU fallback: if the
+shared library is missing, importing this package raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libdpara.so")
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        f"{LIB_PATH} is missing: build it with `python -m paper_2609_27396_b200.build` "
+        "(nvcc, sm_100a). This package has no CPU fallback.")
+
+lib = C.CDLL(LIB_PATH)
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = 0, -1, -2, -3, -4, -5
+STATUS_BAD_TOKEN, STATUS_TIMEOUT = 1, 2
+BF16, F32 = 0, 1
+
+
+class Shape(C.Structure):
+    _fields_ = [("batch", C.c_int32), ("n_boundaries", C.c_int32), ("block", C.c_int32), ("n_q_heads", C.c_int32),
+                ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32), ("prefix_base", C.c_int32), ("n_spine", C.c_int32),
+                ("boundary_lo", C.c_int32), ("boundary_hi", C.c_int32), ("softmax_scale", C.c_float)]
+
+
+class AttnIO(C.Structure):
+    _fields_ = [("q", C.c_void_p), ("k_ctx", C.c_void_p), ("v_ctx", C.c_void_p), ("ctx_offsets", C.c_void_p),
+                ("host_ctx_offsets", C.c_void_p), ("k_spine", C.c_void_p), ("v_spine", C.c_void_p),
+                ("k_blk", C.c_void_p), ("v_blk", C.c_void_p), ("out", C.c_void_p), ("out_dtype", C.c_int32),
+                ("out_lse", C.c_void_p)]
+
+
+class LayerIO(C.Structure):
+    _fields_ = [("x", C.c_void_p), ("w_qkv", C.c_void_p), ("w_o", C.c_void_p), ("w_gate_up", C.c_void_p),
+                ("w_down", C.c_void_p), ("rms1_w", C.c_void_p), ("rms2_w", C.c_void_p), ("qnorm_w", C.c_void_p),
+                ("knorm_w", C.c_void_p), ("rms_eps", C.c_float), ("rope_theta", C.c_float), ("use_rope", C.c_int32),
+                ("hidden", C.c_int32), ("intermediate", C.c_int32), ("y_f32", C.c_void_p), ("y_bf16", C.c_void_p)]
+
+
+class VerifyIO(C.Structure):
+    _fields_ = [("batch", C.c_int32), ("n_boundaries", C.c_int32), ("vocab", C.c_int32), ("block", C.c_int32),
+                ("hidden", C.c_int32), ("mode", C.c_int32), ("target", C.c_void_p), ("draft_probs", C.c_void_p),
+                ("draft_tokens", C.c_void_p), ("uniforms", C.c_void_p), ("reps", C.c_void_p), ("accept_len", C.c_void_p),
+                ("bonus", C.c_void_p), ("gather_idx", C.c_void_p), ("out_tokens", C.c_void_p), ("selected", C.c_void_p)]
+
+
+lib.dpara_draft_workspace_bytes.restype = C.c_size_t
+lib.dpara_draft_workspace_bytes.argtypes = [C.POINTER(Shape), C.c_void_p, C.POINTER(LayerIO), C.c_int]
+lib.dpara_draft_all_boundaries.restype = C.c_int
+lib.dpara_draft_all_boundaries.argtypes = [C.POINTER(Shape), C.POINTER(AttnIO), C.POINTER(LayerIO), C.c_void_p,
+                                           C.c_size_t, C.c_void_p, C.c_void_p]
+lib.dpara_verify_workspace_bytes.restype = C.c_size_t
+lib.dpara_verify_workspace_bytes.argtypes = [C.POINTER(VerifyIO)]
+lib.dpara_verify_select.restype = C.c_int
+lib.dpara_verify_select.argtypes = [C.POINTER(VerifyIO), C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
+lib.dpara_status_string.restype = C.c_char_p
+lib.dpara_status_string.argtypes = [C.c_int]
+lib.dpara_version.restype = C.c_int32
+
+EXPORTED = ["dpara_draft_workspace_bytes", "dpara_draft_all_boundaries", "dpara_verify_workspace_bytes",
+            "dpara_verify_select", "dpara_status_string", "dpara_version"]
+
+
+class DparaError(RuntimeError):
+    def __init__(self, code: int):
+        self.code = code
+        super().__init__(f"dpara: {lib.dpara_status_string(code).decode()} ({code})")
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_contiguous():
+        raise ValueError("dpara: tensors must be contiguous")
+    return t.data_ptr()
+
+
+def _stream_ptr(stream) -> int:
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return s.cuda_stream
+
+
+def _host_offsets(ctx_offsets: Sequence[int]):
+    arr = (C.c_int64 * len(ctx_offsets))(*[int(x) for x in ctx_offsets])
+    return arr
+
+
+class DraftPlan:
+    """Fixed-address buffers for repeated draft calls on one shape (shape struct, host and device copies
+    of the context offsets, workspace, status word).  Building the plan allocates; calling it does not."""
+
+    def __init__(self, *, ctx_offsets: Sequence[int], n_boundaries: int, block: int, n_q_heads: int, n_kv_heads: int,
+                 head_dim: int, prefix_base: int = 1, n_spine: Optional[int] = None, boundary_lo: int = 0,
+                 boundary_hi: Optional[int] = None, softmax_scale: float = 0.0, layer: Optional[LayerIO] = None,
+                 device="cuda"):
+        b = len(ctx_offsets) - 1
+        self.shape = Shape(b, n_boundaries, block, n_q_heads, n_kv_heads, head_dim, prefix_base,
+                           n_boundaries if n_spine is None else n_spine, boundary_lo,
+                           n_boundaries if boundary_hi is None else boundary_hi, softmax_scale)
+        self.host_off = _host_offsets(ctx_offsets)
+        self.dev_off = torch.tensor([int(x) for x in ctx_offsets], dtype=torch.int64, device=device)
+        self.layer = layer
+        need = lib.dpara_draft_workspace_bytes(C.byref(self.shape), C.cast(self.host_off, C.c_void_p),
+                                               C.byref(layer) if layer is not None else None, 1 if layer is not None else 0)
+        self.workspace_bytes = int(need)
+        self.workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=device)
+        self.status = torch.zeros(1, dtype=torch.int32, device=device)
+
+    def __call__(self, *, q=None, k_ctx=None, v_ctx=None, k_spine=None, v_spine=None, k_blk=None, v_blk=None,
+                 out=None, out_lse=None, stream=None) -> None:
+        io = AttnIO(_ptr(q), _ptr(k_ctx), _ptr(v_ctx), self.dev_off.data_ptr(), C.cast(self.host_off, C.c_void_p).value,
+                    _ptr(k_spine), _ptr(v_spine), _ptr(k_blk), _ptr(v_blk), _ptr(out),
+                    F32 if (out is not None and out.dtype == torch.float32) else BF16, _ptr(out_lse))
+        rc = lib.dpara_draft_all_boundaries(C.byref(self.shape), C.byref(io),
+                                            C.byref(self.layer) if self.layer is not None else None,
+                                            self.workspace.data_ptr(), self.workspace.numel(), self.status.data_ptr(),
+                                            _stream_ptr(stream))
+        if rc != OK:
+            raise DparaError(rc)
+
+
+def make_layer_io(*, x, w_qkv, w_o, w_gate_up, w_down, rms1_w=None, rms2_w=None, qnorm_w=None, knorm_w=None,
+                  rms_eps=1e-6, rope_theta=1e6, use_rope=True, y_f32=None, y_bf16=None) -> LayerIO:
+    hidden = x.shape[-1]
+    inter = w_down.shape[-1]
+    return LayerIO(_ptr(x), _ptr(w_qkv), _ptr(w_o), _ptr(w_gate_up), _ptr(w_down), _ptr(rms1_w), _ptr(rms2_w),
+                   _ptr(qnorm_w), _ptr(knorm_w), rms_eps, rope_theta, 1 if use_rope else 0, hidden, inter,
+                   _ptr(y_f32), _ptr(y_bf16))
+
+
+def draft_all_boundaries(q, k_ctx, v_ctx, ctx_offsets: Sequence[int], k_spine, v_spine, k_blk=None, v_blk=None, *,
+                         prefix_base: int = 1, boundary_lo: int = 0, boundary_hi: Optional[int] = None,
+                         softmax_scale: float = 0.0, out_dtype=torch.bfloat16, want_lse: bool = False, stream=None):
+    """All-boundary attention (dpara_draft_all_boundaries, attention-only mode).
+    q [b][J][Bq][Hq][D] bf16 CUDA tensor; returns out (same shape, out_dtype) and optionally lse."""
+    b, J, Bq, Hq, D = q.shape
+    Hkv = k_spine.shape[2]
+    plan = DraftPlan(ctx_offsets=ctx_offsets, n_boundaries=J, block=Bq, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=D,
+                     prefix_base=prefix_base, n_spine=k_spine.shape[1], boundary_lo=boundary_lo, boundary_hi=boundary_hi,
+                     softmax_scale=softmax_scale, device=q.device)
+    out = torch.zeros(q.shape, dtype=out_dtype, device=q.device)
+    lse = torch.full((b, J, Bq, Hq), float("-inf"), dtype=torch.float32, device=q.device) if want_lse else None
+    plan(q=q, k_ctx=k_ctx, v_ctx=v_ctx, k_spine=k_spine, v_spine=v_spine, k_blk=k_blk, v_blk=v_blk, out=out, out_lse=lse,
+         stream=stream)
+    return (out, lse, plan.status) if want_lse else (out, plan.status)
+
+
+class VerifyPlan:
+    """Fixed-address outputs and workspace for repeated verify/select calls on one shape."""
+
+    def __init__(self, *, batch: int, n_boundaries: int, vocab: int, block: int, hidden: int, mode: int, device="cuda"):
+        self.io = VerifyIO(batch, n_boundaries, vocab, block, hidden, mode)
+        self.accept_len = torch.zeros(batch, dtype=torch.int32, device=device)
+        self.bonus = torch.zeros(batch, dtype=torch.int32, device=device)
+        self.gather_idx = torch.zeros(batch, dtype=torch.int32, device=device)
+        self.out_tokens = torch.zeros(batch, n_boundaries, dtype=torch.int32, device=device)
+        self.selected = torch.zeros(batch, block, hidden, dtype=torch.bfloat16, device=device)
+        self.status = torch.zeros(1, dtype=torch.int32, device=device)
+        self.io.accept_len, self.io.bonus = self.accept_len.data_ptr(), self.bonus.data_ptr()
+        self.io.gather_idx, self.io.out_tokens = self.gather_idx.data_ptr(), self.out_tokens.data_ptr()
+        self.io.selected = self.selected.data_ptr()
+        need = lib.dpara_verify_workspace_bytes(C.byref(self.io))
+        self.workspace_bytes = int(need)
+        self.workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=device)
+
+    def __call__(self, *, target, draft_tokens, reps=None, draft_probs=None, uniforms=None, stream=None) -> None:
+        io = self.io
+        io.target, io.draft_tokens = _ptr(target), _ptr(draft_tokens)
+        io.draft_probs, io.uniforms, io.reps = _ptr(draft_probs), _ptr(uniforms), _ptr(reps)
+        rc = lib.dpara_verify_select(C.byref(io), self.workspace.data_ptr(), self.workspace.numel(),
+                                     self.status.data_ptr(), _stream_ptr(stream))
+        if rc != OK:
+            raise DparaError(rc)
+
+
+def verify_select(target, draft_tokens, reps=None, *, mode: int = 0, draft_probs=None, uniforms=None, stream=None):
+    """Accepted length, bonus token, selected branch (dpara_verify_select).  Returns a dict of CUDA tensors."""
+    b, J, V = target.shape
+    block, hidden = (reps.shape[2], reps.shape[3]) if reps is not None else (1, 8)
+    plan = VerifyPlan(batch=b, n_boundaries=J, vocab=V, block=block, hidden=hidden, mode=mode, device=target.device)
+    plan(target=target, draft_tokens=draft_tokens, reps=reps, draft_probs=draft_probs, uniforms=uniforms, stream=stream)
+    return dict(accept_len=plan.accept_len, bonus=plan.bonus, gather_idx=plan.gather_idx, out_tokens=plan.out_tokens,
+                selected=plan.selected if reps is not None else None, status=plan.status)

@@ -1,0 +1,81 @@
+// C-ABI entry points of the draft call: argument validation, workspace sizing, kernel selection by shape.
+#include "attention_params.cuh"
+#include "layer.cuh"
+
+using namespace dpara;
+
+namespace dpara {
+
+static dpara_status validate_shape(const dpara_shape *s) {
+  if (!s) return DPARA_ERR_INVALID_ARG;
+  if (s->batch <= 0 || s->n_boundaries <= 0 || s->block <= 0 || s->n_q_heads <= 0 || s->n_kv_heads <= 0) return DPARA_ERR_INVALID_ARG;
+  if (s->n_spine < 0 || s->prefix_base < 0) return DPARA_ERR_INVALID_ARG;
+  if (s->boundary_lo < 0 || s->boundary_hi > s->n_boundaries || s->boundary_lo > s->boundary_hi) return DPARA_ERR_INVALID_ARG;
+  if (!(s->softmax_scale >= 0.f)) return DPARA_ERR_INVALID_ARG;
+  if (s->head_dim != 64 && s->head_dim != 128) return DPARA_ERR_UNSUPPORTED;
+  if (s->n_q_heads % s->n_kv_heads != 0) return DPARA_ERR_UNSUPPORTED;
+  if (s->n_q_heads / s->n_kv_heads > 16 || s->block > 64 || s->n_spine > 64) return DPARA_ERR_UNSUPPORTED;
+  return DPARA_OK;
+}
+
+static dpara_status validate_offsets(const dpara_shape *s, const int64_t *h) {
+  if (!h) return DPARA_ERR_INVALID_ARG;
+  if (h[0] < 0) return DPARA_ERR_INVALID_ARG;
+  for (int n = 0; n < s->batch; ++n)
+    if (h[n + 1] < h[n]) return DPARA_ERR_INVALID_ARG;
+  return DPARA_OK;
+}
+
+}  // namespace dpara
+
+extern "C" size_t dpara_draft_workspace_bytes(const dpara_shape *shape, const int64_t *host_ctx_offsets,
+                                              const dpara_layer_io *layer, int full_layer) {
+  if (validate_shape(shape) != DPARA_OK || validate_offsets(shape, host_ctx_offsets) != DPARA_OK) return 0;
+  size_t bytes = attention_workspace_bytes(shape, host_ctx_offsets);
+  if (full_layer) {
+    if (!layer) return 0;
+    bytes += layer_workspace_bytes(shape, layer);
+  }
+  return bytes;
+}
+
+extern "C" dpara_status dpara_draft_all_boundaries(const dpara_shape *shape, const dpara_attn_io *io,
+                                                   const dpara_layer_io *layer, void *workspace, size_t workspace_bytes,
+                                                   int32_t *status_word, void *stream) {
+  dpara_status s = validate_shape(shape);
+  if (s != DPARA_OK) return s;
+  if (!io) return DPARA_ERR_INVALID_ARG;
+  s = validate_offsets(shape, io->host_ctx_offsets);
+  if (s != DPARA_OK) return s;
+  if (!io->ctx_offsets) return DPARA_ERR_INVALID_ARG;
+  const bool has_ctx = io->host_ctx_offsets[shape->batch] > 0;
+  if (has_ctx && (!io->k_ctx || !io->v_ctx)) return DPARA_ERR_INVALID_ARG;
+  if (shape->n_spine > 0 && (!io->k_spine || !io->v_spine)) return DPARA_ERR_INVALID_ARG;
+  if ((io->k_blk == nullptr) != (io->v_blk == nullptr)) return DPARA_ERR_INVALID_ARG;
+  if (io->out_dtype != DPARA_BF16 && io->out_dtype != DPARA_F32) return DPARA_ERR_INVALID_ARG;
+  if (!aligned16(io->k_ctx) || !aligned16(io->v_ctx) || !aligned16(io->k_spine) || !aligned16(io->v_spine) ||
+      !aligned16(io->q) || !aligned16(io->k_blk) || !aligned16(io->v_blk) || !aligned16(io->out))
+    return DPARA_ERR_INVALID_ARG;
+  const size_t need = dpara_draft_workspace_bytes(shape, io->host_ctx_offsets, layer, layer != nullptr);
+  if (need > 0 && (!workspace || workspace_bytes < need || !aligned16(workspace))) return DPARA_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+
+  if (layer) return launch_layer(shape, io, layer, workspace, status_word, st);
+
+  if (!io->q || !io->out) return DPARA_ERR_INVALID_ARG;
+  return launch_attention(shape, io, workspace, status_word, st);
+}
+
+extern "C" const char *dpara_status_string(dpara_status s) {
+  switch (s) {
+    case DPARA_OK: return "ok";
+    case DPARA_ERR_INVALID_ARG: return "invalid argument";
+    case DPARA_ERR_UNSUPPORTED: return "unsupported shape";
+    case DPARA_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case DPARA_ERR_CUDA: return "CUDA call failed";
+    case DPARA_ERR_TIMEOUT: return "device-side wait timed out";
+  }
+  return "unknown status";
+}
+
+extern "C" int32_t dpara_version(void) { return 1000; }

@@ -1,0 +1,35 @@
+// Chooses the attention kernel for a shape and fills its parameters.
+#include <math.h>
+
+#include "layer.cuh"
+
+namespace dpara {
+
+void fill_attn_params(AttnParams &P, const dpara_shape *s, const dpara_attn_io *io, int32_t *status_word) {
+  P.q = static_cast<const uint16_t *>(io->q);
+  P.k_ctx = static_cast<const uint16_t *>(io->k_ctx);
+  P.v_ctx = static_cast<const uint16_t *>(io->v_ctx);
+  P.ctx_offsets = io->ctx_offsets;
+  P.k_spine = static_cast<const uint16_t *>(io->k_spine);
+  P.v_spine = static_cast<const uint16_t *>(io->v_spine);
+  P.k_blk = static_cast<const uint16_t *>(io->k_blk);
+  P.v_blk = static_cast<const uint16_t *>(io->v_blk);
+  P.out = io->out;
+  P.out_lse = io->out_lse;
+  P.out_f32 = io->out_dtype == DPARA_F32;
+  P.b = s->batch; P.J = s->n_boundaries; P.Bq = s->block; P.Hq = s->n_q_heads; P.Hkv = s->n_kv_heads;
+  P.D = s->head_dim; P.G = s->n_q_heads / s->n_kv_heads; P.S = s->n_spine; P.pb = s->prefix_base;
+  P.lo = s->boundary_lo; P.hi = s->boundary_hi;
+  P.scale = s->softmax_scale > 0.f ? s->softmax_scale : 1.0f / sqrtf((float)s->head_dim);
+  P.status_word = status_word;
+}
+
+size_t attention_workspace_bytes(const dpara_shape *, const int64_t *) { return 0; }
+
+dpara_status launch_attention(const dpara_shape *shape, const dpara_attn_io *io, void *, int32_t *status_word, cudaStream_t st) {
+  AttnParams P;
+  fill_attn_params(P, shape, io, status_word);
+  return launch_attention_simt(P, st);
+}
+
+}  // namespace dpara

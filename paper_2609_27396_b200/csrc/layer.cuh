@@ -1,0 +1,17 @@
+// Host-side entry points shared between the translation units of the draft call.
+#pragma once
+#include "attention_params.cuh"
+
+namespace dpara {
+
+// attention-only scratch (split-KV partials); 0 when the chosen kernel needs none
+size_t attention_workspace_bytes(const dpara_shape *shape, const int64_t *host_ctx_offsets);
+dpara_status launch_attention(const dpara_shape *shape, const dpara_attn_io *io, void *workspace, int32_t *status_word,
+                              cudaStream_t st);
+
+// full backbone block around the attention
+size_t layer_workspace_bytes(const dpara_shape *shape, const dpara_layer_io *layer);
+dpara_status launch_layer(const dpara_shape *shape, const dpara_attn_io *io, const dpara_layer_io *layer, void *workspace,
+                          int32_t *status_word, cudaStream_t st);
+
+}  // namespace dpara

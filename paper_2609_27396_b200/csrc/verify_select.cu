@@ -1,0 +1,438 @@
+// Verification outcome + branch selection (Alg. 1 lines 2-3; Sec. 2.1; App. C).
+//
+// Both modes are ONE launch: the vocabulary work is spread over the whole GPU (CTAs over
+// (request row, vocabulary chunk), 16-byte streaming loads), partial results meet in a small
+// workspace, and the last CTA to finish a request does that request's position scan, writes
+// (accept_len, bonus, out_tokens) and gathers the selected branch's representation.
+// No CTA ever waits for another: "last" is decided by an atomic ticket.
+#include "common.cuh"
+
+namespace dpara {
+
+constexpr int kVsThreads = 256;
+constexpr int kGreedyChunk = 8192;  // floats per CTA: 8 x 16 B in flight per thread
+constexpr int kSampChunk = 4096;    // floats per CTA and per row
+constexpr int kMaxJ = 64;
+
+// Monotone map float -> uint32 (a < b  <=>  key(a) < key(b)), -0 folded onto +0, NaN -> 0 (below -inf).
+__device__ __forceinline__ uint32_t order_key(float f) {
+  f = __fadd_rn(f, 0.0f);
+  uint32_t u = __float_as_uint(f);
+  uint32_t k = u ^ (((uint32_t)((int32_t)u >> 31)) | 0x80000000u);
+  return (f != f) ? 0u : k;
+}
+
+__device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    unsigned long long t = __shfl_xor_sync(0xffffffffu, v, o);
+    v = t > v ? t : v;
+  }
+  return v;
+}
+
+__device__ __forceinline__ unsigned long long warp_sum_u64(unsigned long long v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// Copy of the selected branch: reps[n][r] -> selected[n], `bytes` per request.
+__device__ __forceinline__ void gather_branch(const uint8_t *__restrict__ reps, uint8_t *__restrict__ selected, int n, int J,
+                                              int r, size_t bytes, int tid, int nthreads) {
+  const uint8_t *src = reps + ((size_t)n * J + r) * bytes;
+  uint8_t *dst = selected + (size_t)n * bytes;
+  if ((bytes & 15) == 0 && ((reinterpret_cast<uintptr_t>(src) | reinterpret_cast<uintptr_t>(dst)) & 15) == 0) {
+    const uint4 *s = reinterpret_cast<const uint4 *>(src);
+    uint4 *d = reinterpret_cast<uint4 *>(dst);
+    size_t nv = bytes >> 4;
+    for (size_t i = tid; i < nv; i += nthreads) d[i] = __ldg(s + i);
+  } else {
+    for (size_t i = tid; i < bytes; i += nthreads) dst[i] = src[i];
+  }
+}
+
+struct VerifyParams {
+  const float *target;
+  const float *draft_probs;
+  const int32_t *tokens;
+  const float *uniforms;
+  const uint8_t *reps;
+  int32_t *accept_len, *bonus, *gather_idx, *out_tokens;
+  uint8_t *selected;
+  int32_t *status_word;
+  unsigned long long *ws64;  // greedy: keys[b*J]; sampling: chunk sums [b][nchunks][2]
+  unsigned int *counters;    // [b], zeroed before the launch
+  int J, V, nchunks, vec_ok;
+  size_t rep_bytes;  // Bq * hidden * 2
+};
+
+__device__ __forceinline__ void write_result(const VerifyParams &P, int n, int r, int tok, bool bad) {
+  P.accept_len[n] = r;
+  P.bonus[n] = tok;
+  P.gather_idx[n] = r;
+  if (P.out_tokens) {
+    for (int i = 0; i < P.J; ++i)
+      P.out_tokens[(size_t)n * P.J + i] = i < r ? P.tokens[(size_t)n * (P.J - 1) + i] : (i == r ? tok : -1);
+  }
+  if (bad && P.status_word) atomicOr(reinterpret_cast<unsigned int *>(P.status_word), DPARA_STATUS_BAD_TOKEN);
+}
+
+// ------------------------------------------------------------------------------------------ greedy
+__global__ void __launch_bounds__(kVsThreads) verify_greedy_kernel(const VerifyParams P) {
+  const int tid = threadIdx.x;
+  const int row = blockIdx.y;  // n * J + i
+  const int n = row / P.J;
+  const float *__restrict__ p = P.target + (size_t)row * P.V;
+  const int base = blockIdx.x * kGreedyChunk;
+  const int end = min(P.V, base + kGreedyChunk);
+
+  uint32_t bk = 0, bi = 0xffffffffu;  // best key / its index; strict '>' keeps the lowest index
+  if (P.vec_ok) {
+    float4 v[8];
+#pragma unroll
+    for (int it = 0; it < 8; ++it) {
+      int idx = base + (it * kVsThreads + tid) * 4;
+      v[it] = idx < end ? __ldcs(reinterpret_cast<const float4 *>(p + idx)) : make_float4(0, 0, 0, 0);
+    }
+#pragma unroll
+    for (int it = 0; it < 8; ++it) {
+      int idx = base + (it * kVsThreads + tid) * 4;
+      if (idx < end) {
+        uint32_t k;
+        k = order_key(v[it].x); if (k > bk) { bk = k; bi = idx; }
+        k = order_key(v[it].y); if (k > bk) { bk = k; bi = idx + 1; }
+        k = order_key(v[it].z); if (k > bk) { bk = k; bi = idx + 2; }
+        k = order_key(v[it].w); if (k > bk) { bk = k; bi = idx + 3; }
+      }
+    }
+  } else {
+    for (int idx = base + tid; idx < end; idx += kVsThreads) {
+      uint32_t k = order_key(__ldcs(p + idx));
+      if (k > bk) { bk = k; bi = idx; }
+    }
+  }
+  unsigned long long key = ((unsigned long long)bk << 32) | (unsigned long long)(0xffffffffu - bi);
+  key = warp_max_u64(key);
+  __shared__ unsigned long long s_k[kVsThreads / 32];
+  __shared__ int s_flag;
+  if ((tid & 31) == 0) s_k[tid >> 5] = key;
+  __syncthreads();
+  if (tid == 0) {
+    unsigned long long m = s_k[0];
+#pragma unroll
+    for (int w = 1; w < kVsThreads / 32; ++w) m = s_k[w] > m ? s_k[w] : m;
+    if (m) atomicMax(P.ws64 + row, m);
+    __threadfence();
+    unsigned int t = atomicAdd(P.counters + n, 1u);
+    s_flag = (t == (unsigned int)(P.J * P.nchunks) - 1u);
+  }
+  __syncthreads();
+  if (!s_flag) return;
+
+  // ---- last CTA of request n: position scan, outputs, gather
+  __threadfence();
+  __shared__ int s_a[kMaxJ];
+  __shared__ int s_r;
+  if (tid < P.J) {
+    unsigned long long k = __ldcg(P.ws64 + (size_t)n * P.J + tid);
+    s_a[tid] = k == 0ull ? 0 : (int)(0xffffffffu - (uint32_t)(k & 0xffffffffull));  // all-NaN row -> 0
+  }
+  __syncthreads();
+  if (tid == 0) {
+    int r = 0;
+    bool bad = false;
+    while (r < P.J - 1) {
+      int t = P.tokens[(size_t)n * (P.J - 1) + r];
+      if (t < 0 || t >= P.V) { bad = true; break; }
+      if (t != s_a[r]) break;
+      ++r;
+    }
+    s_r = r;
+    write_result(P, n, r, s_a[r], bad);
+  }
+  __syncthreads();
+  if (P.reps) gather_branch(P.reps, P.selected, n, P.J, s_r, P.rep_bytes, tid, kVsThreads);
+}
+
+// ------------------------------------------------------------------------------------------ sampling
+__device__ __forceinline__ unsigned long long fx_weight(float d) {
+  d = d > 0.0f ? d : 0.0f;  // negatives and NaN carry no weight
+  return __float2ull_rz(d * 4294967296.0f);
+}
+
+// primary weight (residual, or p itself when no draft was rejected) and fallback weight (p)
+__device__ __forceinline__ void weights_of(float p, float q, bool residual, unsigned long long &w0, unsigned long long &w1) {
+  w1 = fx_weight(p);
+  w0 = residual ? fx_weight(__fsub_rn(p, q)) : w1;
+}
+
+__global__ void __launch_bounds__(kVsThreads) verify_sampling_kernel(const VerifyParams P) {
+  const int tid = threadIdx.x;
+  const int n = blockIdx.y;
+  const int c = blockIdx.x;
+  const int g = P.J - 1;
+  __shared__ int s_r, s_bad, s_flag;
+  __shared__ unsigned long long s_w[2][kVsThreads / 32];
+
+  // accepted length: every CTA of the request repeats this 2*gamma-scalar scan (L2 hits)
+  if (tid < 32) {
+    unsigned int rej = 0, badm = 0;
+    for (int i0 = 0; i0 < g; i0 += 32) {
+      int i = i0 + tid;
+      bool reject = false, bad = false;
+      if (i < g) {
+        int t = P.tokens[(size_t)n * g + i];
+        if (t < 0 || t >= P.V) {
+          reject = bad = true;
+        } else {
+          float qv = P.draft_probs[((size_t)n * g + i) * P.V + t];
+          float pv = P.target[((size_t)n * P.J + i) * P.V + t];
+          float u = P.uniforms[(size_t)n * P.J + i];
+          reject = !(__fmul_rn(u, qv) < pv);
+        }
+      }
+      rej = __ballot_sync(0xffffffffu, reject);
+      badm = __ballot_sync(0xffffffffu, bad);
+      if (rej) {
+        if (tid == 0) {
+          int f = __ffs(rej) - 1;
+          s_r = i0 + f;
+          s_bad = (badm >> f) & 1u;
+        }
+        break;
+      }
+    }
+    if (!rej && tid == 0) { s_r = g; s_bad = 0; }
+  }
+  __syncthreads();
+  const int r = s_r;
+  const bool residual = r < g;
+  const float *__restrict__ prow = P.target + ((size_t)n * P.J + r) * P.V;
+  const float *__restrict__ qrow = residual ? P.draft_probs + ((size_t)n * g + r) * P.V : prow;
+
+  // chunk sums of both weightings
+  const int base = c * kSampChunk;
+  const int end = min(P.V, base + kSampChunk);
+  unsigned long long a0 = 0, a1 = 0;
+  if (P.vec_ok) {
+#pragma unroll
+    for (int it = 0; it < kSampChunk / (kVsThreads * 4); ++it) {
+      int idx = base + (it * kVsThreads + tid) * 4;
+      if (idx < end) {
+        float4 pv = __ldg(reinterpret_cast<const float4 *>(prow + idx));
+        float4 qv = residual ? __ldg(reinterpret_cast<const float4 *>(qrow + idx)) : pv;
+        unsigned long long w0, w1;
+        weights_of(pv.x, qv.x, residual, w0, w1); a0 += w0; a1 += w1;
+        weights_of(pv.y, qv.y, residual, w0, w1); a0 += w0; a1 += w1;
+        weights_of(pv.z, qv.z, residual, w0, w1); a0 += w0; a1 += w1;
+        weights_of(pv.w, qv.w, residual, w0, w1); a0 += w0; a1 += w1;
+      }
+    }
+  } else {
+    for (int idx = base + tid; idx < end; idx += kVsThreads) {
+      unsigned long long w0, w1;
+      weights_of(prow[idx], qrow[idx], residual, w0, w1);
+      a0 += w0; a1 += w1;
+    }
+  }
+  a0 = warp_sum_u64(a0);
+  a1 = warp_sum_u64(a1);
+  if ((tid & 31) == 0) { s_w[0][tid >> 5] = a0; s_w[1][tid >> 5] = a1; }
+  __syncthreads();
+  if (tid == 0) {
+    unsigned long long t0 = 0, t1 = 0;
+#pragma unroll
+    for (int w = 0; w < kVsThreads / 32; ++w) { t0 += s_w[0][w]; t1 += s_w[1][w]; }
+    unsigned long long *cs = P.ws64 + ((size_t)n * P.nchunks + c) * 2;
+    __stcg(cs, t0);
+    __stcg(cs + 1, t1);
+    __threadfence();
+    unsigned int t = atomicAdd(P.counters + n, 1u);
+    s_flag = (t == (unsigned int)P.nchunks - 1u);
+  }
+  __syncthreads();
+  if (!s_flag) return;
+
+  // ---- last CTA of request n: total weight, threshold, locate the crossing
+  __threadfence();
+  __shared__ unsigned long long s_T, s_basepref;
+  __shared__ int s_chunk, s_which, s_tok;
+  if (tid == 0) {
+    unsigned long long W0 = 0, W1 = 0;
+    for (int k = 0; k < P.nchunks; ++k) {
+      W0 += __ldcg(P.ws64 + ((size_t)n * P.nchunks + k) * 2);
+      W1 += __ldcg(P.ws64 + ((size_t)n * P.nchunks + k) * 2 + 1);
+    }
+    int which = W0 ? 0 : (W1 ? 1 : 2);
+    s_which = which;
+    s_tok = 0;
+    s_chunk = 0;
+    if (which < 2) {
+      unsigned long long Wt = which ? W1 : W0;
+      unsigned int m = __float2uint_rn(P.uniforms[(size_t)n * P.J + g] * 16777216.0f);
+      unsigned long long lo = (unsigned long long)m * Wt;  // low 64 bits
+      unsigned long long hi = __umul64hi((unsigned long long)m, Wt);
+      unsigned long long T = (hi << 40) | (lo >> 24);  // (m * W) >> 24, m < 2^24 so it fits
+      unsigned long long pref = 0;
+      int k = 0;
+      for (; k < P.nchunks - 1; ++k) {
+        unsigned long long s = __ldcg(P.ws64 + ((size_t)n * P.nchunks + k) * 2 + which);
+        if (pref + s > T) break;
+        pref += s;
+      }
+      s_chunk = k;
+      s_T = T;
+      s_basepref = pref;
+    }
+  }
+  __syncthreads();
+  const int which = s_which;
+  if (which < 2) {
+    // thread t owns elements [cb + 16 t, cb + 16 t + 16) of the crossing chunk
+    const int cb = s_chunk * kSampChunk;
+    const int per = kSampChunk / kVsThreads;
+    unsigned long long w[kSampChunk / kVsThreads];
+    unsigned long long loc = 0;
+#pragma unroll
+    for (int e = 0; e < per; ++e) {
+      int idx = cb + tid * per + e;
+      unsigned long long w0 = 0, w1 = 0;
+      if (idx < P.V) weights_of(prow[idx], qrow[idx], residual, w0, w1);
+      w[e] = which ? w1 : w0;
+      loc += w[e];
+    }
+    // block exclusive scan of loc
+    unsigned long long inc = loc;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      unsigned long long t = __shfl_up_sync(0xffffffffu, inc, o);
+      if ((tid & 31) >= o) inc += t;
+    }
+    if ((tid & 31) == 31) s_w[0][tid >> 5] = inc;
+    __syncthreads();
+    unsigned long long woff = 0;
+    for (int k = 0; k < (tid >> 5); ++k) woff += s_w[0][k];
+    unsigned long long excl = s_basepref + woff + inc - loc;
+    const unsigned long long T = s_T;
+    if (excl <= T && excl + loc > T) {  // exactly one thread
+      unsigned long long acc = excl;
+      int tok = cb + tid * per;
+#pragma unroll
+      for (int e = 0; e < per; ++e) {
+        acc += w[e];
+        if (acc > T) { tok = cb + tid * per + e; break; }
+      }
+      s_tok = tok;
+    }
+    __syncthreads();
+  } else {
+    // no weight anywhere in p_r: lowest-index maximum of the row
+    uint32_t bk = 0, bi = 0xffffffffu;
+    for (int idx = tid; idx < P.V; idx += kVsThreads) {
+      uint32_t k = order_key(prow[idx]);
+      if (k > bk) { bk = k; bi = idx; }
+    }
+    unsigned long long key = warp_max_u64(((unsigned long long)bk << 32) | (unsigned long long)(0xffffffffu - bi));
+    if ((tid & 31) == 0) s_w[0][tid >> 5] = key;
+    __syncthreads();
+    if (tid == 0) {
+      unsigned long long m = 0;
+      for (int k = 0; k < kVsThreads / 32; ++k) m = s_w[0][k] > m ? s_w[0][k] : m;
+      s_tok = m == 0ull ? 0 : (int)(0xffffffffu - (uint32_t)(m & 0xffffffffull));
+    }
+    __syncthreads();
+  }
+  if (tid == 0) write_result(P, n, r, s_tok, s_bad != 0);
+  if (P.reps) gather_branch(P.reps, P.selected, n, P.J, r, P.rep_bytes, tid, kVsThreads);
+}
+
+static int chunks_of(const dpara_verify_io *io) {
+  int ch = io->mode == 0 ? kGreedyChunk : kSampChunk;
+  return (io->vocab + ch - 1) / ch;
+}
+
+// workspace: [64-bit area][counters]
+static size_t ws64_count(const dpara_verify_io *io) {
+  return io->mode == 0 ? (size_t)io->batch * io->n_boundaries : (size_t)io->batch * chunks_of(io) * 2;
+}
+
+static dpara_status validate_dims(const dpara_verify_io *io) {
+  if (!io) return DPARA_ERR_INVALID_ARG;
+  if (io->batch <= 0 || io->n_boundaries <= 0 || io->vocab <= 0) return DPARA_ERR_INVALID_ARG;
+  if (io->mode != 0 && io->mode != 1) return DPARA_ERR_INVALID_ARG;
+  if (io->n_boundaries > kMaxJ) return DPARA_ERR_UNSUPPORTED;
+  if (io->batch > 65535) return DPARA_ERR_UNSUPPORTED;
+  if ((long long)io->batch * io->n_boundaries > 65535 && io->mode == 0) return DPARA_ERR_UNSUPPORTED;
+  return DPARA_OK;
+}
+
+static dpara_status validate_verify(const dpara_verify_io *io) {
+  dpara_status s = validate_dims(io);
+  if (s != DPARA_OK) return s;
+  if (!io->target || !io->accept_len || !io->bonus || !io->gather_idx) return DPARA_ERR_INVALID_ARG;
+  if (io->n_boundaries > 1 && !io->draft_tokens) return DPARA_ERR_INVALID_ARG;
+  if (io->mode == 1 && (!io->uniforms || (io->n_boundaries > 1 && !io->draft_probs))) return DPARA_ERR_INVALID_ARG;
+  if (io->reps) {
+    if (!io->selected || io->block <= 0 || io->hidden <= 0) return DPARA_ERR_INVALID_ARG;
+  }
+  return DPARA_OK;
+}
+
+}  // namespace dpara
+
+using namespace dpara;
+
+extern "C" size_t dpara_verify_workspace_bytes(const dpara_verify_io *io) {
+  if (validate_dims(io) != DPARA_OK) return 0;
+  return align_up(ws64_count(io) * 8, 256) + align_up((size_t)io->batch * 4, 256);
+}
+
+namespace dpara {
+// Shared by the public entry point; `ws` must hold dpara_verify_workspace_bytes(io) bytes.
+dpara_status launch_verify(const dpara_verify_io *io, void *ws, int32_t *status_word, cudaStream_t st) {
+  VerifyParams P;
+  P.target = io->target;
+  P.draft_probs = io->draft_probs;
+  P.tokens = io->draft_tokens;
+  P.uniforms = io->uniforms;
+  P.reps = static_cast<const uint8_t *>(io->reps);
+  P.accept_len = io->accept_len;
+  P.bonus = io->bonus;
+  P.gather_idx = io->gather_idx;
+  P.out_tokens = io->out_tokens;
+  P.selected = static_cast<uint8_t *>(io->selected);
+  P.status_word = status_word;
+  P.J = io->n_boundaries;
+  P.V = io->vocab;
+  P.nchunks = chunks_of(io);
+  P.rep_bytes = (size_t)io->block * io->hidden * 2;
+  size_t n64 = ws64_count(io);
+  size_t cnt_off = align_up(n64 * 8, 256);
+  P.ws64 = static_cast<unsigned long long *>(ws);
+  P.counters = reinterpret_cast<unsigned int *>(static_cast<uint8_t *>(ws) + cnt_off);
+  bool vec = (io->vocab % 4 == 0) && aligned16(io->target) && (io->mode == 0 || io->n_boundaries == 1 || aligned16(io->draft_probs));
+  P.vec_ok = vec ? 1 : 0;
+  // greedy needs keys and counters at zero; sampling only the counters
+  if (io->mode == 0) {
+    if (cudaMemsetAsync(ws, 0, cnt_off + (size_t)io->batch * 4, st) != cudaSuccess) return DPARA_ERR_CUDA;
+    dim3 grid(P.nchunks, io->batch * io->n_boundaries);
+    verify_greedy_kernel<<<grid, kVsThreads, 0, st>>>(P);
+  } else {
+    if (cudaMemsetAsync(P.counters, 0, (size_t)io->batch * 4, st) != cudaSuccess) return DPARA_ERR_CUDA;
+    dim3 grid(P.nchunks, io->batch);
+    verify_sampling_kernel<<<grid, kVsThreads, 0, st>>>(P);
+  }
+  DPARA_CHECK_LAUNCH();
+  return DPARA_OK;
+}
+}  // namespace dpara
+
+extern "C" dpara_status dpara_verify_select(const dpara_verify_io *io, void *workspace, size_t workspace_bytes,
+                                            int32_t *status_word, void *stream) {
+  dpara_status s = validate_verify(io);
+  if (s != DPARA_OK) return s;
+  size_t need = dpara_verify_workspace_bytes(io);
+  if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 7u)) return DPARA_ERR_WORKSPACE;
+  return launch_verify(io, workspace, status_word, static_cast<cudaStream_t>(stream));
+}

@@ -1,0 +1,99 @@
+"""GPU parity of the all-boundary attention against the oracle: max |delta| <= 1e-2 on representations
+(the stated bound for bf16 inputs with fp32 accumulation); fp32 outputs are held to a tighter bound that
+the arithmetic supports (probabilities rounded to bf16 before the PV product: relative 2^-9 per term)."""
+import numpy as np
+import pytest
+import torch
+
+import workloads as W
+from oracle import attention as OA
+
+pytestmark = pytest.mark.gpu
+
+TOL_BF16_OUT = 1e-2     # spec bound on representations
+TOL_F32_OUT = 4e-3      # fp32 output: only the internal bf16 rounding of probabilities remains
+
+
+def _oracle(inp, with_blk=True, **kw):
+    return OA.draft_all_boundaries(inp.q, inp.k_ctx, inp.v_ctx, inp.ctx_offsets, inp.k_spine, inp.v_spine,
+                                   inp.k_blk if with_blk else None, inp.v_blk if with_blk else None,
+                                   prefix_base=inp.shape.prefix_base, **kw)
+
+
+def _compare(inp, with_blk=True, lo=0, hi=None, scale=0.0):
+    from gpu_util import run_attention
+    ref, ref_lse = _oracle(inp, with_blk, boundary_lo=lo, boundary_hi=hi, scale=scale)
+    out, lse, status = run_attention(inp, out_dtype=torch.float32, want_lse=True, with_blk=with_blk,
+                                     boundary_lo=lo, boundary_hi=hi, softmax_scale=scale)
+    d = np.abs(out.cpu().numpy().astype(np.float64) - ref).max()
+    assert d <= TOL_F32_OUT, d
+    l = lse.cpu().numpy().astype(np.float64)
+    fin = np.isfinite(ref_lse)
+    assert np.array_equal(np.isfinite(l), fin)
+    assert np.abs(l[fin] - ref_lse[fin]).max() < 2e-3
+    out16, status = run_attention(inp, out_dtype=torch.bfloat16, want_lse=False, with_blk=with_blk,
+                                  boundary_lo=lo, boundary_hi=hi, softmax_scale=scale)
+    d16 = np.abs(out16.float().cpu().numpy().astype(np.float64) - ref).max()
+    assert d16 <= TOL_BF16_OUT, d16
+    assert int(status.item()) == 0
+    return d, d16
+
+
+def test_cfg1_tiny():
+    w = W.workload(1)
+    _compare(W.make_attn_inputs(w.attn, w.seed))
+
+
+@pytest.mark.parametrize("shape", [
+    W.AttnShape((300,), 8, 2, 128, 8, 8),                 # cfg2-like, several 128-key tiles + ragged tail
+    W.AttnShape((129, 1, 257, 64), 10, 2, 128, 4, 16),    # group size 5 (cfg3-like), ragged batch
+    W.AttnShape((200, 77), 4, 4, 64, 5, 4),               # no grouping, D = 64
+    W.AttnShape((0, 5), 4, 2, 64, 3, 2),                  # an empty context
+    W.AttnShape((140,), 16, 1, 128, 3, 3),                # one KV head, group 16, odd block
+    W.AttnShape((520,), 8, 2, 128, 16, 16, 1, 16),        # 16 boundaries x 16 slots
+])
+def test_shapes(shape):
+    _compare(W.make_attn_inputs(shape, 77))
+
+
+def test_prefix_base_zero_and_no_block_keys():
+    sh = W.AttnShape((150, 0), 4, 2, 64, 4, 3, 0)
+    inp = W.make_attn_inputs(sh, 5)
+    _compare(inp)
+    _compare(inp, with_blk=False)      # request 1, boundary 0: no visible key at all -> zeros, lse = -inf
+
+
+def test_boundary_range_and_scale():
+    sh = W.AttnShape((260,), 8, 2, 128, 6, 4)
+    inp = W.make_attn_inputs(sh, 6)
+    _compare(inp, lo=5, hi=6)          # the single-boundary (conventional) draft step
+    _compare(inp, lo=2, hi=4, scale=0.05)
+
+
+def test_cfg2_full_size():
+    w = W.workload(2)
+    _compare(W.make_attn_inputs(w.attn, w.seed))
+
+
+def test_cfg3_full_size_sampled_rows():
+    """Full b = 16 ragged batch in the launch configuration the benchmark times; the oracle checks a
+    seeded sample of query rows that covers every request and boundary."""
+    from gpu_util import dev_bf16
+    import paper_2609_27396_b200 as dp
+    w = W.workload(3)
+    inp = W.make_attn_inputs(w.attn, w.seed)
+    sh = inp.shape
+    out, status = dp.draft_all_boundaries(dev_bf16(inp.q), dev_bf16(inp.k_ctx), dev_bf16(inp.v_ctx),
+                                          [int(x) for x in inp.ctx_offsets], dev_bf16(inp.k_spine), dev_bf16(inp.v_spine),
+                                          dev_bf16(inp.k_blk), dev_bf16(inp.v_blk), out_dtype=torch.bfloat16)
+    torch.cuda.synchronize()
+    rng = np.random.default_rng(1)
+    rows = [(n, j, int(rng.integers(sh.block)), int(rng.integers(sh.n_q_heads)))
+            for n in range(sh.batch) for j in range(sh.n_boundaries)]
+    ref = OA.draft_rows(inp.q, inp.k_ctx, inp.v_ctx, inp.ctx_offsets, inp.k_spine, inp.v_spine, inp.k_blk, inp.v_blk, rows)
+    o = out.float().cpu().numpy()
+    got = np.stack([o[n, j, i, h] for (n, j, i, h) in rows]).astype(np.float64)
+    assert np.abs(got - ref).max() <= TOL_BF16_OUT
+    assert int(status.item()) == 0
+    # invariant at any size: rows are convex combinations, so |out| <= max |v| seen by that KV head
+    assert np.isfinite(o).all()

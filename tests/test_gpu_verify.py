@@ -1,0 +1,121 @@
+"""GPU parity of dpara_verify_select against the oracle: bit-exact integers and bit-exact gathered rows."""
+import numpy as np
+import pytest
+import torch
+
+import workloads as W
+from oracle import verify as OV
+
+pytestmark = pytest.mark.gpu
+
+
+def _check(v, mode):
+    from gpu_util import run_verify, check_verify
+    res = run_verify(v, mode)
+    if mode == 0:
+        ref = OV.verify_greedy(v.target, v.draft_tokens, v.reps)
+    else:
+        ref = OV.verify_sampling(v.target, v.draft_probs, v.draft_tokens, v.uniforms, v.reps)
+    check_verify(res, ref)
+    return ref
+
+
+@pytest.mark.parametrize("V", [1000, 1001, 8192, 8196, 40000, 151936])
+def test_greedy_parity_sizes(V):
+    sh = W.VerifyShape(5, 6, V, 4, 256, "greedy", 0.7, 1.0)
+    v = W.make_verify_inputs(sh, 100 + V, force_full=[0], force_zero=[1])
+    ref = _check(v, 0)
+    assert ref["accept_len"][0] == 5 and ref["accept_len"][1] == 0
+
+
+def test_greedy_cfg1_and_cfg2():
+    for idx in (1, 2):
+        w = W.workload(idx)
+        _check(W.make_verify_inputs(w.verify, w.seed), 0)
+
+
+def test_greedy_cfg3_full_size():
+    w = W.workload(3)
+    v = W.make_verify_inputs(w.verify, w.seed, force_full=[3], force_zero=[5])
+    ref = _check(v, 0)
+    assert len(set(ref["accept_len"].tolist())) >= 4
+
+
+def test_greedy_ties_and_specials():
+    """Duplicate maxima inside one 16-byte vector, across threads, across CTAs (chunks), at the first and
+    last vocabulary index; -0/+0; NaN and -inf rows."""
+    V, J = 20000, 8
+    rng = np.random.default_rng(3)
+    logits = rng.standard_normal((2, J, V)).astype(np.float32)
+    big = np.float32(50.0)
+    logits[0, 0, [5, 6]] = big                    # same float4
+    logits[0, 1, [100, 9000]] = big               # different CTAs (chunk = 8192)
+    logits[0, 2, [V - 1, 3]] = big                # last index vs early index
+    logits[0, 3, [0, V - 1]] = big                # first and last
+    logits[0, 4, :] = -np.inf                     # all -inf -> 0
+    logits[0, 5, :] = np.nan                      # all NaN -> 0
+    logits[0, 6, :] = np.nan
+    logits[0, 6, 777] = -np.inf                   # -inf beats NaN
+    logits[0, 7, :] = -1.0
+    logits[0, 7, 4097] = -0.0
+    logits[0, 7, 12000] = 0.0                     # -0 == +0: lower index wins
+    logits[1, 0, 8191] = big
+    logits[1, 0, 8192] = big                      # chunk edge
+    a0 = [5, 100, 3, 0, 0, 0, 777, 4097]
+    toks = np.zeros((2, J - 1), np.int32)
+    toks[0] = a0[:J - 1]
+    toks[1] = -5                                   # out of range -> rejected, status bit
+    v = W.VerifyInputs(W.VerifyShape(2, J, V, 2, 64), logits, toks, W.make_verify_inputs(W.VerifyShape(2, J, V, 2, 64), 1).reps)
+    ref = _check(v, 0)
+    assert ref["accept_len"][0] == J - 1 and ref["bonus"][0] == 4097
+    assert ref["accept_len"][1] == 0 and ref["bonus"][1] == 8191 and ref["status"] == 1
+
+
+def test_greedy_single_boundary_and_repeat():
+    from gpu_util import run_verify, check_verify
+    sh = W.VerifyShape(3, 1, 5000, 2, 64, "greedy", 0.5, 1.0)
+    v = W.make_verify_inputs(sh, 9)
+    ref = _check(v, 0)
+    assert np.all(ref["accept_len"] == 0)
+    # two runs give identical bits (no race on the ticket/atomic path)
+    sh = W.VerifyShape(8, 16, 30000, 4, 128, "greedy", 0.8, 2.0)
+    v = W.make_verify_inputs(sh, 10)
+    r1, r2 = run_verify(v, 0), run_verify(v, 0)
+    for k in ("accept_len", "bonus", "out_tokens", "selected"):
+        assert torch.equal(r1[k], r2[k])
+
+
+@pytest.mark.parametrize("V", [16, 1001, 4096, 5000, 151936])
+def test_sampling_parity_sizes(V):
+    sh = W.VerifyShape(6, 5, V, 4, 128, "sampling", 0.0, 3.0)
+    v = W.make_verify_inputs(sh, 200 + V, force_full=[2])
+    ref = _check(v, 1)
+    assert ref["accept_len"][2] == 4
+
+
+def test_sampling_cfg4_full_size():
+    w = W.workload(4)
+    v = W.make_verify_inputs(w.verify, w.seed, force_full=[1])
+    ref = _check(v, 1)
+    assert ref["accept_len"][1] == 15 and len(set(ref["accept_len"].tolist())) >= 3
+
+
+def test_sampling_fallbacks():
+    # rejected position with an empty residual -> p_r; all-zero target row -> lowest-index maximum;
+    # extreme uniforms; out-of-range token
+    V, J = 6000, 3
+    p = np.zeros((4, J, V), np.float32)
+    q = np.zeros((4, J - 1, V), np.float32)
+    p[:, :, 10] = 0.5; p[:, :, 4500] = 0.25
+    q[:, :, 10] = 0.5; q[:, :, 4500] = 0.5
+    toks = np.full((4, J - 1), 4500, np.int32)
+    u = np.full((4, J), 0.75, np.float32)
+    p[1, 0, :] = 0                                  # request 1: row 0 all zero -> rejected (0 < 0 false), argmax fallback
+    u[2, :] = 0.0                                   # request 2: u = 0 accepts while p > 0; bonus with m = 0
+    u[2, J - 1] = np.float32((2 ** 24 - 1) * 2.0 ** -24)
+    toks[3, 0] = V + 3                              # request 3: bad token
+    reps = W.make_verify_inputs(W.VerifyShape(4, J, V, 2, 64), 1).reps
+    v = W.VerifyInputs(W.VerifyShape(4, J, V, 2, 64, "sampling"), p, toks, reps, q, u)
+    ref = _check(v, 1)
+    assert ref["accept_len"].tolist() == [0, 0, 2, 0] and ref["bonus"][0] == 4500 and ref["bonus"][1] == 0
+    assert ref["bonus"][2] == 4500 and ref["status"] == 1
