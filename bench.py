@@ -1,0 +1,385 @@
+#!/usr/bin/env python
+"""Benchmark of the all-boundary draft step (one process per GPU).
+
+A step = one pass of the whole hot path over one synthetic batch: the all-boundary attention
+(dpara_draft_all_boundaries) followed by greedy verify/select with the fused branch gather
+(dpara_verify_select) on the attention's own output.  Default workload: the Qwen3-14B-shaped b = 16
+ragged batch (cfg3); the b = 1 Qwen3-8B-shaped step (cfg2) is timed as well and reported under "b1".
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload cfg3|cfg2]
+
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle on the host cores instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import workloads as W  # noqa: E402
+
+METRIC = "all_boundary_draft_step_us"
+L2_FLUSH_BYTES = 256 << 20
+
+
+# ----------------------------------------------------------------------------- algorithmic work
+def attention_flops(sh: W.AttnShape) -> float:
+    """4 * D flops per (query row, visible key): QK^T and PV."""
+    rows_per_boundary = sh.block * sh.n_q_heads
+    tot = 0.0
+    for L in sh.ctx_lens:
+        for j in range(sh.n_boundaries):
+            keys = L + min(j + sh.prefix_base, sh.spine) + sh.block
+            tot += 4.0 * sh.head_dim * rows_per_boundary * keys
+    return tot
+
+
+def attention_bytes(sh: W.AttnShape, out_bytes: int = 2) -> float:
+    """Every input read once, every output written once."""
+    kv = 2 * 2 * sh.n_kv_heads * sh.head_dim
+    b, J, Bq = sh.batch, sh.n_boundaries, sh.block
+    q = b * J * Bq * sh.n_q_heads * sh.head_dim
+    return sum(sh.ctx_lens) * kv + b * sh.spine * kv + b * J * Bq * kv + q * 2 + q * out_bytes
+
+
+def verify_bytes(v: W.VerifyShape) -> float:
+    gather = v.batch * v.block * v.hidden * 2
+    return v.batch * v.n_boundaries * v.vocab * 4 + 2 * gather
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return dict(hbm_gbs=d["hbm_gbs"], bf16_tflops=d["bf16_tflops"], bf16_tflops_sustained=d.get("bf16_tflops_sustained"),
+                    source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+# ----------------------------------------------------------------------------- clocks sampler
+class ClockSampler:
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.index), "-lms", "100"], stdout=subprocess.PIPE, text=True)
+            threading.Thread(target=self._pump, daemon=True).start()
+        except Exception:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        sm, mx, reasons = [], None, set()
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx = float(r[1])
+            except Exception:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        busy = [x for x in sm if mx and x > 0.5 * mx] or sm
+        return {"sm_mhz": statistics.median(busy) if busy else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# ----------------------------------------------------------------------------- the CUDA arm
+class StepRunner:
+    """Owns device-resident inputs, fixed plans and (for the end-to-end leg) pinned host copies."""
+
+    def __init__(self, wl: W.Workload, seed: int):
+        import torch
+        import paper_2609_27396_b200 as dp
+        self.torch, self.dp, self.wl = torch, dp, wl
+        a, v = wl.attn, wl.verify
+        self.inp = W.make_attn_inputs(a, seed)
+        self.ver = W.make_verify_inputs(v, seed, reps=np.zeros((1,), np.uint16))
+        bf = lambda bits: torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).view(torch.bfloat16)
+        i = self.inp
+        self.host = dict(q=bf(i.q), k_ctx=bf(i.k_ctx), v_ctx=bf(i.v_ctx), k_spine=bf(i.k_spine), v_spine=bf(i.v_spine),
+                         k_blk=bf(i.k_blk), v_blk=bf(i.v_blk), target=torch.from_numpy(self.ver.target),
+                         draft_tokens=torch.from_numpy(self.ver.draft_tokens))
+        self.dev = {k: t.cuda() for k, t in self.host.items()}
+        self.out = torch.zeros((a.batch, a.n_boundaries, a.block, a.n_q_heads, a.head_dim), dtype=torch.bfloat16, device="cuda")
+        self.plan = dp.DraftPlan(ctx_offsets=[int(x) for x in i.ctx_offsets], n_boundaries=a.n_boundaries, block=a.block,
+                                 n_q_heads=a.n_q_heads, n_kv_heads=a.n_kv_heads, head_dim=a.head_dim,
+                                 prefix_base=a.prefix_base, n_spine=a.spine)
+        self.plan1 = dp.DraftPlan(ctx_offsets=[int(x) for x in i.ctx_offsets], n_boundaries=a.n_boundaries, block=a.block,
+                                  n_q_heads=a.n_q_heads, n_kv_heads=a.n_kv_heads, head_dim=a.head_dim,
+                                  prefix_base=a.prefix_base, n_spine=a.spine, boundary_lo=a.n_boundaries - 1)
+        self.vplan = dp.VerifyPlan(batch=v.batch, n_boundaries=v.n_boundaries, vocab=v.vocab, block=v.block,
+                                   hidden=v.hidden, mode=0)
+        self.reps = self.out.view(a.batch, a.n_boundaries, a.block, a.hidden)
+        self.flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device="cuda")
+        self.pinned = None
+
+    def attention(self, plan=None, src=None):
+        d = src or self.dev
+        (plan or self.plan)(q=d["q"], k_ctx=d["k_ctx"], v_ctx=d["v_ctx"], k_spine=d["k_spine"], v_spine=d["v_spine"],
+                            k_blk=d["k_blk"], v_blk=d["v_blk"], out=self.out)
+
+    def verify(self, src=None):
+        d = src or self.dev
+        self.vplan(target=d["target"], draft_tokens=d["draft_tokens"], reps=self.reps)
+
+    def step(self):
+        self.attention()
+        self.verify()
+
+    def timed_steps(self, k: int, single_boundary: bool = False):
+        """k steps, each bracketed by CUDA events on the launching stream, L2 flushed in between.
+        Returns per-step (total_ms, attention_ms, verify_ms)."""
+        torch = self.torch
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(k)]
+        for s in range(k):
+            self.flush.zero_()
+            ev[s][0].record()
+            self.attention(self.plan1 if single_boundary else None)
+            ev[s][1].record()
+            if not single_boundary:
+                self.verify()
+            ev[s][2].record()
+        torch.cuda.synchronize()
+        return [(e[0].elapsed_time(e[2]), e[0].elapsed_time(e[1]), e[1].elapsed_time(e[2])) for e in ev]
+
+    # end to end: host (pinned) buffers in, results back on the host, copies inside the timed region
+    def setup_e2e(self):
+        torch = self.torch
+        self.pinned = {k: t.pin_memory() for k, t in self.host.items()}
+        self.stage = {k: torch.empty_like(t, device="cuda") for k, t in self.host.items()}
+        vp = self.vplan
+        self.res_host = {k: torch.empty_like(getattr(vp, k), device="cpu").pin_memory()
+                         for k in ("accept_len", "bonus", "gather_idx", "out_tokens", "selected")}
+        self.h2d_bytes = sum(t.numel() * t.element_size() for t in self.pinned.values())
+        self.d2h_bytes = sum(t.numel() * t.element_size() for t in self.res_host.values())
+
+    def e2e_steps(self, k: int):
+        torch = self.torch
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(k)]
+        for s in range(k):
+            self.flush.zero_()
+            ev[s][0].record()
+            for key, t in self.pinned.items():
+                self.stage[key].copy_(t, non_blocking=True)
+            self.attention(src=self.stage)
+            self.verify(src=self.stage)
+            for key, t in self.res_host.items():
+                t.copy_(getattr(self.vplan, key), non_blocking=True)
+            ev[s][1].record()
+        torch.cuda.synchronize()
+        return [e[0].elapsed_time(e[1]) for e in ev]
+
+
+# ----------------------------------------------------------------------------- the oracle arm (host cores)
+def oracle_sample(wl: W.Workload, seed: int, n_pairs: int, n_verify_req: int, inp=None, ver=None):
+    """Times the oracle, as it stands, on a bounded sample of the step: `n_pairs` (request, boundary)
+    attentions (all slots, all heads) and greedy verify/select of `n_verify_req` requests.  Returns
+    (seconds, estimated seconds for the full step, description)."""
+    from oracle import attention as OA
+    from oracle import verify as OV
+    a, v = wl.attn, wl.verify
+    inp = inp or W.make_attn_inputs(a, seed)
+    ver = ver or W.make_verify_inputs(v, seed)
+    rng = np.random.default_rng(seed)
+    budget_s = 15.0 if n_pairs <= 0 else None          # n_pairs <= 0: as many pairs as fit in ~15 s (at most all)
+    if n_pairs <= 0:
+        n_pairs = a.batch * a.n_boundaries
+    pairs = [(int(rng.integers(a.batch)), int(rng.integers(a.n_boundaries))) for _ in range(n_pairs)]
+    t0 = time.perf_counter()
+    flops = 0.0
+    done = 0
+    for (n, j) in pairs:
+        if budget_s is not None and done >= 4 and time.perf_counter() - t0 > budget_s:
+            break
+        done += 1
+        lo = int(inp.ctx_offsets[n]); hi = int(inp.ctx_offsets[n + 1])
+        sub_off = np.array([0, hi - lo], dtype=np.int64)
+        OA.draft_all_boundaries(inp.q[n:n + 1], inp.k_ctx[lo:hi], inp.v_ctx[lo:hi], sub_off, inp.k_spine[n:n + 1],
+                                inp.v_spine[n:n + 1], inp.k_blk[n:n + 1], inp.v_blk[n:n + 1], prefix_base=a.prefix_base,
+                                boundary_lo=j, boundary_hi=j + 1)
+        flops += 4.0 * a.head_dim * a.block * a.n_q_heads * ((hi - lo) + min(j + a.prefix_base, a.spine) + a.block)
+    t_att = time.perf_counter() - t0
+    nv = min(n_verify_req, v.batch)
+    t0 = time.perf_counter()
+    OV.verify_greedy(ver.target[:nv], ver.draft_tokens[:nv], ver.reps[:nv] if ver.reps.ndim == 4 else None)
+    t_ver = time.perf_counter() - t0
+    est = t_att * attention_flops(a) / max(flops, 1.0) + t_ver * v.batch / nv
+    desc = (f"{done} seeded (request, boundary) attentions of {a.batch * a.n_boundaries} + greedy verify of "
+            f"{nv}/{v.batch} requests; full-step time extrapolated by flops / requests")
+    return t_att + t_ver, est, desc
+
+
+def oracle_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        if n:
+            return int(max(n))
+    except Exception:
+        pass
+    return len(os.sched_getaffinity(0))
+
+
+# ----------------------------------------------------------------------------- main
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg3", choices=["cfg2", "cfg3"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    wl = W.workload({"cfg2": 2, "cfg3": 3}[args.workload])
+    cfg = {"workload": f"{wl.name}: b={wl.attn.batch}, ctx={'ragged U[512,4096] sum=' + str(sum(wl.attn.ctx_lens)) if wl.index == 3 else wl.attn.ctx_lens[0]}, "
+                       f"Hq/Hkv={wl.attn.n_q_heads}/{wl.attn.n_kv_heads}, D={wl.attn.head_dim}, boundaries={wl.attn.n_boundaries}, "
+                       f"block={wl.attn.block}, vocab={wl.verify.vocab}, hidden={wl.verify.hidden}; step = all-boundary attention + greedy verify/select",
+           "l2": f"{L2_FLUSH_BYTES >> 20} MiB flush write between timed steps", "parallelism": f"batch-sharded x{world} (no collective)"}
+
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        steps = max(1, min(args.steps, 3))
+        times, est = [], []
+        inp, ver = W.make_attn_inputs(wl.attn, wl.seed), W.make_verify_inputs(wl.verify, wl.seed)
+        for s in range(args.warmup and 1):
+            oracle_sample(wl, wl.seed, 1, 1, inp, ver)
+        for s in range(steps):
+            t, e, desc = oracle_sample(wl, wl.seed + s, 6, 2, inp, ver)
+            times.append(t); est.append(e)
+        us = statistics.mean(est) * 1e6
+        cores = oracle_threads()
+        print(json.dumps({"impl": "reference", "metric": METRIC, "value": us, "unit": "us", "n_gpus": args.gpus, "steps": steps,
+                          "warmup": 1 if args.warmup else 0, "ms_per_step": us / 1e3, "higher_is_better": False, "scaling": "weak",
+                          "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": cfg,
+                          "cpu_baseline": {"value": us, "unit": "us", "cores": cores, "kind": "oracle", "sample": desc},
+                          "e2e": {"value": us, "unit": "us", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
+        return
+
+    import torch
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    import paper_2609_27396_b200 as dp
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(x: float) -> float:
+        if dist is None:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    run = StepRunner(wl, wl.seed + 1000 * rank)
+    for _ in range(max(args.warmup, 3)):
+        run.step()
+    barrier()
+    launches0 = dp.lib.dpara_kernel_launches()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    per = run.timed_steps(args.steps)
+    barrier()
+    launches = dp.lib.dpara_kernel_launches() - launches0
+    # keep the GPU busy a little longer so that the 100 ms sampler sees clocks under this load
+    t_end = time.time() + 0.6
+    while rank == 0 and time.time() < t_end:
+        run.step()
+    torch.cuda.synchronize()
+    clocks = sampler.stop() if rank == 0 else None
+    total_ms = max_over_ranks(sum(p[0] for p in per))
+    att_ms = statistics.mean(p[1] for p in per)
+    ver_ms = statistics.mean(p[2] for p in per)
+    step_us = total_ms / args.steps * 1e3
+
+    # end to end through the public call with host buffers
+    run.setup_e2e()
+    run.e2e_steps(2)
+    barrier()
+    e2e = run.e2e_steps(max(3, min(args.steps, 10)))
+    barrier()
+    e2e_us = max_over_ranks(statistics.mean(e2e)) * 1e3
+
+    peaks = measured_peaks()
+    fl = attention_flops(wl.attn)
+    by = attention_bytes(wl.attn)
+    ach_tf = fl / (att_ms * 1e-3) / 1e12
+    ach_gb = by / (att_ms * 1e-3) / 1e9
+    traffic = None
+    tp = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(tp):
+        traffic = json.load(open(tp)).get(f"attention_{args.workload}")
+    roofline = {"kernel": "all-boundary attention", "bound": "tensor", "achieved": ach_tf, "peak": peaks["bf16_tflops"],
+                "unit": "TFLOP/s", "frac": ach_tf / peaks["bf16_tflops"], "traffic": traffic, "peak_source": peaks["source"] + " (burst)",
+                "hbm": {"achieved": ach_gb, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach_gb / peaks["hbm_gbs"],
+                        "note": "same launch against the HBM roofline (algorithmic bytes)"},
+                "algorithmic": {"flops": fl, "bytes": by, "us": att_ms * 1e3},
+                "verify_select": {"bound": "hbm", "achieved": verify_bytes(wl.verify) / (ver_ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
+                                  "unit": "GB/s", "frac": verify_bytes(wl.verify) / (ver_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                                  "us": ver_ms * 1e3, "bytes": verify_bytes(wl.verify)}}
+
+    out = {"metric": METRIC, "value": step_us, "unit": "us", "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+           "ms_per_step": step_us / 1e3, "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+           "data": "synthetic", "config": cfg, "clocks": clocks, "gpu_launches": int(launches),
+           "e2e": {"value": e2e_us, "unit": "us", "h2d_bytes_per_step": run.h2d_bytes, "d2h_bytes_per_step": run.d2h_bytes},
+           "roofline": roofline, "steps_per_s_all_gpus": world * 1e6 / step_us}
+
+    if rank == 0 and world == 1:
+        # the b = 1 step (cfg2) and the single-boundary (conventional) draft step beside it
+        w2 = W.workload(2)
+        r2 = StepRunner(w2, w2.seed)
+        for _ in range(5):
+            r2.step(); r2.attention(r2.plan1)
+        p2 = r2.timed_steps(max(args.steps, 20))
+        s2 = r2.timed_steps(max(args.steps, 20), single_boundary=True)
+        a2 = statistics.median(p[1] for p in p2) * 1e3
+        out["b1"] = {"workload": w2.name, "step_us": statistics.median(p[0] for p in p2) * 1e3, "attention_us": a2,
+                     "verify_select_us": statistics.median(p[2] for p in p2) * 1e3,
+                     "single_boundary_attention_us": statistics.median(p[1] for p in s2) * 1e3,
+                     "all_over_single": a2 / (statistics.median(p[1] for p in s2) * 1e3), "allowance": w2.attn.n_boundaries,
+                     "attention_gbs": attention_bytes(w2.attn) / (a2 * 1e-6) / 1e9, "attention_tflops": attention_flops(w2.attn) / (a2 * 1e-6) / 1e12}
+        del r2
+        if not args.no_cpu_baseline:
+            t, est, desc = oracle_sample(wl, wl.seed, 0, wl.verify.batch, run.inp, run.ver)
+            out["cpu_baseline"] = {"value": est * 1e6, "unit": "us", "cores": oracle_threads(), "kind": "oracle", "sample": desc,
+                                   "sample_seconds": t}
+    if rank == 0:
+        print(json.dumps(out))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

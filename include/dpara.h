@@ -167,6 +167,10 @@ const char *dpara_status_string(dpara_status s);
 /* Library/ABI version: major * 1000 + minor. */
 int32_t dpara_version(void);
 
+/* Number of kernels this library has launched in this process so far (all calls, all streams).
+ * Bookkeeping for benchmarks; the paper has no counterpart. */
+int64_t dpara_kernel_launches(void);
+
 #ifdef __cplusplus
 }
 #endif

@@ -66,9 +66,10 @@ lib.dpara_verify_select.argtypes = [C.POINTER(VerifyIO), C.c_void_p, C.c_size_t,
 lib.dpara_status_string.restype = C.c_char_p
 lib.dpara_status_string.argtypes = [C.c_int]
 lib.dpara_version.restype = C.c_int32
+lib.dpara_kernel_launches.restype = C.c_int64
 
 EXPORTED = ["dpara_draft_workspace_bytes", "dpara_draft_all_boundaries", "dpara_verify_workspace_bytes",
-            "dpara_verify_select", "dpara_status_string", "dpara_version"]
+            "dpara_verify_select", "dpara_status_string", "dpara_version", "dpara_kernel_launches"]
 
 
 class DparaError(RuntimeError):

@@ -2,9 +2,14 @@
 #include "attention_params.cuh"
 #include "layer.cuh"
 
+#include <atomic>
+
 using namespace dpara;
 
 namespace dpara {
+
+static std::atomic<long long> g_launches{0};
+void count_launches(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
 static dpara_status validate_shape(const dpara_shape *s) {
   if (!s) return DPARA_ERR_INVALID_ARG;
@@ -79,3 +84,5 @@ extern "C" const char *dpara_status_string(dpara_status s) {
 }
 
 extern "C" int32_t dpara_version(void) { return 1000; }
+
+extern "C" int64_t dpara_kernel_launches(void) { return g_launches.load(std::memory_order_relaxed); }

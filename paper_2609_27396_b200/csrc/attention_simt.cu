@@ -107,6 +107,7 @@ dpara_status launch_attention_simt(const AttnParams &P, cudaStream_t st) {
   else
     attn_simt_kernel<64><<<(unsigned)blocks, 128, 0, st>>>(P);
   DPARA_CHECK_LAUNCH();
+  count_launches(1);
   return DPARA_OK;
 }
 

@@ -31,4 +31,7 @@ inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 
     if (e_ != cudaSuccess) return DPARA_ERR_CUDA;              \
   } while (0)
 
+// Process-wide count of kernels this library has launched (evidence for benchmarks; relaxed atomic).
+void count_launches(int n);
+
 }  // namespace dpara

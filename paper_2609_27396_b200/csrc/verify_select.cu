@@ -424,6 +424,7 @@ dpara_status launch_verify(const dpara_verify_io *io, void *ws, int32_t *status_
     verify_sampling_kernel<<<grid, kVsThreads, 0, st>>>(P);
   }
   DPARA_CHECK_LAUNCH();
+  count_launches(1);
   return DPARA_OK;
 }
 }  // namespace dpara
