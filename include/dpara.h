@@ -41,7 +41,8 @@ typedef enum {
   DPARA_ERR_UNSUPPORTED = -2, /* shape outside what the kernels are built for (see each call) */
   DPARA_ERR_WORKSPACE = -3,   /* workspace missing or smaller than *_workspace_bytes() */
   DPARA_ERR_CUDA = -4,        /* a CUDA runtime/driver call failed (launch, tensor-map encode) */
-  DPARA_ERR_TIMEOUT = -5      /* reserved for device-side bounded waits, reported via status_word */
+  DPARA_ERR_TIMEOUT = -5,     /* reserved for device-side bounded waits, reported via status_word */
+  DPARA_ERR_STATIC_LIMIT = -6 /* request needs more scratch than a fixed-scratch entry point owns */
 } dpara_status;
 
 /* bits OR-ed into *status_word by kernels */
@@ -161,6 +162,34 @@ size_t dpara_verify_workspace_bytes(const dpara_verify_io *io);
  * Errors: INVALID_ARG, UNSUPPORTED (J > 64), WORKSPACE, CUDA. */
 dpara_status dpara_verify_select(const dpara_verify_io *io, void *workspace, size_t workspace_bytes,
                                  int32_t *status_word, void *stream);
+
+/* dpara_verify_select for callers that cannot hand over scratch memory.  (The paper has no
+ * counterpart; this is a packaging variant of the call above.)
+ *
+ * Who needs it: a serving process that has given all free device memory to its own KV-cache pool at
+ * start-up, or a decode loop in which an allocation would stall the device between two rounds, has
+ * no way to obtain the workspace the normal call asks for.  This variant computes exactly what
+ * dpara_verify_select computes -- same kernels, same outputs, bit for bit -- but keeps its scratch
+ * in a fixed array of DPARA_VERIFY_STATIC_SCRATCH_BYTES that lives inside the library's device
+ * image.  Every GPU that loads the library carries that array until the process exits.
+ *
+ *  - The call performs no cudaMalloc/cudaFree and calls no allocating routine.  Inputs and outputs
+ *    are still the caller's buffers, as in dpara_verify_io.
+ *  - The first call on each device looks up the array's device address (with that device current)
+ *    and remembers it.  Make that first call during start-up, before any stream capture begins on
+ *    that device.
+ *  - Requests whose scratch need (dpara_verify_workspace_bytes) exceeds the fixed size are refused
+ *    with DPARA_ERR_STATIC_LIMIT and nothing is launched.  For scale: greedy mode with 16 requests
+ *    x 16 boundaries needs 2.3 KB, sampling mode with 8 requests over a 151 936-token vocabulary
+ *    5 KB; the need grows with batch * n_boundaries (greedy) or batch * ceil(vocab / 4096) (sampling).
+ *  - All calls on a device share the one array and it keeps whatever the previous call left; the
+ *    call itself clears the parts that must start at zero.  Two calls that overlap on the same GPU
+ *    (different streams, or different host threads without ordering) race on it and give undefined
+ *    results: order them on one stream or with events.
+ * Errors: as dpara_verify_select, plus DPARA_ERR_STATIC_LIMIT; DPARA_ERR_CUDA if the address lookup
+ * fails. */
+#define DPARA_VERIFY_STATIC_SCRATCH_BYTES (256u * 1024u)
+dpara_status dpara_verify_select_static(const dpara_verify_io *io, int32_t *status_word, void *stream);
 
 const char *dpara_status_string(dpara_status s);
 

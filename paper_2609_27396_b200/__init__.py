@@ -22,7 +22,8 @@ if not os.path.exists(LIB_PATH):
 
 lib = C.CDLL(LIB_PATH)
 
-OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = 0, -1, -2, -3, -4, -5
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_STATIC_LIMIT = 0, -1, -2, -3, -4, -5, -6
+VERIFY_STATIC_SCRATCH_BYTES = 256 * 1024
 STATUS_BAD_TOKEN, STATUS_TIMEOUT = 1, 2
 BF16, F32 = 0, 1
 
@@ -63,13 +64,15 @@ lib.dpara_verify_workspace_bytes.restype = C.c_size_t
 lib.dpara_verify_workspace_bytes.argtypes = [C.POINTER(VerifyIO)]
 lib.dpara_verify_select.restype = C.c_int
 lib.dpara_verify_select.argtypes = [C.POINTER(VerifyIO), C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
+lib.dpara_verify_select_static.restype = C.c_int
+lib.dpara_verify_select_static.argtypes = [C.POINTER(VerifyIO), C.c_void_p, C.c_void_p]
 lib.dpara_status_string.restype = C.c_char_p
 lib.dpara_status_string.argtypes = [C.c_int]
 lib.dpara_version.restype = C.c_int32
 lib.dpara_kernel_launches.restype = C.c_int64
 
 EXPORTED = ["dpara_draft_workspace_bytes", "dpara_draft_all_boundaries", "dpara_verify_workspace_bytes",
-            "dpara_verify_select", "dpara_status_string", "dpara_version", "dpara_kernel_launches"]
+            "dpara_verify_select", "dpara_verify_select_static", "dpara_status_string", "dpara_version", "dpara_kernel_launches"]
 
 
 class DparaError(RuntimeError):
@@ -182,6 +185,21 @@ class VerifyPlan:
                                      self.status.data_ptr(), _stream_ptr(stream))
         if rc != OK:
             raise DparaError(rc)
+
+
+def verify_select_static(plan: "VerifyPlan", *, target, draft_tokens, reps=None, draft_probs=None, uniforms=None,
+                         stream=None) -> None:
+    """dpara_verify_select_static: the same verify/select, for callers that cannot allocate device memory
+    (their own pool owns all of it, or an allocation would stall the decode loop).  Uses the library's
+    fixed scratch array instead of a caller workspace; `plan` only supplies the output tensors.  The first
+    call on a device does a one-time address lookup: make it at start-up, before any stream capture.
+    Calls that overlap on one GPU race on the shared scratch."""
+    io = plan.io
+    io.target, io.draft_tokens = _ptr(target), _ptr(draft_tokens)
+    io.draft_probs, io.uniforms, io.reps = _ptr(draft_probs), _ptr(uniforms), _ptr(reps)
+    rc = lib.dpara_verify_select_static(C.byref(io), plan.status.data_ptr(), _stream_ptr(stream))
+    if rc != OK:
+        raise DparaError(rc)
 
 
 def verify_select(target, draft_tokens, reps=None, *, mode: int = 0, draft_probs=None, uniforms=None, stream=None):

@@ -79,6 +79,7 @@ extern "C" const char *dpara_status_string(dpara_status s) {
     case DPARA_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
     case DPARA_ERR_CUDA: return "CUDA call failed";
     case DPARA_ERR_TIMEOUT: return "device-side wait timed out";
+    case DPARA_ERR_STATIC_LIMIT: return "request needs more scratch than the fixed-scratch entry point owns";
   }
   return "unknown status";
 }

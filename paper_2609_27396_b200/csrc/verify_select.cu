@@ -437,3 +437,45 @@ extern "C" dpara_status dpara_verify_select(const dpara_verify_io *io, void *wor
   if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 7u)) return DPARA_ERR_WORKSPACE;
   return launch_verify(io, workspace, status_word, static_cast<cudaStream_t>(stream));
 }
+
+// ------------------------------------------------------------------------------------------ fixed-scratch variant
+// For callers that cannot allocate (all device memory already handed to their own pool, or an
+// allocation would stall the decode loop): the scratch lives in the library's device image.
+// `g_verify_scratch` below is only a host-side stand-in for the array when named in host code; the
+// device address a kernel can use comes from cudaGetSymbolAddress, looked up once per device with
+// that device current.
+#include <mutex>
+
+static __device__ __align__(256) unsigned char g_verify_scratch[DPARA_VERIFY_STATIC_SCRATCH_BYTES];
+
+namespace dpara {
+constexpr int kMaxDevices = 64;
+static void *g_scratch_addr[kMaxDevices] = {nullptr};
+static std::mutex g_scratch_mutex;
+
+// Device address of the fixed scratch on the CURRENT device (set-up on first use per device).
+static dpara_status static_scratch_ptr(void **out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return DPARA_ERR_CUDA;
+  if (dev < 0 || dev >= kMaxDevices) return DPARA_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> lock(g_scratch_mutex);
+  if (!g_scratch_addr[dev]) {
+    void *p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_verify_scratch) != cudaSuccess || !p) return DPARA_ERR_CUDA;
+    g_scratch_addr[dev] = p;
+  }
+  *out = g_scratch_addr[dev];
+  return DPARA_OK;
+}
+}  // namespace dpara
+
+extern "C" dpara_status dpara_verify_select_static(const dpara_verify_io *io, int32_t *status_word, void *stream) {
+  dpara_status s = validate_verify(io);
+  if (s != DPARA_OK) return s;
+  if (dpara_verify_workspace_bytes(io) > (size_t)DPARA_VERIFY_STATIC_SCRATCH_BYTES) return DPARA_ERR_STATIC_LIMIT;
+  void *scratch = nullptr;
+  s = static_scratch_ptr(&scratch);
+  if (s != DPARA_OK) return s;
+  // launch_verify clears (cudaMemsetAsync on `stream`) the keys/counters that must start at zero
+  return launch_verify(io, scratch, status_word, static_cast<cudaStream_t>(stream));
+}
