@@ -196,6 +196,25 @@ const char *dpara_status_string(dpara_status s);
 /* Library/ABI version: major * 1000 + minor. */
 int32_t dpara_version(void);
 
+/* The projection GEMM of the backbone block on its own (Sec. 3.1 names the block's parts only as
+ * "attention, MLP, and their normalizations"; bf16 operands, fp32 accumulation on the tensor cores):
+ *   out[M][N] = epilogue( a[M][K] * w[N][K]^T ),  a and w bf16 row-major (weights stored [out][in]).
+ * epilogue 0: out bf16.   epilogue 1: out fp32 = resid + product (resid [M][N], bf16 when
+ * resid_dtype == DPARA_BF16 else fp32), optional bf16 copy in out_bf16.   epilogue 2: w holds 2N rows,
+ * [0,N) gate and [N,2N) up; out bf16 = silu(a Wg^T) * (a Wu^T).
+ * No workspace.  Errors: INVALID_ARG (null/misaligned), UNSUPPORTED (K % 64 != 0 or N % 8 != 0), CUDA. */
+typedef struct {
+  const void *a;
+  const void *w;
+  int32_t M, N, K;
+  int32_t epilogue;
+  const void *resid;
+  int32_t resid_dtype;
+  void *out;
+  void *out_bf16;
+} dpara_gemm_io;
+dpara_status dpara_gemm_bf16(const dpara_gemm_io *io, int32_t *status_word, void *stream);
+
 /* Number of kernels this library has launched in this process so far (all calls, all streams).
  * Bookkeeping for benchmarks; the paper has no counterpart. */
 int64_t dpara_kernel_launches(void);

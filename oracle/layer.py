@@ -47,6 +47,18 @@ def silu(x: np.ndarray) -> np.ndarray:
     return x / (1.0 + np.exp(-x))
 
 
+def linear(x: np.ndarray, w: np.ndarray) -> np.ndarray:
+    """x [M][K] times w [N][K] transposed (weights stored [out][in]), float64."""
+    return x @ w.T
+
+
+def swiglu_linear(x: np.ndarray, w_gate_up: np.ndarray) -> np.ndarray:
+    """silu(x Wg^T) * (x Wu^T) with w_gate_up rows [0, I) = gate and [I, 2I) = up; rounded to bf16."""
+    I = w_gate_up.shape[0] // 2
+    gu = linear(x, w_gate_up)
+    return _r16(silu(gu[:, :I]) * gu[:, I:])
+
+
 def rope(x: np.ndarray, pos: np.ndarray, theta: float) -> np.ndarray:
     """Rotate-half rotary embedding.  x [..., R, D] with one position per row R (pos [R]).
     Pair (d, d + D/2) is rotated by angle pos * theta^(-2d/D)."""

@@ -75,6 +75,32 @@ EXPORTED = ["dpara_draft_workspace_bytes", "dpara_draft_all_boundaries", "dpara_
             "dpara_verify_select", "dpara_verify_select_static", "dpara_status_string", "dpara_version", "dpara_kernel_launches"]
 
 
+class GemmIO(C.Structure):
+    _fields_ = [("a", C.c_void_p), ("w", C.c_void_p), ("M", C.c_int32), ("N", C.c_int32), ("K", C.c_int32),
+                ("epilogue", C.c_int32), ("resid", C.c_void_p), ("resid_dtype", C.c_int32), ("out", C.c_void_p),
+                ("out_bf16", C.c_void_p)]
+
+
+lib.dpara_gemm_bf16.restype = C.c_int
+lib.dpara_gemm_bf16.argtypes = [C.POINTER(GemmIO), C.c_void_p, C.c_void_p]
+EXPORTED.append("dpara_gemm_bf16")
+
+
+def gemm_bf16(a, w, *, epilogue: int = 0, resid=None, want_bf16_copy: bool = False, status=None, stream=None):
+    """dpara_gemm_bf16: out = epilogue(a @ w.T); a [M][K], w [N][K] (epilogue 2: [2N][K]) bf16 CUDA tensors."""
+    M, K = a.shape
+    N = w.shape[0] // 2 if epilogue == 2 else w.shape[0]
+    out = torch.empty((M, N), dtype=torch.float32 if epilogue == 1 else torch.bfloat16, device=a.device)
+    out16 = torch.empty((M, N), dtype=torch.bfloat16, device=a.device) if (want_bf16_copy and epilogue == 1) else None
+    st = status if status is not None else torch.zeros(1, dtype=torch.int32, device=a.device)
+    io = GemmIO(_ptr(a), _ptr(w), M, N, K, epilogue, _ptr(resid),
+                BF16 if (resid is not None and resid.dtype == torch.bfloat16) else F32, _ptr(out), _ptr(out16))
+    rc = lib.dpara_gemm_bf16(C.byref(io), st.data_ptr(), _stream_ptr(stream))
+    if rc != OK:
+        raise DparaError(rc)
+    return (out, out16, st) if out16 is not None else (out, st)
+
+
 class DparaError(RuntimeError):
     def __init__(self, code: int):
         self.code = code

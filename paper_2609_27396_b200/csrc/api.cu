@@ -87,3 +87,14 @@ extern "C" const char *dpara_status_string(dpara_status s) {
 extern "C" int32_t dpara_version(void) { return 1000; }
 
 extern "C" int64_t dpara_kernel_launches(void) { return g_launches.load(std::memory_order_relaxed); }
+
+#include "gemm.cuh"
+
+extern "C" dpara_status dpara_gemm_bf16(const dpara_gemm_io *io, int32_t *status_word, void *stream) {
+  if (!io) return DPARA_ERR_INVALID_ARG;
+  if (io->epilogue < 0 || io->epilogue > 2) return DPARA_ERR_INVALID_ARG;
+  GemmArgs g;
+  g.a = io->a; g.w = io->w; g.M = io->M; g.N = io->N; g.K = io->K; g.epi = io->epilogue;
+  g.resid = io->resid; g.resid_bf16 = io->resid_dtype == DPARA_BF16; g.out = io->out; g.out_bf16 = io->out_bf16;
+  return launch_gemm_tc(g, status_word, static_cast<cudaStream_t>(stream));
+}

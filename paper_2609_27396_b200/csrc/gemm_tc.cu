@@ -1,0 +1,220 @@
+// bf16 GEMM  out[M][N] = epilogue( a[M][K] * w[N][K]^T )  on the 5th-generation tensor cores.
+//
+// One CTA computes a 128 x 256 output tile: a TMA producer warp streams 64-wide K slabs of both
+// operands (128-byte swizzle) through a 4-stage shared-memory ring, one elected thread issues
+// tcgen05.mma (M = 128, N = 256, K = 16, fp32 accumulator in 256 TMEM columns), four warps read the
+// accumulator back with tcgen05.ld and apply the epilogue:
+//   0  bf16 store                                   (QKV projection)
+//   1  fp32 out = resid + acc  (+ bf16 copy)        (O and down projections with the residual add)
+//   2  bf16 out = silu(gate) * up                   (gate/up projection: the tile's 256 accumulator
+//                                                    columns are 128 gate columns and the matching 128
+//                                                    up columns, so the activation never leaves the SM)
+// Every mbarrier wait is bounded; on expiry the CTA sets DPARA_STATUS_TIMEOUT and drains.
+#include "gemm.cuh"
+#include "sm100_ptx.cuh"
+
+namespace dpara {
+using namespace ptx;
+
+namespace {
+constexpr int kBM = 128, kBN = 256, kBK = 64, kStages = 4;
+constexpr int kABytes = kBM * kBK * 2;         // 16 KB
+constexpr int kBBytes = kBN * kBK * 2;         // 32 KB (two 128-row boxes)
+constexpr int kStageBytes = kABytes + kBBytes;  // 48 KB
+constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*align*/ + 256 /*barriers*/;
+constexpr int kThreads = 192;                   // warps 0-3 epilogue, 4 TMA, 5 MMA
+}  // namespace
+
+struct GemmKernelParams {
+  CUtensorMap map_a;
+  CUtensorMap map_b;
+  int M, N, K;
+  int epi;
+  int up_row_offset;
+  void *out;
+  const void *resid;
+  int resid_bf16;
+  void *out_bf16;
+  int32_t *status;
+};
+
+__device__ __forceinline__ float silu_f(float g) { return g / (1.0f + __expf(-g)); }
+
+__global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_constant__ GemmKernelParams P) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t *full = reinterpret_cast<uint64_t *>(smem + kStages * kStageBytes);
+  uint64_t *empty = full + kStages;
+  uint64_t *acc_full = empty + kStages;
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_full + 1);
+  volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n_tile = blockIdx.x, m_tile = blockIdx.y;
+  const int nkb = P.K / kBK;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(full + s, 1);
+      mbar_init(empty + s, 1);
+    }
+    mbar_init(acc_full, 1);
+    *abort_flag = 0;
+    fence_barrier_init();
+  }
+  if (warp == 5) {
+    tmem_alloc(tmem_slot, 256);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+
+  if (warp == 4) {
+    if (lane == 0) {
+      prefetch_tensormap(&P.map_a);
+      prefetch_tensormap(&P.map_b);
+      const int brow0 = P.epi == 2 ? n_tile * 128 : n_tile * kBN;
+      const int brow1 = P.epi == 2 ? P.up_row_offset + n_tile * 128 : n_tile * kBN + 128;
+      for (int kb = 0; kb < nkb; ++kb) {
+        const int s = kb % kStages;
+        const uint32_t ph = (kb / kStages) & 1;
+        if (!mbar_wait(empty + s, ph ^ 1u, abort_flag)) break;
+        uint8_t *sa = smem + s * kStageBytes;
+        mbar_arrive_expect_tx(full + s, kStageBytes);
+        tma_load_2d(sa, &P.map_a, full + s, kb * kBK, m_tile * kBM);
+        tma_load_2d(sa + kABytes, &P.map_b, full + s, kb * kBK, brow0);
+        tma_load_2d(sa + kABytes + 128 * kBK * 2, &P.map_b, full + s, kb * kBK, brow1);
+      }
+    }
+  } else if (warp == 5) {
+    if (lane == 0) {
+      constexpr uint32_t idesc = idesc_bf16_f32(kBM, kBN, false, false);
+      bool ok = true;
+      for (int kb = 0; kb < nkb && ok; ++kb) {
+        const int s = kb % kStages;
+        const uint32_t ph = (kb / kStages) & 1;
+        ok = mbar_wait(full + s, ph, abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t sa = smem_u32(smem + s * kStageBytes);
+#pragma unroll
+        for (int kk = 0; kk < kBK / 16; ++kk) {
+          const uint64_t ad = smem_desc_sw128(sa + kk * 32, 16, 1024);
+          const uint64_t bd = smem_desc_sw128(sa + kABytes + kk * 32, 16, 1024);
+          mma_ss(tmem, ad, bd, idesc, (kb | kk) != 0);
+        }
+        mma_commit(empty + s);
+      }
+      mma_commit(acc_full);
+    }
+  } else {
+    // ---------------- epilogue: thread = one accumulator row
+    const bool ok = __all_sync(0xffffffffu, mbar_wait(acc_full, 0, abort_flag));  // warp-uniform: tcgen05.ld is warp-wide
+    tc_fence_after();
+    const int row = m_tile * kBM + warp * 32 + lane;
+    const uint32_t taddr = tmem + ((uint32_t)(warp * 32) << 16);
+    if (ok) {
+      if (P.epi == 2) {
+        const int col0 = n_tile * 128;
+#pragma unroll 1
+        for (int c = 0; c < 4; ++c) {
+          uint32_t g[32], u[32];
+          tmem_ld32(taddr + c * 32, g);
+          tmem_ld32(taddr + 128 + c * 32, u);
+          tmem_wait_ld();
+          if (row < P.M) {
+            uint16_t *o = static_cast<uint16_t *>(P.out) + (size_t)row * P.N + col0 + c * 32;
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+              if (col0 + c * 32 + v * 8 < P.N) {
+                uint32_t w[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                  float a0 = silu_f(__uint_as_float(g[v * 8 + 2 * e])) * __uint_as_float(u[v * 8 + 2 * e]);
+                  float a1 = silu_f(__uint_as_float(g[v * 8 + 2 * e + 1])) * __uint_as_float(u[v * 8 + 2 * e + 1]);
+                  w[e] = pack_bf16(a0, a1);
+                }
+                *reinterpret_cast<uint4 *>(o + v * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+              }
+            }
+          }
+        }
+      } else {
+        const int col0 = n_tile * kBN;
+#pragma unroll 1
+        for (int c = 0; c < kBN / 32; ++c) {
+          uint32_t r[32];
+          tmem_ld32(taddr + c * 32, r);
+          tmem_wait_ld();
+          if (row < P.M) {
+            const int cb = col0 + c * 32;
+            if (P.epi == 0) {
+              uint16_t *o = static_cast<uint16_t *>(P.out) + (size_t)row * P.N + cb;
+#pragma unroll
+              for (int v = 0; v < 4; ++v) {
+                if (cb + v * 8 < P.N) {
+                  uint32_t w[4];
+#pragma unroll
+                  for (int e = 0; e < 4; ++e)
+                    w[e] = pack_bf16(__uint_as_float(r[v * 8 + 2 * e]), __uint_as_float(r[v * 8 + 2 * e + 1]));
+                  *reinterpret_cast<uint4 *>(o + v * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+                }
+              }
+            } else {
+              float *o = static_cast<float *>(P.out) + (size_t)row * P.N + cb;
+#pragma unroll
+              for (int v = 0; v < 8; ++v) {
+                if (cb + v * 4 < P.N) {
+                  float x[4];
+                  if (P.resid_bf16) {
+                    uint2 rr = *reinterpret_cast<const uint2 *>(static_cast<const uint16_t *>(P.resid) + (size_t)row * P.N + cb + v * 4);
+                    x[0] = bf16lo(rr.x); x[1] = bf16hi(rr.x); x[2] = bf16lo(rr.y); x[3] = bf16hi(rr.y);
+                  } else {
+                    float4 rr = *reinterpret_cast<const float4 *>(static_cast<const float *>(P.resid) + (size_t)row * P.N + cb + v * 4);
+                    x[0] = rr.x; x[1] = rr.y; x[2] = rr.z; x[3] = rr.w;
+                  }
+#pragma unroll
+                  for (int e = 0; e < 4; ++e) x[e] += __uint_as_float(r[v * 4 + e]);
+                  *reinterpret_cast<float4 *>(o + v * 4) = make_float4(x[0], x[1], x[2], x[3]);
+                  if (P.out_bf16) {
+                    uint16_t *ob = static_cast<uint16_t *>(P.out_bf16) + (size_t)row * P.N + cb + v * 4;
+                    *reinterpret_cast<uint2 *>(ob) = make_uint2(pack_bf16(x[0], x[1]), pack_bf16(x[2], x[3]));
+                  }
+                }
+              }
+            }
+          }
+        }
+      }
+    }
+  }
+  // ---------------- teardown
+  if (threadIdx.x == 0 && *abort_flag && P.status) atomicOr(reinterpret_cast<unsigned int *>(P.status), DPARA_STATUS_TIMEOUT);
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 5) tmem_dealloc(tmem, 256);
+}
+
+dpara_status launch_gemm_tc(const GemmArgs &g, int32_t *status, cudaStream_t st) {
+  if (g.M <= 0 || g.N <= 0 || g.K <= 0) return DPARA_ERR_INVALID_ARG;
+  if (g.K % kBK != 0 || g.N % 8 != 0) return DPARA_ERR_UNSUPPORTED;
+  if (!g.a || !g.w || !g.out || (g.epi == 1 && !g.resid)) return DPARA_ERR_INVALID_ARG;
+  if (!aligned16(g.a) || !aligned16(g.w) || !aligned16(g.out) || !aligned16(g.resid) || !aligned16(g.out_bf16)) return DPARA_ERR_INVALID_ARG;
+  GemmKernelParams P;
+  const int w_rows = g.epi == 2 ? 2 * g.N : g.N;
+  if (!make_tmap_bf16_2d(&P.map_a, g.a, g.K, g.M, (uint64_t)g.K * 2, kBK, kBM)) return DPARA_ERR_CUDA;
+  if (!make_tmap_bf16_2d(&P.map_b, g.w, g.K, w_rows, (uint64_t)g.K * 2, kBK, 128)) return DPARA_ERR_CUDA;
+  P.M = g.M; P.N = g.N; P.K = g.K; P.epi = g.epi; P.up_row_offset = g.N;
+  P.out = g.out; P.resid = g.resid; P.resid_bf16 = g.resid_bf16; P.out_bf16 = g.out_bf16; P.status = status;
+  if (cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess) return DPARA_ERR_CUDA;
+  const int tile_cols = g.epi == 2 ? 128 : kBN;
+  dim3 grid((g.N + tile_cols - 1) / tile_cols, (g.M + kBM - 1) / kBM);
+  gemm_tc_kernel<<<grid, kThreads, kSmemBytes, st>>>(P);
+  DPARA_CHECK_LAUNCH();
+  count_launches(1);
+  return DPARA_OK;
+}
+
+}  // namespace dpara
