@@ -1,6 +1,7 @@
 // Chooses the attention kernel for a shape and fills its parameters.
 #include <math.h>
 
+#include "attention_tc.cuh"
 #include "layer.cuh"
 
 namespace dpara {
@@ -24,11 +25,18 @@ void fill_attn_params(AttnParams &P, const dpara_shape *s, const dpara_attn_io *
   P.status_word = status_word;
 }
 
-size_t attention_workspace_bytes(const dpara_shape *, const int64_t *) { return 0; }
+size_t attention_workspace_bytes(const dpara_shape *shape, const int64_t *host_off) {
+  TcPlan plan = plan_attention_tc(shape, host_off);
+  return plan.eligible ? align_up(plan.workspace_bytes, 256) : 0;
+}
 
-dpara_status launch_attention(const dpara_shape *shape, const dpara_attn_io *io, void *, int32_t *status_word, cudaStream_t st) {
+dpara_status launch_attention(const dpara_shape *shape, const dpara_attn_io *io, void *workspace, int32_t *status_word,
+                              cudaStream_t st) {
   AttnParams P;
   fill_attn_params(P, shape, io, status_word);
+  if (P.hi <= P.lo) return DPARA_OK;
+  TcPlan plan = plan_attention_tc(shape, io->host_ctx_offsets);
+  if (plan.eligible) return launch_attention_tc(P, plan, io->host_ctx_offsets, workspace, st);
   return launch_attention_simt(P, st);
 }
 
