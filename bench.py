@@ -31,6 +31,9 @@ import workloads as W  # noqa: E402
 
 METRIC = "all_boundary_draft_step_us"
 L2_FLUSH_BYTES = 256 << 20
+# dram__bytes_read.sum + dram__bytes_write.sum of one attention launch, from the ncu capture summarised in
+# profiles/attention_tc_cfg3_b16.md (bytes per launch; None where no capture exists)
+NCU_DRAM_TRAFFIC = {"cfg3": 269349120, "cfg2": None}
 
 
 # ----------------------------------------------------------------------------- algorithmic work
@@ -337,10 +340,7 @@ def main():
     by = attention_bytes(wl.attn)
     ach_tf = fl / (att_ms * 1e-3) / 1e12
     ach_gb = by / (att_ms * 1e-3) / 1e9
-    traffic = None
-    tp = os.path.join(ROOT, "profiles", "traffic.json")
-    if os.path.exists(tp):
-        traffic = json.load(open(tp)).get(f"attention_{args.workload}")
+    traffic = NCU_DRAM_TRAFFIC.get(args.workload)
     roofline = {"kernel": "all-boundary attention", "bound": "tensor", "achieved": ach_tf, "peak": peaks["bf16_tflops"],
                 "unit": "TFLOP/s", "frac": ach_tf / peaks["bf16_tflops"], "traffic": traffic, "peak_source": peaks["source"] + " (burst)",
                 "hbm": {"achieved": ach_gb, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach_gb / peaks["hbm_gbs"],
