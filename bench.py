@@ -196,6 +196,56 @@ class StepRunner:
         return [e[0].elapsed_time(e[1]) for e in ev]
 
 
+class LayerRunner:
+    """The full-layer, long-context workload (cfg5): one draft call runs the whole backbone block around the
+    all-boundary attention; greedy verify/select then gathers from the block's bf16 output."""
+
+    def __init__(self, wl: W.Workload, seed: int):
+        import torch
+        import paper_2609_27396_b200 as dp
+        self.torch = torch
+        a, v, l = wl.attn, wl.verify, wl.layer
+        ain = W.make_attn_inputs(a, seed, with_q=False, with_blk=False)
+        lin = W.make_layer_inputs(l, a, seed)
+        ver = W.make_verify_inputs(v, seed, reps=np.zeros((1,), np.uint16))
+        bf = lambda bits: torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda().view(torch.bfloat16)
+        self.t = {k: bf(getattr(lin, k)) for k in ("x", "w_qkv", "w_o", "w_gate_up", "w_down", "rms1_w", "rms2_w", "qnorm_w", "knorm_w")}
+        self.kv = {k: bf(getattr(ain, k)) for k in ("k_ctx", "v_ctx", "k_spine", "v_spine")}
+        self.y = torch.zeros((a.batch, a.n_boundaries, a.block, l.hidden), dtype=torch.float32, device="cuda")
+        self.y16 = torch.zeros((a.batch, a.n_boundaries, a.block, l.hidden), dtype=torch.bfloat16, device="cuda")
+        lio = dp.make_layer_io(**self.t, rms_eps=l.rms_eps, rope_theta=l.rope_theta, use_rope=l.use_rope, y_f32=self.y, y_bf16=self.y16)
+        self.plan = dp.DraftPlan(ctx_offsets=[int(x) for x in ain.ctx_offsets], n_boundaries=a.n_boundaries, block=a.block,
+                                 n_q_heads=a.n_q_heads, n_kv_heads=a.n_kv_heads, head_dim=a.head_dim, prefix_base=a.prefix_base,
+                                 n_spine=a.spine, layer=lio)
+        self.vplan = dp.VerifyPlan(batch=v.batch, n_boundaries=v.n_boundaries, vocab=v.vocab, block=v.block, hidden=v.hidden, mode=0)
+        self.target = torch.from_numpy(ver.target).cuda()
+        self.tokens = torch.from_numpy(ver.draft_tokens).cuda()
+        self.flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device="cuda")
+
+    def step(self):
+        self.plan(**self.kv)
+        self.vplan(target=self.target, draft_tokens=self.tokens, reps=self.y16)
+
+    def timed_steps(self, k: int):
+        torch = self.torch
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(k)]
+        for s in range(k):
+            self.flush.zero_()
+            ev[s][0].record()
+            self.plan(**self.kv)
+            ev[s][1].record()
+            self.vplan(target=self.target, draft_tokens=self.tokens, reps=self.y16)
+            ev[s][2].record()
+        torch.cuda.synchronize()
+        return [(e[0].elapsed_time(e[2]), e[0].elapsed_time(e[1]), e[1].elapsed_time(e[2])) for e in ev]
+
+
+def layer_gemm_flops(a: W.AttnShape, l: W.LayerShape) -> float:
+    M = a.batch * a.n_boundaries * a.block
+    qd, kd = a.n_q_heads * a.head_dim, a.n_kv_heads * a.head_dim
+    return 2.0 * M * (l.hidden * (qd + 2 * kd) + qd * l.hidden + 3 * l.hidden * l.intermediate)
+
+
 # ----------------------------------------------------------------------------- the oracle arm (host cores)
 def oracle_sample(wl: W.Workload, seed: int, n_pairs: int, n_verify_req: int, inp=None, ver=None):
     """Times the oracle, as it stands, on a bounded sample of the step: `n_pairs` (request, boundary)
@@ -255,6 +305,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg3", choices=["cfg2", "cfg3"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-layer", action="store_true", help="skip the full-layer (cfg5) leg")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -298,14 +349,12 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    def max_over_ranks(x: float) -> float:
-        if dist is None:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+    from paper_2609_27396_b200.dist_util import max_over_ranks as _mor, rank_seed
 
-    run = StepRunner(wl, wl.seed + 1000 * rank)
+    def max_over_ranks(x: float) -> float:
+        return _mor(x, device="cuda")
+
+    run = StepRunner(wl, rank_seed(wl.seed, rank))
     for _ in range(max(args.warmup, 3)):
         run.step()
     barrier()
@@ -371,6 +420,19 @@ def main():
                      "all_over_single": a2 / (statistics.median(p[1] for p in s2) * 1e3), "allowance": w2.attn.n_boundaries,
                      "attention_gbs": attention_bytes(w2.attn) / (a2 * 1e-6) / 1e9, "attention_tflops": attention_flops(w2.attn) / (a2 * 1e-6) / 1e12}
         del r2
+        if not args.no_layer:
+            w5 = W.workload(5)
+            r5 = LayerRunner(w5, w5.seed)
+            for _ in range(3):
+                r5.step()
+            p5 = r5.timed_steps(max(5, min(args.steps, 10)))
+            d5 = statistics.median(p[1] for p in p5) * 1e3
+            fl5 = attention_flops(w5.attn) + layer_gemm_flops(w5.attn, w5.layer)
+            out["layer_cfg5"] = {"workload": w5.name, "step_us": statistics.median(p[0] for p in p5) * 1e3, "draft_layer_us": d5,
+                                 "verify_select_us": statistics.median(p[2] for p in p5) * 1e3,
+                                 "flops": fl5, "tflops": fl5 / (d5 * 1e-6) / 1e12,
+                                 "tensor_frac_of_measured_sustained": fl5 / (d5 * 1e-6) / 1e12 / (peaks["bf16_tflops_sustained"] or peaks["bf16_tflops"])}
+            del r5
         if not args.no_cpu_baseline:
             t, est, desc = oracle_sample(wl, wl.seed, 0, wl.verify.batch, run.inp, run.ver)
             out["cpu_baseline"] = {"value": est * 1e6, "unit": "us", "cores": oracle_threads(), "kind": "oracle", "sample": desc,
