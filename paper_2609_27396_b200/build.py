@@ -32,7 +32,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if not force and not needs_build():
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    cmd = [nvcc] + NVCC_FLAGS + ["-o", LIB] + sources()
+    extra = os.environ.get("DPARA_NVCC_EXTRA", "").split()      # e.g. -DNAME=1 for kernel experiments
+    cmd = [nvcc] + NVCC_FLAGS + extra + ["-o", LIB] + sources()
     r = subprocess.run(cmd, capture_output=True, text=True)
     log = os.path.join(HERE, "build.log")
     with open(log, "w") as f:

@@ -5,7 +5,7 @@
 // of all G query heads that share the KV head, and every K/V byte streamed from HBM serves all
 // boundaries and all heads of the group at once.
 //
-//   warp 8      TMA producer: Q tiles once, then K/V tiles of 128 keys through a 2-stage ring.
+//   warp 8      TMA producer: Q tiles once, then K and V tiles of 128 keys through one ring of tile slots.
 //               The context needs no mask at all (every row sees the whole cache); the spine prefix
 //               and the boundaries' own blocks are packed into ONE extra "tail" tile per CTA.
 //   warp 9      one thread issues tcgen05.mma:  S_t = Q_t K^T  (A, B from shared memory) and
@@ -27,8 +27,8 @@ using namespace ptx;
 
 namespace {
 constexpr int kThreads = 320;
-constexpr int kStages = 2;
 constexpr float kRescaleLog2 = 8.0f;
+constexpr int kMaxOrdered = 128;
 }  // namespace
 
 struct TcParams {
@@ -38,6 +38,10 @@ struct TcParams {
   float *part_o;   // [item][2][128][D]
   float *part_ml;  // [item][2][128][2]
   float c_log2;    // softmax scale * log2(e)
+  // requests in order of decreasing context length: the block scheduler hands out CTAs in grid order, so
+  // launching the long requests first leaves the short ones to fill the tail of a ragged batch
+  uint8_t req_order[kMaxOrdered];
+  int use_order;
 };
 
 template <int D>
@@ -45,7 +49,10 @@ struct TcCfg {
   static constexpr int kSlabs = D / 64;
   static constexpr int kSlabBytes = 128 * 128;         // 128 rows x 64 bf16
   static constexpr int kTileBytes = kSlabs * kSlabBytes;  // Q, K or V tile
-  static constexpr int kSmemBytes = 2 * kTileBytes + kStages * 2 * kTileBytes + 1024 + 512;
+  // K and V tiles travel through ONE ring of tile-sized slots (K0 V0 K1 V1 ...), as deep as shared memory
+  // allows next to the two Q tiles: the producer runs ~1.5 iterations ahead of the MMA issuer
+  static constexpr int kSlots = (227 * 1024 - 2 * kTileBytes - 2048) / kTileBytes > 8 ? 8 : (227 * 1024 - 2 * kTileBytes - 2048) / kTileBytes;
+  static constexpr int kSmemBytes = 2 * kTileBytes + kSlots * kTileBytes + 1024 + 512;
   static constexpr int kOBase = 256;                    // TMEM column of O0
 };
 
@@ -56,14 +63,16 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t *sQ = smem;                                   // 2 tiles
-  uint8_t *sKV = smem + 2 * Cfg::kTileBytes;            // per stage: K tile, V tile
-  uint64_t *bars = reinterpret_cast<uint64_t *>(sKV + kStages * 2 * Cfg::kTileBytes);
-  uint64_t *kv_full = bars, *kv_empty = bars + 2, *q_full = bars + 4, *s_full = bars + 5, *p_full = bars + 7, *pv_done = bars + 9;
-  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 11);
+  uint8_t *sKV = smem + 2 * Cfg::kTileBytes;            // ring of K / V tile slots
+  constexpr int kSlots = Cfg::kSlots;
+  uint64_t *bars = reinterpret_cast<uint64_t *>(sKV + kSlots * Cfg::kTileBytes);
+  uint64_t *kv_full = bars, *kv_empty = bars + kSlots, *q_full = bars + 2 * kSlots, *s_full = q_full + 1, *p_full = q_full + 3,
+           *pv_done = q_full + 5;
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(q_full + 7);
   volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int n = blockIdx.z, g = blockIdx.y;
+  const int n = P.use_order ? (int)P.req_order[blockIdx.z] : (int)blockIdx.z, g = blockIdx.y;
   const int pair = blockIdx.x / P.nsplit, split = blockIdx.x % P.nsplit;
   const int ntq = min(2, P.n_tiles - pair * 2);
   const long long c0 = A.ctx_offsets[n];
@@ -101,9 +110,9 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
   }
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kStages; ++s) { mbar_init(kv_full + s, 1); mbar_init(kv_empty + s, 1); }
+    for (int s = 0; s < kSlots; ++s) { mbar_init(kv_full + s, 1); mbar_init(kv_empty + s, 1); }
     mbar_init(q_full, 1);
-    for (int t = 0; t < 2; ++t) { mbar_init(s_full + t, 1); mbar_init(p_full + t, 128); mbar_init(pv_done + t, 1); }
+    for (int t = 0; t < 2; ++t) { mbar_init(s_full + t, 1); mbar_init(p_full + t, 4); mbar_init(pv_done + t, 1); }
     *abort_flag = 0;
     fence_barrier_init();
   }
@@ -124,40 +133,37 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
         for (int sl = 0; sl < Cfg::kSlabs; ++sl)
           tma_load_3d(sQ + t * Cfg::kTileBytes + sl * Cfg::kSlabBytes, &P.map_q, q_full, sl * 64, g * A.G, qrow0 + t * P.JI_T);
     }
-    for (int it = 0; it < n_iter; ++it) {
-      const int s = it & 1;
-      const uint32_t ph = (it >> 1) & 1;
-      if (!__all_sync(0xffffffffu, mbar_wait(kv_empty + s, ph ^ 1u, abort_flag))) break;
-      uint8_t *sK = sKV + s * 2 * Cfg::kTileBytes, *sV = sK + Cfg::kTileBytes;
+    // load q = 2 it is the K tile of iteration it, load 2 it + 1 its V tile; slot = q % kSlots
+    for (int q = 0; q < 2 * n_iter; ++q) {
+      const int it = q >> 1, is_v = q & 1;
+      const int sl = q % kSlots;
+      const uint32_t ph = (q / kSlots) & 1;
+      if (!__all_sync(0xffffffffu, mbar_wait(kv_empty + sl, ph ^ 1u, abort_flag))) break;
+      uint8_t *dst = sKV + sl * Cfg::kTileBytes;
       if (it < n_ctx_it) {
         if (lane == 0) {
           const int row = (int)(c0 + (long long)(t0 + it) * 128);
-          mbar_arrive_expect_tx(kv_full + s, 2 * Cfg::kTileBytes);
-          for (int sl = 0; sl < Cfg::kSlabs; ++sl) {
-            tma_load_3d(sK + sl * Cfg::kSlabBytes, &P.map_kc, kv_full + s, sl * 64, g, row);
-            tma_load_3d(sV + sl * Cfg::kSlabBytes, &P.map_vc, kv_full + s, sl * 64, g, row);
-          }
+          mbar_arrive_expect_tx(kv_full + sl, Cfg::kTileBytes);
+          for (int sb = 0; sb < Cfg::kSlabs; ++sb)
+            tma_load_3d(dst + sb * Cfg::kSlabBytes, is_v ? &P.map_vc : &P.map_kc, kv_full + sl, sb * 64, g, row);
         }
       } else {
-        // tail tile: rows the TMA boxes do not cover must still hold finite V (P = 0 there): clear the V tile
-        for (int o = lane * 16; o < Cfg::kTileBytes; o += 32 * 16) *reinterpret_cast<uint4 *>(sV + o) = make_uint4(0, 0, 0, 0);
-        fence_proxy_async();
-        __syncwarp();
+        if (is_v) {
+          // tail tile: rows the TMA boxes do not cover must still hold finite V (P = 0 there): clear the V tile
+          for (int o = lane * 16; o < Cfg::kTileBytes; o += 32 * 16) *reinterpret_cast<uint4 *>(dst + o) = make_uint4(0, 0, 0, 0);
+          fence_proxy_async();
+          __syncwarp();
+        }
         if (lane == 0) {
           uint32_t bytes = 0;
-          if (A.S > 0) bytes += 2u * A.S * 128 * Cfg::kSlabs;
-          if (P.has_blk) bytes += 2u * P.R_blk * 128 * Cfg::kSlabs;
-          mbar_arrive_expect_tx(kv_full + s, bytes);
-          for (int sl = 0; sl < Cfg::kSlabs; ++sl) {
-            if (A.S > 0) {
-              tma_load_3d(sK + sl * Cfg::kSlabBytes, &P.map_ks, kv_full + s, sl * 64, g, n * A.S);
-              tma_load_3d(sV + sl * Cfg::kSlabBytes, &P.map_vs, kv_full + s, sl * 64, g, n * A.S);
-            }
-            if (P.has_blk) {
-              const int brow = (n * A.J + jb0) * A.Bq;
-              tma_load_3d(sK + sl * Cfg::kSlabBytes + P.S8 * 128, &P.map_kb, kv_full + s, sl * 64, g, brow);
-              tma_load_3d(sV + sl * Cfg::kSlabBytes + P.S8 * 128, &P.map_vb, kv_full + s, sl * 64, g, brow);
-            }
+          if (A.S > 0) bytes += (uint32_t)A.S * 128 * Cfg::kSlabs;
+          if (P.has_blk) bytes += (uint32_t)P.R_blk * 128 * Cfg::kSlabs;
+          mbar_arrive_expect_tx(kv_full + sl, bytes);
+          for (int sb = 0; sb < Cfg::kSlabs; ++sb) {
+            if (A.S > 0) tma_load_3d(dst + sb * Cfg::kSlabBytes, is_v ? &P.map_vs : &P.map_ks, kv_full + sl, sb * 64, g, n * A.S);
+            if (P.has_blk)
+              tma_load_3d(dst + sb * Cfg::kSlabBytes + P.S8 * 128, is_v ? &P.map_vb : &P.map_kb, kv_full + sl, sb * 64, g,
+                          (n * A.J + jb0) * A.Bq);
           }
         }
       }
@@ -168,42 +174,44 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
       constexpr uint32_t idesc_qk = idesc_bf16_f32(128, 128, false, false);
       constexpr uint32_t idesc_pv = idesc_bf16_f32(128, D, false, true);
       const uint32_t q_addr = smem_u32(sQ), kv_addr = smem_u32(sKV);
-      auto issue_qk = [&](int t, int s) {
-        const uint32_t qa = q_addr + t * Cfg::kTileBytes, ka = kv_addr + s * 2 * Cfg::kTileBytes;
+      auto issue_qk = [&](int t, int it) {
+        const uint32_t qa = q_addr + t * Cfg::kTileBytes, ka = kv_addr + ((2 * it) % kSlots) * Cfg::kTileBytes;
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {
           const uint32_t off = (kk >> 2) * Cfg::kSlabBytes + (kk & 3) * 32;
           mma_ss(tmem + t * 128, smem_desc_sw128(qa + off, 16, 1024), smem_desc_sw128(ka + off, 16, 1024), idesc_qk, kk != 0);
         }
         mma_commit(s_full + t);
+        if (t == ntq - 1) mma_commit(kv_empty + (2 * it) % kSlots);      // K tile consumed by every query tile
       };
-      auto issue_pv = [&](int t, int s, bool acc) {
-        const uint32_t va = kv_addr + s * 2 * Cfg::kTileBytes + Cfg::kTileBytes;
+      auto issue_pv = [&](int t, int it) {
+        const uint32_t va = kv_addr + ((2 * it + 1) % kSlots) * Cfg::kTileBytes;
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk)
           mma_ts(tmem + Cfg::kOBase + t * D, tmem + t * 128 + kk * 8, smem_desc_sw128(va + kk * 2048, Cfg::kSlabBytes, 1024),
-                 idesc_pv, acc || kk != 0);
+                 idesc_pv, it > 0 || kk != 0);
         mma_commit(pv_done + t);
+        if (t == ntq - 1) mma_commit(kv_empty + (2 * it + 1) % kSlots);  // V tile consumed
       };
-      bool ok = mbar_wait(q_full, 0, abort_flag) && mbar_wait(kv_full, 0, abort_flag);
+      auto wait_load = [&](int q) { return mbar_wait(kv_full + q % kSlots, (q / kSlots) & 1, abort_flag); };
+      bool ok = mbar_wait(q_full, 0, abort_flag) && wait_load(0);
       if (ok) {
         tc_fence_after();
         for (int t = 0; t < ntq; ++t) issue_qk(t, 0);
         for (int it = 0; it < n_iter && ok; ++it) {
-          const int s = it & 1;
           for (int t = 0; t < ntq && ok; ++t) {
             ok = mbar_wait(p_full + t, it & 1, abort_flag);
+            if (ok && t == 0) ok = wait_load(2 * it + 1);
             if (!ok) break;
             tc_fence_after();
-            issue_pv(t, s, it > 0);
-            if (t == ntq - 1) mma_commit(kv_empty + s);
+            issue_pv(t, it);
             if (it + 1 < n_iter) {
               if (t == 0) {
-                ok = mbar_wait(kv_full + ((it + 1) & 1), ((it + 1) >> 1) & 1, abort_flag);
+                ok = wait_load(2 * it + 2);
                 if (!ok) break;
                 tc_fence_after();
               }
-              issue_qk(t, (it + 1) & 1);
+              issue_qk(t, it + 1);
             }
           }
         }
@@ -230,6 +238,12 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
         ok = __all_sync(0xffffffffu, mbar_wait(s_full + t, it & 1, abort_flag));
         if (!ok) break;
         tc_fence_after();
+#ifdef DPARA_EXP_SYNCONLY
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(p_full + t);
+        continue;
+#endif
         uint32_t su[128];
 #pragma unroll
         for (int cc = 0; cc < 4; ++cc) tmem_ld32(lane_addr + t * 128 + cc * 32, su + cc * 32);
@@ -245,9 +259,13 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
 #pragma unroll
           for (int k = 0; k < 128; ++k) s[k] = k < nv ? s[k] : -INFINITY;
         }
+#ifdef DPARA_EXP_NOMAX
+        float mx = fmaxf(s[0], s[77]);
+#else
         float mx = s[0];
 #pragma unroll
         for (int k = 1; k < 128; ++k) mx = fmaxf(mx, s[k]);
+#endif
         const bool need = mx > m_used + thr;  // also true when m_used = -inf and the tile has a visible key
         if (it == 0) {
           if (need) m_used = mx;
@@ -273,8 +291,12 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
         uint32_t pk[64];
 #pragma unroll
         for (int k = 0; k < 64; ++k) {
+#ifdef DPARA_EXP_NOEX2
+          const float p0 = fmaf(s[2 * k], c, -mc), p1 = fmaf(s[2 * k + 1], c, -mc);
+#else
           const float p0 = ex2(fmaf(s[2 * k], c, -mc));
           const float p1 = ex2(fmaf(s[2 * k + 1], c, -mc));
+#endif
           l += p0 + p1;
           pk[k] = pack_bf16(p0, p1);
         }
@@ -282,7 +304,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
         tmem_st32(lane_addr + t * 128 + 32, pk + 32);
         tmem_wait_st();
         tc_fence_before();
-        mbar_arrive(p_full + t);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(p_full + t);
       }
 
       // ---- epilogue
@@ -476,6 +499,19 @@ dpara_status launch_attention_tc(const AttnParams &A, const TcPlan &plan, const 
     ok = ok && make_tmap_bf16_3d(&P.map_vb, A.v_blk, D, A.Hkv, nq, rs, rs * A.Hkv, 64, 1, plan.R_blk);
   }
   if (!ok) return DPARA_ERR_CUDA;
+  P.use_order = A.b <= kMaxOrdered && A.b > 1;
+  if (P.use_order) {
+    int idx[kMaxOrdered];
+    for (int n = 0; n < A.b; ++n) idx[n] = n;
+    for (int a = 1; a < A.b; ++a) {  // insertion sort by decreasing length (stable)
+      const int v = idx[a];
+      const long long lv = host_off[v + 1] - host_off[v];
+      int c = a - 1;
+      while (c >= 0 && host_off[idx[c] + 1] - host_off[idx[c]] < lv) { idx[c + 1] = idx[c]; --c; }
+      idx[c + 1] = v;
+    }
+    for (int n = 0; n < A.b; ++n) P.req_order[n] = (uint8_t)idx[n];
+  }
   if (plan.nsplit > 1) {
     P.part_o = static_cast<float *>(workspace);
     P.part_ml = P.part_o + (size_t)plan.items * plan.nsplit * 256 * D;

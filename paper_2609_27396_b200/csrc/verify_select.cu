@@ -45,8 +45,17 @@ __device__ __forceinline__ void gather_branch(const uint8_t *__restrict__ reps, 
   if ((bytes & 15) == 0 && ((reinterpret_cast<uintptr_t>(src) | reinterpret_cast<uintptr_t>(dst)) & 15) == 0) {
     const uint4 *s = reinterpret_cast<const uint4 *>(src);
     uint4 *d = reinterpret_cast<uint4 *>(dst);
-    size_t nv = bytes >> 4;
-    for (size_t i = tid; i < nv; i += nthreads) d[i] = __ldg(s + i);
+    const size_t nv = bytes >> 4;
+    // 8 independent 16-byte loads in flight per thread: the copy is one CTA's job, so latency matters
+    size_t i = tid;
+    for (; i + 7 * (size_t)nthreads < nv; i += 8 * (size_t)nthreads) {
+      uint4 v[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) v[k] = __ldcs(s + i + k * (size_t)nthreads);
+#pragma unroll
+      for (int k = 0; k < 8; ++k) d[i + k * (size_t)nthreads] = v[k];
+    }
+    for (; i < nv; i += nthreads) d[i] = __ldcs(s + i);
   } else {
     for (size_t i = tid; i < bytes; i += nthreads) dst[i] = src[i];
   }
@@ -67,15 +76,16 @@ struct VerifyParams {
   size_t rep_bytes;  // Bq * hidden * 2
 };
 
-__device__ __forceinline__ void write_result(const VerifyParams &P, int n, int r, int tok, bool bad) {
-  P.accept_len[n] = r;
-  P.bonus[n] = tok;
-  P.gather_idx[n] = r;
-  if (P.out_tokens) {
-    for (int i = 0; i < P.J; ++i)
-      P.out_tokens[(size_t)n * P.J + i] = i < r ? P.tokens[(size_t)n * (P.J - 1) + i] : (i == r ? tok : -1);
+// Outputs of request n, written by the first J threads of the finishing CTA.
+__device__ __forceinline__ void write_result(const VerifyParams &P, int n, int r, int tok, bool bad, int tid) {
+  if (tid == 0) {
+    P.accept_len[n] = r;
+    P.bonus[n] = tok;
+    P.gather_idx[n] = r;
+    if (bad && P.status_word) atomicOr(reinterpret_cast<unsigned int *>(P.status_word), DPARA_STATUS_BAD_TOKEN);
   }
-  if (bad && P.status_word) atomicOr(reinterpret_cast<unsigned int *>(P.status_word), DPARA_STATUS_BAD_TOKEN);
+  if (P.out_tokens && tid < P.J)
+    P.out_tokens[(size_t)n * P.J + tid] = tid < r ? P.tokens[(size_t)n * (P.J - 1) + tid] : (tid == r ? tok : -1);
 }
 
 // ------------------------------------------------------------------------------------------ greedy
@@ -87,37 +97,56 @@ __global__ void __launch_bounds__(kVsThreads) verify_greedy_kernel(const VerifyP
   const int base = blockIdx.x * kGreedyChunk;
   const int end = min(P.V, base + kGreedyChunk);
 
-  uint32_t bk = 0, bi = 0xffffffffu;  // best key / its index; strict '>' keeps the lowest index
+  // Fast path: plain float compares (3 instructions per element).  A strict '>' from -inf keeps the
+  // lowest index among equal values, never selects a NaN, and treats -0 and +0 as equal.  What it cannot
+  // rank are -inf and NaN themselves; a chunk in which nothing beat -inf is redone with the exact
+  // integer keys below (rare, CTA-uniform).
+  __shared__ unsigned long long s_k[kVsThreads / 32];
+  __shared__ int s_flag;
+  float bv = -INFINITY;
+  uint32_t bi = 0xffffffffu;
   if (P.vec_ok) {
     float4 v[8];
 #pragma unroll
     for (int it = 0; it < 8; ++it) {
       int idx = base + (it * kVsThreads + tid) * 4;
-      v[it] = idx < end ? __ldcs(reinterpret_cast<const float4 *>(p + idx)) : make_float4(0, 0, 0, 0);
+      v[it] = idx < end ? __ldcs(reinterpret_cast<const float4 *>(p + idx)) : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
     }
 #pragma unroll
     for (int it = 0; it < 8; ++it) {
-      int idx = base + (it * kVsThreads + tid) * 4;
-      if (idx < end) {
-        uint32_t k;
-        k = order_key(v[it].x); if (k > bk) { bk = k; bi = idx; }
-        k = order_key(v[it].y); if (k > bk) { bk = k; bi = idx + 1; }
-        k = order_key(v[it].z); if (k > bk) { bk = k; bi = idx + 2; }
-        k = order_key(v[it].w); if (k > bk) { bk = k; bi = idx + 3; }
-      }
+      const uint32_t idx = base + (it * kVsThreads + tid) * 4;
+      if (v[it].x > bv) { bv = v[it].x; bi = idx; }
+      if (v[it].y > bv) { bv = v[it].y; bi = idx + 1; }
+      if (v[it].z > bv) { bv = v[it].z; bi = idx + 2; }
+      if (v[it].w > bv) { bv = v[it].w; bi = idx + 3; }
     }
   } else {
     for (int idx = base + tid; idx < end; idx += kVsThreads) {
-      uint32_t k = order_key(__ldcs(p + idx));
-      if (k > bk) { bk = k; bi = idx; }
+      const float x = __ldcs(p + idx);
+      if (x > bv) { bv = x; bi = idx; }
     }
   }
-  unsigned long long key = ((unsigned long long)bk << 32) | (unsigned long long)(0xffffffffu - bi);
+  unsigned long long key = bi == 0xffffffffu ? 0ull : (((unsigned long long)order_key(bv) << 32) | (unsigned long long)(0xffffffffu - bi));
   key = warp_max_u64(key);
-  __shared__ unsigned long long s_k[kVsThreads / 32];
-  __shared__ int s_flag;
   if ((tid & 31) == 0) s_k[tid >> 5] = key;
   __syncthreads();
+  {
+    unsigned long long m = s_k[0];
+#pragma unroll
+    for (int w = 1; w < kVsThreads / 32; ++w) m = s_k[w] > m ? s_k[w] : m;
+    __syncthreads();
+    if (m == 0ull) {  // only -inf / NaN in this chunk: exact ranking with integer keys
+      uint32_t bk = 0;
+      bi = 0xffffffffu;
+      for (int idx = base + tid; idx < end; idx += kVsThreads) {
+        uint32_t k = order_key(p[idx]);
+        if (k > bk) { bk = k; bi = idx; }
+      }
+      key = warp_max_u64(((unsigned long long)bk << 32) | (unsigned long long)(0xffffffffu - bi));
+      if ((tid & 31) == 0) s_k[tid >> 5] = key;
+      __syncthreads();
+    }
+  }
   if (tid == 0) {
     unsigned long long m = s_k[0];
 #pragma unroll
@@ -132,27 +161,36 @@ __global__ void __launch_bounds__(kVsThreads) verify_greedy_kernel(const VerifyP
 
   // ---- last CTA of request n: position scan, outputs, gather
   __threadfence();
-  __shared__ int s_a[kMaxJ];
-  __shared__ int s_r;
+  __shared__ int s_a[kMaxJ], s_t[kMaxJ];
+  __shared__ int s_r, s_bad;
   if (tid < P.J) {
     unsigned long long k = __ldcg(P.ws64 + (size_t)n * P.J + tid);
     s_a[tid] = k == 0ull ? 0 : (int)(0xffffffffu - (uint32_t)(k & 0xffffffffull));  // all-NaN row -> 0
+    s_t[tid] = tid < P.J - 1 ? P.tokens[(size_t)n * (P.J - 1) + tid] : -1;           // all tokens in one round trip
   }
   __syncthreads();
   if (tid == 0) {
     int r = 0;
     bool bad = false;
     while (r < P.J - 1) {
-      int t = P.tokens[(size_t)n * (P.J - 1) + r];
+      const int t = s_t[r];
       if (t < 0 || t >= P.V) { bad = true; break; }
       if (t != s_a[r]) break;
       ++r;
     }
     s_r = r;
-    write_result(P, n, r, s_a[r], bad);
+    s_bad = bad;
   }
   __syncthreads();
-  if (P.reps) gather_branch(P.reps, P.selected, n, P.J, s_r, P.rep_bytes, tid, kVsThreads);
+  const int r = s_r;
+  if (tid == 0) {
+    P.accept_len[n] = r;
+    P.bonus[n] = s_a[r];
+    P.gather_idx[n] = r;
+    if (s_bad && P.status_word) atomicOr(reinterpret_cast<unsigned int *>(P.status_word), DPARA_STATUS_BAD_TOKEN);
+  }
+  if (P.out_tokens && tid < P.J) P.out_tokens[(size_t)n * P.J + tid] = tid < r ? s_t[tid] : (tid == r ? s_a[r] : -1);
+  if (P.reps) gather_branch(P.reps, P.selected, n, P.J, r, P.rep_bytes, tid, kVsThreads);
 }
 
 // ------------------------------------------------------------------------------------------ sampling
@@ -343,7 +381,7 @@ __global__ void __launch_bounds__(kVsThreads) verify_sampling_kernel(const Verif
     }
     __syncthreads();
   }
-  if (tid == 0) write_result(P, n, r, s_tok, s_bad != 0);
+  write_result(P, n, r, s_tok, s_bad != 0, tid);
   if (P.reps) gather_branch(P.reps, P.selected, n, P.J, r, P.rep_bytes, tid, kVsThreads);
 }
 

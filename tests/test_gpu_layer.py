@@ -1,7 +1,8 @@
 """GPU parity of the full backbone block (dpara_draft_all_boundaries with a layer) against the oracle's
 block, boundary by boundary.
 
-Bound on the fp32 output y: |delta| <= 1e-2 * max(1, |y|), i.e. the stated 1e-2 at unit scale.  Derivation:
+Bound on the fp32 output y: |delta| <= 1e-2 * max(1, rms(y)), i.e. the stated 1e-2 at unit scale (the error
+is additive noise of the down projection, independent of the element's own size).  Derivation:
 the oracle mirrors the block's bf16 rounding points, but the tensor-core attention rounds probabilities to
 bf16 before the PV product, so its output differs from the oracle's by ~1e-3 relative; that flips the bf16
 rounding of `a` on a large share of elements, which perturbs h1 by ~3e-5, flips ~1 % of the bf16 `hn`
@@ -80,5 +81,5 @@ def test_cfg5_full_size_sampled_boundaries():
     for (n, j) in sorted(picks):
         ref = orc.boundary(n, j)["y"].astype(np.float64)
         d = np.abs(y[n, j] - ref)
-        assert np.all(d <= TOL * np.maximum(1.0, np.abs(ref))), (n, j, float(d.max()))
+        assert np.all(d <= TOL * max(1.0, float(np.sqrt((ref * ref).mean())))), (n, j, float(d.max()))
         assert np.sqrt((d * d).mean()) <= 5e-3
