@@ -26,7 +26,7 @@ namespace dpara {
 using namespace ptx;
 
 namespace {
-constexpr int kThreads = 320;
+constexpr int kThreads = 384;  // warps 0-7 softmax, 8 TMA producer, 9 MMA issuer, 10-11 idle (complete the third warpgroup)
 constexpr float kRescaleLog2 = 8.0f;
 constexpr int kMaxOrdered = 128;
 }  // namespace
@@ -34,7 +34,7 @@ constexpr int kMaxOrdered = 128;
 struct TcParams {
   CUtensorMap map_q, map_kc, map_vc, map_ks, map_vs, map_kb, map_vb;
   AttnParams a;
-  int JI_T, n_ji, n_tiles, n_pairs, nsplit, S8, R_blk, has_blk, has_tail;
+  int JI_T, n_ji, n_tiles, n_pairs, nsplit, S8, R_blk, has_blk, has_tail, n_items;
   float *part_o;   // [item][2][128][D]
   float *part_ml;  // [item][2][128][2]
   float c_log2;    // softmax scale * log2(e)
@@ -56,6 +56,39 @@ struct TcCfg {
   static constexpr int kOBase = 256;                    // TMEM column of O0
 };
 
+// One unit of work of a persistent CTA.
+struct Item {
+  int n, g, pair, split, ntq, L, t0, t1, nctx, n_ctx_it, n_iter, jb0, slot;
+  long long c0;
+  bool do_tail;
+};
+
+__device__ __forceinline__ Item decode_item(const TcParams &P, int id) {
+  const AttnParams &A = P.a;
+  Item I;
+  const int X = P.n_pairs * P.nsplit;
+  const int x = id % X, y = (id / X) % A.Hkv, z = id / (X * A.Hkv);
+  I.n = P.use_order ? (int)P.req_order[z] : z;
+  I.g = y;
+  I.pair = x / P.nsplit;
+  I.split = x % P.nsplit;
+  I.ntq = min(2, P.n_tiles - I.pair * 2);
+  I.c0 = A.ctx_offsets[I.n];
+  I.L = (int)(A.ctx_offsets[I.n + 1] - I.c0);
+  I.nctx = (I.L + 127) >> 7;
+  I.t0 = (int)((long long)I.split * I.nctx / P.nsplit);
+  I.t1 = (int)((long long)(I.split + 1) * I.nctx / P.nsplit);
+  I.n_ctx_it = I.t1 - I.t0;
+  I.do_tail = P.has_tail && I.split == P.nsplit - 1;
+  I.n_iter = I.n_ctx_it + (I.do_tail ? 1 : 0);
+  I.jb0 = A.lo + (I.pair * 2 * P.JI_T) / A.Bq;  // first boundary whose block keys sit in the tail tile
+  I.slot = ((I.n * A.Hkv + I.g) * P.n_pairs + I.pair) * P.nsplit + I.split;
+  return I;
+}
+
+// Persistent kernel: CTA c works through items c, c + gridDim.x, ... of the (longest request first) item
+// list; barrier phases and the K/V slot ring run on across items, so the producer already streams the next
+// item's Q/K/V while the softmax warps write the previous item's output.
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_constant__ TcParams P) {
   using Cfg = TcCfg<D>;
@@ -66,52 +99,18 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
   uint8_t *sKV = smem + 2 * Cfg::kTileBytes;            // ring of K / V tile slots
   constexpr int kSlots = Cfg::kSlots;
   uint64_t *bars = reinterpret_cast<uint64_t *>(sKV + kSlots * Cfg::kTileBytes);
-  uint64_t *kv_full = bars, *kv_empty = bars + kSlots, *q_full = bars + 2 * kSlots, *s_full = q_full + 1, *p_full = q_full + 3,
-           *pv_done = q_full + 5;
-  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(q_full + 7);
+  uint64_t *kv_full = bars, *kv_empty = bars + kSlots, *q_full = bars + 2 * kSlots, *q_empty = q_full + 1, *s_full = q_full + 2,
+           *p_full = q_full + 4, *pv_done = q_full + 6;
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(q_full + 8);
   volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int n = P.use_order ? (int)P.req_order[blockIdx.z] : (int)blockIdx.z, g = blockIdx.y;
-  const int pair = blockIdx.x / P.nsplit, split = blockIdx.x % P.nsplit;
-  const int ntq = min(2, P.n_tiles - pair * 2);
-  const long long c0 = A.ctx_offsets[n];
-  const int L = (int)(A.ctx_offsets[n + 1] - c0);
-  const int nctx = (L + 127) >> 7;
-  const int t0 = (int)((long long)split * nctx / P.nsplit), t1 = (int)((long long)(split + 1) * nctx / P.nsplit);
-  const int n_ctx_it = t1 - t0;
-  const bool do_tail = P.has_tail && split == P.nsplit - 1;
-  const int n_iter = n_ctx_it + (do_tail ? 1 : 0);
-  const int item = ((n * A.Hkv + g) * P.n_pairs + pair) * P.nsplit + split;
-  const int jb0 = A.lo + (pair * 2 * P.JI_T) / A.Bq;    // first boundary whose block keys sit in the tail tile
-
   if (A.status_word && (*reinterpret_cast<volatile int32_t *>(A.status_word) & (int32_t)DPARA_STATUS_TIMEOUT)) return;
-
-  if (n_iter == 0) {  // nothing visible to this work item
-    for (int r = threadIdx.x; r < 256; r += kThreads) {
-      if (P.nsplit > 1) {
-        P.part_ml[((size_t)item * 256 + r) * 2] = -INFINITY;
-        P.part_ml[((size_t)item * 256 + r) * 2 + 1] = 0.f;
-      } else {
-        const int t = r >> 7, rr = r & 127;
-        const int ji = (pair * 2 + t) * P.JI_T + rr / A.G;
-        if (t < ntq && rr < P.JI_T * A.G && ji < P.n_ji) {
-          const int j = A.lo + ji / A.Bq, i = ji % A.Bq, h = g * A.G + rr % A.G;
-          const size_t o = ((((size_t)n * A.J + j) * A.Bq + i) * A.Hq + h);
-          for (int d = 0; d < D; ++d) {
-            if (A.out_f32) static_cast<float *>(A.out)[o * D + d] = 0.f;
-            else static_cast<uint16_t *>(A.out)[o * D + d] = 0;
-          }
-          if (A.out_lse) A.out_lse[o] = -INFINITY;
-        }
-      }
-    }
-    return;
-  }
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kSlots; ++s) { mbar_init(kv_full + s, 1); mbar_init(kv_empty + s, 1); }
     mbar_init(q_full, 1);
+    mbar_init(q_empty, 1);
     for (int t = 0; t < 2; ++t) { mbar_init(s_full + t, 1); mbar_init(p_full + t, 4); mbar_init(pv_done + t, 1); }
     *abort_flag = 0;
     fence_barrier_init();
@@ -122,155 +121,209 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
 
+  // register budget: the softmax warpgroups need the registers (a 128-wide score row per thread), the
+  // producer / MMA warpgroup almost none
+  if (warp >= 8) {
+  asm volatile("setmaxnreg.dec.sync.aligned.u32 96;");
   if (warp == 8) {
     // ------------------------------------------------------------------ producer
     if (lane == 0) {
       prefetch_tensormap(&P.map_q);
-      if (L > 0) { prefetch_tensormap(&P.map_kc); prefetch_tensormap(&P.map_vc); }
-      const int qrow0 = (n * A.J + A.lo) * A.Bq + pair * 2 * P.JI_T;
-      mbar_arrive_expect_tx(q_full, (uint32_t)(ntq * P.JI_T * A.G * 128 * Cfg::kSlabs));
-      for (int t = 0; t < ntq; ++t)
-        for (int sl = 0; sl < Cfg::kSlabs; ++sl)
-          tma_load_3d(sQ + t * Cfg::kTileBytes + sl * Cfg::kSlabBytes, &P.map_q, q_full, sl * 64, g * A.G, qrow0 + t * P.JI_T);
     }
-    // load q = 2 it is the K tile of iteration it, load 2 it + 1 its V tile; slot = q % kSlots
-    for (int q = 0; q < 2 * n_iter; ++q) {
-      const int it = q >> 1, is_v = q & 1;
-      const int sl = q % kSlots;
-      const uint32_t ph = (q / kSlots) & 1;
-      if (!__all_sync(0xffffffffu, mbar_wait(kv_empty + sl, ph ^ 1u, abort_flag))) break;
-      uint8_t *dst = sKV + sl * Cfg::kTileBytes;
-      if (it < n_ctx_it) {
-        if (lane == 0) {
-          const int row = (int)(c0 + (long long)(t0 + it) * 128);
-          mbar_arrive_expect_tx(kv_full + sl, Cfg::kTileBytes);
+    int ld = 0, k = 0;  // running K/V load counter, processed-item counter
+    bool ok = true;
+    for (int id = blockIdx.x; id < P.n_items && ok; id += gridDim.x) {
+      const Item I = decode_item(P, id);
+      if (I.n_iter == 0) continue;
+      // the Q buffer is free once the previous item's last QK has completed
+      ok = __all_sync(0xffffffffu, mbar_wait(q_empty, (k & 1) ^ 1u, abort_flag));
+      if (!ok) break;
+      if (lane == 0) {
+        const int qrow0 = (I.n * A.J + A.lo) * A.Bq + I.pair * 2 * P.JI_T;
+        mbar_arrive_expect_tx(q_full, (uint32_t)(I.ntq * P.JI_T * A.G * 128 * Cfg::kSlabs));
+        for (int t = 0; t < I.ntq; ++t)
           for (int sb = 0; sb < Cfg::kSlabs; ++sb)
-            tma_load_3d(dst + sb * Cfg::kSlabBytes, is_v ? &P.map_vc : &P.map_kc, kv_full + sl, sb * 64, g, row);
-        }
-      } else {
-        if (is_v) {
-          // tail tile: rows the TMA boxes do not cover must still hold finite V (P = 0 there): clear the V tile
-          for (int o = lane * 16; o < Cfg::kTileBytes; o += 32 * 16) *reinterpret_cast<uint4 *>(dst + o) = make_uint4(0, 0, 0, 0);
-          fence_proxy_async();
-          __syncwarp();
-        }
-        if (lane == 0) {
-          uint32_t bytes = 0;
-          if (A.S > 0) bytes += (uint32_t)A.S * 128 * Cfg::kSlabs;
-          if (P.has_blk) bytes += (uint32_t)P.R_blk * 128 * Cfg::kSlabs;
-          mbar_arrive_expect_tx(kv_full + sl, bytes);
-          for (int sb = 0; sb < Cfg::kSlabs; ++sb) {
-            if (A.S > 0) tma_load_3d(dst + sb * Cfg::kSlabBytes, is_v ? &P.map_vs : &P.map_ks, kv_full + sl, sb * 64, g, n * A.S);
-            if (P.has_blk)
-              tma_load_3d(dst + sb * Cfg::kSlabBytes + P.S8 * 128, is_v ? &P.map_vb : &P.map_kb, kv_full + sl, sb * 64, g,
-                          (n * A.J + jb0) * A.Bq);
-          }
-        }
+            tma_load_3d(sQ + t * Cfg::kTileBytes + sb * Cfg::kSlabBytes, &P.map_q, q_full, sb * 64, I.g * A.G, qrow0 + t * P.JI_T);
       }
-    }
-  } else if (warp == 9) {
-    // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      constexpr uint32_t idesc_qk = idesc_bf16_f32(128, 128, false, false);
-      constexpr uint32_t idesc_pv = idesc_bf16_f32(128, D, false, true);
-      const uint32_t q_addr = smem_u32(sQ), kv_addr = smem_u32(sKV);
-      auto issue_qk = [&](int t, int it) {
-        const uint32_t qa = q_addr + t * Cfg::kTileBytes, ka = kv_addr + ((2 * it) % kSlots) * Cfg::kTileBytes;
-#pragma unroll
-        for (int kk = 0; kk < D / 16; ++kk) {
-          const uint32_t off = (kk >> 2) * Cfg::kSlabBytes + (kk & 3) * 32;
-          mma_ss(tmem + t * 128, smem_desc_sw128(qa + off, 16, 1024), smem_desc_sw128(ka + off, 16, 1024), idesc_qk, kk != 0);
-        }
-        mma_commit(s_full + t);
-        if (t == ntq - 1) mma_commit(kv_empty + (2 * it) % kSlots);      // K tile consumed by every query tile
-      };
-      auto issue_pv = [&](int t, int it) {
-        const uint32_t va = kv_addr + ((2 * it + 1) % kSlots) * Cfg::kTileBytes;
-#pragma unroll
-        for (int kk = 0; kk < 8; ++kk)
-          mma_ts(tmem + Cfg::kOBase + t * D, tmem + t * 128 + kk * 8, smem_desc_sw128(va + kk * 2048, Cfg::kSlabBytes, 1024),
-                 idesc_pv, it > 0 || kk != 0);
-        mma_commit(pv_done + t);
-        if (t == ntq - 1) mma_commit(kv_empty + (2 * it + 1) % kSlots);  // V tile consumed
-      };
-      auto wait_load = [&](int q) { return mbar_wait(kv_full + q % kSlots, (q / kSlots) & 1, abort_flag); };
-      bool ok = mbar_wait(q_full, 0, abort_flag) && wait_load(0);
-      if (ok) {
-        tc_fence_after();
-        for (int t = 0; t < ntq; ++t) issue_qk(t, 0);
-        for (int it = 0; it < n_iter && ok; ++it) {
-          for (int t = 0; t < ntq && ok; ++t) {
-            ok = mbar_wait(p_full + t, it & 1, abort_flag);
-            if (ok && t == 0) ok = wait_load(2 * it + 1);
-            if (!ok) break;
-            tc_fence_after();
-            issue_pv(t, it);
-            if (it + 1 < n_iter) {
-              if (t == 0) {
-                ok = wait_load(2 * it + 2);
-                if (!ok) break;
-                tc_fence_after();
-              }
-              issue_qk(t, it + 1);
+      // load q = 2 it is the K tile of iteration it, load 2 it + 1 its V tile; slot = (ld + q) % kSlots
+      for (int q = 0; q < 2 * I.n_iter; ++q) {
+        const int it = q >> 1, is_v = q & 1;
+        const int sl = (ld + q) % kSlots;
+        const uint32_t ph = ((ld + q) / kSlots) & 1;
+        ok = __all_sync(0xffffffffu, mbar_wait(kv_empty + sl, ph ^ 1u, abort_flag));
+        if (!ok) break;
+        uint8_t *dst = sKV + sl * Cfg::kTileBytes;
+        if (it < I.n_ctx_it) {
+          if (lane == 0) {
+            const int row = (int)(I.c0 + (long long)(I.t0 + it) * 128);
+            mbar_arrive_expect_tx(kv_full + sl, Cfg::kTileBytes);
+            for (int sb = 0; sb < Cfg::kSlabs; ++sb)
+              tma_load_3d(dst + sb * Cfg::kSlabBytes, is_v ? &P.map_vc : &P.map_kc, kv_full + sl, sb * 64, I.g, row);
+          }
+        } else {
+          if (is_v) {
+            // tail tile: rows the TMA boxes do not cover must still hold finite V (P = 0 there): clear the V tile
+            for (int o = lane * 16; o < Cfg::kTileBytes; o += 32 * 16) *reinterpret_cast<uint4 *>(dst + o) = make_uint4(0, 0, 0, 0);
+            fence_proxy_async();
+            __syncwarp();
+          }
+          if (lane == 0) {
+            uint32_t bytes = 0;
+            if (A.S > 0) bytes += (uint32_t)A.S * 128 * Cfg::kSlabs;
+            if (P.has_blk) bytes += (uint32_t)P.R_blk * 128 * Cfg::kSlabs;
+            mbar_arrive_expect_tx(kv_full + sl, bytes);
+            for (int sb = 0; sb < Cfg::kSlabs; ++sb) {
+              if (A.S > 0) tma_load_3d(dst + sb * Cfg::kSlabBytes, is_v ? &P.map_vs : &P.map_ks, kv_full + sl, sb * 64, I.g, I.n * A.S);
+              if (P.has_blk)
+                tma_load_3d(dst + sb * Cfg::kSlabBytes + P.S8 * 128, is_v ? &P.map_vb : &P.map_kb, kv_full + sl, sb * 64, I.g,
+                            (I.n * A.J + I.jb0) * A.Bq);
             }
           }
         }
       }
+      ld += 2 * I.n_iter;
+      ++k;
     }
-  } else {
-    // ------------------------------------------------------------------ softmax + epilogue: thread = row
-    const int t = warp >> 2;
-    if (t < ntq) {
-      const int wq = warp & 3;
-      const int r = wq * 32 + lane;
-      const uint32_t lane_addr = tmem + ((uint32_t)(wq * 32) << 16);
-      const int ji = (pair * 2 + t) * P.JI_T + r / A.G;
-      const bool valid = (r < P.JI_T * A.G) && (ji < P.n_ji);
-      const int j = A.lo + ji / A.Bq, i = ji % A.Bq, h = g * A.G + r % A.G;
-      const int na = max(0, min(j + A.pb, A.S));
-      const int b0 = P.has_blk ? P.S8 + (j - jb0) * A.Bq : 0, b1 = P.has_blk ? b0 + A.Bq : 0;
-      const float c = P.c_log2;
-      const float thr = kRescaleLog2 / c;
-      float m_used = -INFINITY, l = 0.f;
+  } else if (warp == 9) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      // The issuing thread is on the critical path of every tile, so its instruction count matters:
+      // descriptors are built once and advanced with plain adds (the address field counts 16-byte units),
+      // ring slots and phases are tracked incrementally (no divisions).
+      constexpr uint32_t idesc_qk = idesc_bf16_f32(128, 128, false, false);
+      constexpr uint32_t idesc_pv = idesc_bf16_f32(128, D, false, true);
+      constexpr uint32_t kTile16 = Cfg::kTileBytes >> 4;
+      const uint64_t qdesc[2] = {smem_desc_sw128(smem_u32(sQ), 16, 1024), smem_desc_sw128(smem_u32(sQ) + Cfg::kTileBytes, 16, 1024)};
+      const uint64_t kdesc0 = smem_desc_sw128(smem_u32(sKV), 16, 1024);                 // K tile: K-major operand
+      const uint64_t vdesc0 = smem_desc_sw128(smem_u32(sKV), Cfg::kSlabBytes, 1024);    // V tile: MN-major operand
+      int ring_slot = 0, k = 0;
+      uint32_t ring_phase = 0, ph_p[2] = {0, 0};
       bool ok = true;
-
-      for (int it = 0; it < n_iter; ++it) {
-        ok = __all_sync(0xffffffffu, mbar_wait(s_full + t, it & 1, abort_flag));
+      auto next_load = [&](int &slot_out) {  // wait for the next tile of the K/V ring (loads are consumed in order)
+        slot_out = ring_slot;
+        const bool r = mbar_wait(kv_full + ring_slot, ring_phase, abort_flag);
+        if (++ring_slot == kSlots) { ring_slot = 0; ring_phase ^= 1u; }
+        return r;
+      };
+      for (int id = blockIdx.x; id < P.n_items && ok; id += gridDim.x) {
+        const Item I = decode_item(P, id);
+        if (I.n_iter == 0) continue;
+        const int ntq = I.ntq, n_iter = I.n_iter;
+        auto issue_qk = [&](int t, int kslot, bool last_it) {
+          const uint64_t qa = qdesc[t], ka = kdesc0 + (uint64_t)(kslot * kTile16);
+#pragma unroll
+          for (int kk = 0; kk < D / 16; ++kk) {
+            const uint32_t off = ((kk >> 2) * Cfg::kSlabBytes + (kk & 3) * 32) >> 4;
+            if (kk == 0) mma_ss_c<false>(tmem + t * 128, qa + off, ka + off, idesc_qk);
+            else mma_ss_c<true>(tmem + t * 128, qa + off, ka + off, idesc_qk);
+          }
+          mma_commit(s_full + t);
+          if (t == ntq - 1) {
+            mma_commit(kv_empty + kslot);           // K tile consumed by every query tile
+            if (last_it) mma_commit(q_empty);       // last use of this item's Q tiles
+          }
+        };
+        auto issue_pv = [&](int t, int vslot, bool acc) {
+          const uint64_t va = vdesc0 + (uint64_t)(vslot * kTile16);
+          const uint32_t o_t = tmem + Cfg::kOBase + t * D, p_t = tmem + t * 128;
+          mma_ts(o_t, p_t, va, idesc_pv, acc);
+#pragma unroll
+          for (int kk = 1; kk < 8; ++kk) mma_ts_c<true>(o_t, p_t + kk * 8, va + (uint64_t)(kk * (2048 >> 4)), idesc_pv);
+          mma_commit(pv_done + t);
+          if (t == ntq - 1) mma_commit(kv_empty + vslot);  // V tile consumed
+        };
+        int kslot = 0, vslot = 0;
+        ok = mbar_wait(q_full, k & 1, abort_flag) && next_load(kslot);
         if (!ok) break;
         tc_fence_after();
-#ifdef DPARA_EXP_SYNCONLY
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(p_full + t);
+        for (int t = 0; t < ntq; ++t) issue_qk(t, kslot, n_iter == 1);
+        for (int it = 0; it < n_iter && ok; ++it) {
+          const bool more = it + 1 < n_iter;
+          for (int t = 0; t < ntq && ok; ++t) {
+            ok = mbar_wait(p_full + t, ph_p[t], abort_flag);
+            ph_p[t] ^= 1u;
+            if (ok && t == 0) ok = next_load(vslot);
+            if (!ok) break;
+            tc_fence_after();
+            issue_pv(t, vslot, it > 0);
+            if (more) {
+              if (t == 0) {
+                ok = next_load(kslot);
+                if (!ok) break;
+                tc_fence_after();
+              }
+              issue_qk(t, kslot, it + 2 == n_iter);
+            }
+          }
+        }
+        ++k;
+      }
+    }
+  }
+  } else {
+    // ------------------------------------------------------------------ softmax + epilogue: thread = row
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 200;");
+    const int t = warp >> 2;
+    const int wq = warp & 3;
+    const int r = wq * 32 + lane;
+    const uint32_t lane_addr = tmem + ((uint32_t)(wq * 32) << 16);
+    const float c = P.c_log2;
+    const float thr = kRescaleLog2 / c;
+    int cnt = 0;  // iterations this tile's barriers have been through
+    bool ok = true;
+    for (int id = blockIdx.x; id < P.n_items && ok; id += gridDim.x) {
+      const Item I = decode_item(P, id);
+      const int ji = (I.pair * 2 + t) * P.JI_T + r / A.G;
+      const bool valid = (t < I.ntq) && (r < P.JI_T * A.G) && (ji < P.n_ji);
+      const int j = A.lo + ji / A.Bq, i = ji % A.Bq, h = I.g * A.G + r % A.G;
+      const size_t orow = (((size_t)I.n * A.J + j) * A.Bq + i) * A.Hq + h;
+      const size_t pslot = (((size_t)I.slot * 2 + t) * 128 + r);
+      if (I.n_iter == 0 || t >= I.ntq) {
+        // nothing visible to this work item, or no second tile in the last pair
+        if (P.nsplit > 1) {
+          P.part_ml[pslot * 2] = -INFINITY;
+          P.part_ml[pslot * 2 + 1] = 0.f;
+        } else if (valid) {
+          for (int d = 0; d < D; ++d) {
+            if (A.out_f32) static_cast<float *>(A.out)[orow * D + d] = 0.f;
+            else static_cast<uint16_t *>(A.out)[orow * D + d] = 0;
+          }
+          if (A.out_lse) A.out_lse[orow] = -INFINITY;
+        }
         continue;
-#endif
+      }
+      const int n_iter = I.n_iter;
+      const int na = max(0, min(j + A.pb, A.S));
+      const int b0 = P.has_blk ? P.S8 + (j - I.jb0) * A.Bq : 0, b1 = P.has_blk ? b0 + A.Bq : 0;
+      float m_used = -INFINITY, l = 0.f;
+
+      for (int it = 0; it < n_iter; ++it) {
+        ok = __all_sync(0xffffffffu, mbar_wait(s_full + t, (cnt + it) & 1, abort_flag));
+        if (!ok) break;
+        tc_fence_after();
         uint32_t su[128];
 #pragma unroll
         for (int cc = 0; cc < 4; ++cc) tmem_ld32(lane_addr + t * 128 + cc * 32, su + cc * 32);
         tmem_wait_ld();
         float s[128];
 #pragma unroll
-        for (int k = 0; k < 128; ++k) s[k] = __uint_as_float(su[k]);
-        if (it >= n_ctx_it) {
+        for (int kx = 0; kx < 128; ++kx) s[kx] = __uint_as_float(su[kx]);
+        if (it >= I.n_ctx_it) {
 #pragma unroll
-          for (int k = 0; k < 128; ++k) s[k] = ((k < na) || (k >= b0 && k < b1)) ? s[k] : -INFINITY;
-        } else if (it == n_ctx_it - 1 && t1 == nctx && (L & 127)) {
-          const int nv = L & 127;
+          for (int kx = 0; kx < 128; ++kx) s[kx] = ((kx < na) || (kx >= b0 && kx < b1)) ? s[kx] : -INFINITY;
+        } else if (it == I.n_ctx_it - 1 && I.t1 == I.nctx && (I.L & 127)) {
+          const int nv = I.L & 127;
 #pragma unroll
-          for (int k = 0; k < 128; ++k) s[k] = k < nv ? s[k] : -INFINITY;
+          for (int kx = 0; kx < 128; ++kx) s[kx] = kx < nv ? s[kx] : -INFINITY;
         }
-#ifdef DPARA_EXP_NOMAX
-        float mx = fmaxf(s[0], s[77]);
-#else
-        float mx = s[0];
+        float mx = fmaxf(s[0], s[1]);
 #pragma unroll
-        for (int k = 1; k < 128; ++k) mx = fmaxf(mx, s[k]);
-#endif
+        for (int kx = 2; kx < 128; kx += 2) mx = max3(mx, s[kx], s[kx + 1]);
         const bool need = mx > m_used + thr;  // also true when m_used = -inf and the tile has a visible key
         if (it == 0) {
           if (need) m_used = mx;
         } else if (__any_sync(0xffffffffu, need)) {
-          ok = __all_sync(0xffffffffu, mbar_wait(pv_done + t, (it - 1) & 1, abort_flag));
+          ok = __all_sync(0xffffffffu, mbar_wait(pv_done + t, (cnt + it - 1) & 1, abort_flag));
           if (!ok) break;
           tc_fence_after();
           const float f = need ? ex2((m_used - mx) * c) : 1.0f;
@@ -280,7 +333,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
             tmem_ld32(lane_addr + Cfg::kOBase + t * D + cc * 32, o);
             tmem_wait_ld();
 #pragma unroll
-            for (int k = 0; k < 32; ++k) o[k] = __float_as_uint(__uint_as_float(o[k]) * f);
+            for (int kx = 0; kx < 32; ++kx) o[kx] = __float_as_uint(__uint_as_float(o[kx]) * f);
             tmem_st32(lane_addr + Cfg::kOBase + t * D + cc * 32, o);
           }
           tmem_wait_st();
@@ -289,16 +342,21 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
         }
         const float mc = (m_used == -INFINITY ? 0.f : m_used) * c;
         uint32_t pk[64];
+        {
+          // packed fp32x2 scale/shift and row sum (half the FMA/ADD issue slots of the scalar form)
+          const uint64_t c2 = pack2(c, c), nmc2 = pack2(-mc, -mc);
+          uint64_t l2 = pack2(0.f, 0.f);
 #pragma unroll
-        for (int k = 0; k < 64; ++k) {
-#ifdef DPARA_EXP_NOEX2
-          const float p0 = fmaf(s[2 * k], c, -mc), p1 = fmaf(s[2 * k + 1], c, -mc);
-#else
-          const float p0 = ex2(fmaf(s[2 * k], c, -mc));
-          const float p1 = ex2(fmaf(s[2 * k + 1], c, -mc));
-#endif
-          l += p0 + p1;
-          pk[k] = pack_bf16(p0, p1);
+          for (int kx = 0; kx < 64; ++kx) {
+            float x0, x1;
+            unpack2(fma2(pack2(s[2 * kx], s[2 * kx + 1]), c2, nmc2), x0, x1);
+            const float p0 = ex2(x0), p1 = ex2(x1);
+            l2 = add2(l2, pack2(p0, p1));
+            pk[kx] = pack_bf16(p0, p1);
+          }
+          float la, lb;
+          unpack2(l2, la, lb);
+          l += la + lb;
         }
         tmem_st32(lane_addr + t * 128, pk);
         tmem_st32(lane_addr + t * 128 + 32, pk + 32);
@@ -308,55 +366,50 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
         if (lane == 0) mbar_arrive(p_full + t);
       }
 
-      // ---- epilogue
-      if (ok) ok = __all_sync(0xffffffffu, mbar_wait(pv_done + t, (n_iter - 1) & 1, abort_flag));
-      if (ok) {
-        tc_fence_after();
-        const size_t orow = (((size_t)n * A.J + j) * A.Bq + i) * A.Hq + h;
-        const float inv = l > 0.f ? 1.0f / l : 0.f;
+      // ---- epilogue of this item (the MMA issuer cannot touch O_t again before this tile's next p_full arrive)
+      if (ok) ok = __all_sync(0xffffffffu, mbar_wait(pv_done + t, (cnt + n_iter - 1) & 1, abort_flag));
+      if (!ok) break;
+      tc_fence_after();
+      const float inv = l > 0.f ? 1.0f / l : 0.f;
 #pragma unroll 1
-        for (int cc = 0; cc < D / 32; ++cc) {
-          uint32_t o[32];
-          tmem_ld32(lane_addr + Cfg::kOBase + t * D + cc * 32, o);
-          tmem_wait_ld();
-          if (P.nsplit > 1) {
-            float4 *dst = reinterpret_cast<float4 *>(P.part_o + (((size_t)item * 2 + t) * 128 + r) * D + cc * 32);
+      for (int cc = 0; cc < D / 32; ++cc) {
+        uint32_t o[32];
+        tmem_ld32(lane_addr + Cfg::kOBase + t * D + cc * 32, o);
+        tmem_wait_ld();
+        if (P.nsplit > 1) {
+          float4 *dst = reinterpret_cast<float4 *>(P.part_o + pslot * D + cc * 32);
+#pragma unroll
+          for (int v = 0; v < 8; ++v)
+            dst[v] = make_float4(__uint_as_float(o[4 * v]), __uint_as_float(o[4 * v + 1]), __uint_as_float(o[4 * v + 2]),
+                                 __uint_as_float(o[4 * v + 3]));
+        } else if (valid) {
+          if (A.out_f32) {
+            float4 *dst = reinterpret_cast<float4 *>(static_cast<float *>(A.out) + orow * D + cc * 32);
 #pragma unroll
             for (int v = 0; v < 8; ++v)
-              dst[v] = make_float4(__uint_as_float(o[4 * v]), __uint_as_float(o[4 * v + 1]), __uint_as_float(o[4 * v + 2]),
-                                   __uint_as_float(o[4 * v + 3]));
-          } else if (valid) {
-            if (A.out_f32) {
-              float4 *dst = reinterpret_cast<float4 *>(static_cast<float *>(A.out) + orow * D + cc * 32);
+              dst[v] = make_float4(__uint_as_float(o[4 * v]) * inv, __uint_as_float(o[4 * v + 1]) * inv,
+                                   __uint_as_float(o[4 * v + 2]) * inv, __uint_as_float(o[4 * v + 3]) * inv);
+          } else {
+            uint4 *dst = reinterpret_cast<uint4 *>(static_cast<uint16_t *>(A.out) + orow * D + cc * 32);
 #pragma unroll
-              for (int v = 0; v < 8; ++v)
-                dst[v] = make_float4(__uint_as_float(o[4 * v]) * inv, __uint_as_float(o[4 * v + 1]) * inv,
-                                     __uint_as_float(o[4 * v + 2]) * inv, __uint_as_float(o[4 * v + 3]) * inv);
-            } else {
-              uint4 *dst = reinterpret_cast<uint4 *>(static_cast<uint16_t *>(A.out) + orow * D + cc * 32);
+            for (int v = 0; v < 4; ++v) {
+              uint32_t w[4];
 #pragma unroll
-              for (int v = 0; v < 4; ++v) {
-                uint32_t w[4];
-#pragma unroll
-                for (int e = 0; e < 4; ++e)
-                  w[e] = pack_bf16(__uint_as_float(o[8 * v + 2 * e]) * inv, __uint_as_float(o[8 * v + 2 * e + 1]) * inv);
-                dst[v] = make_uint4(w[0], w[1], w[2], w[3]);
-              }
+              for (int e = 0; e < 4; ++e)
+                w[e] = pack_bf16(__uint_as_float(o[8 * v + 2 * e]) * inv, __uint_as_float(o[8 * v + 2 * e + 1]) * inv);
+              dst[v] = make_uint4(w[0], w[1], w[2], w[3]);
             }
           }
         }
-        if (P.nsplit > 1) {
-          P.part_ml[(((size_t)item * 2 + t) * 128 + r) * 2] = m_used;
-          P.part_ml[(((size_t)item * 2 + t) * 128 + r) * 2 + 1] = l;
-        } else if (valid && A.out_lse) {
-          A.out_lse[orow] = l > 0.f ? (m_used * c + log2f(l)) * 0.6931471805599453f : -INFINITY;
-        }
       }
-    } else if (P.nsplit > 1) {
-      // absent second tile of the last pair: its partial slots must read as empty
-      const int r = (warp & 3) * 32 + lane;
-      P.part_ml[(((size_t)item * 2 + 1) * 128 + r) * 2] = -INFINITY;
-      P.part_ml[(((size_t)item * 2 + 1) * 128 + r) * 2 + 1] = 0.f;
+      tc_fence_before();  // the O_t reads above are ordered before this warp's next p_full arrive
+      if (P.nsplit > 1) {
+        P.part_ml[pslot * 2] = m_used;
+        P.part_ml[pslot * 2 + 1] = l;
+      } else if (valid && A.out_lse) {
+        A.out_lse[orow] = l > 0.f ? (m_used * c + log2f(l)) * 0.6931471805599453f : -INFINITY;
+      }
+      cnt += n_iter;
     }
   }
 
@@ -460,7 +513,9 @@ template <int D>
 static dpara_status launch_tc_d(const TcParams &P, const TcPlan &plan, cudaStream_t st) {
   using Cfg = TcCfg<D>;
   if (cudaFuncSetAttribute(attn_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes) != cudaSuccess) return DPARA_ERR_CUDA;
-  dim3 grid(P.n_pairs * P.nsplit, P.a.Hkv, P.a.b);
+  int dev = 0, sms = kNumSM;
+  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int grid = P.n_items < sms ? P.n_items : sms;  // persistent: at most one CTA per SM
   attn_tc_kernel<D><<<grid, kThreads, Cfg::kSmemBytes, st>>>(P);
   DPARA_CHECK_LAUNCH();
   count_launches(1);
@@ -480,6 +535,7 @@ dpara_status launch_attention_tc(const AttnParams &A, const TcPlan &plan, const 
   P.JI_T = plan.JI_T; P.n_ji = plan.n_ji; P.n_tiles = plan.n_tiles; P.n_pairs = plan.n_pairs; P.nsplit = plan.nsplit;
   P.S8 = plan.S8; P.R_blk = plan.R_blk; P.has_blk = A.k_blk != nullptr;
   P.has_tail = (A.S > 0) || P.has_blk;
+  P.n_items = (int)(plan.items * plan.nsplit);
   P.c_log2 = A.scale * 1.4426950408889634f;
   const int D = A.D;
   const uint64_t rs = (uint64_t)D * 2;

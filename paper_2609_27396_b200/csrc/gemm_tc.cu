@@ -91,6 +91,9 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
   } else if (warp == 5) {
     if (lane == 0) {
       constexpr uint32_t idesc = idesc_bf16_f32(kBM, kBN, false, false);
+      // descriptors are built once; stage and K-step offsets are added in 16-byte units
+      const uint64_t adesc0 = smem_desc_sw128(smem_u32(smem), 16, 1024);
+      const uint64_t bdesc0 = smem_desc_sw128(smem_u32(smem) + kABytes, 16, 1024);
       bool ok = true;
       for (int kb = 0; kb < nkb && ok; ++kb) {
         const int s = kb % kStages;
@@ -98,13 +101,10 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
         ok = mbar_wait(full + s, ph, abort_flag);
         if (!ok) break;
         tc_fence_after();
-        const uint32_t sa = smem_u32(smem + s * kStageBytes);
+        const uint64_t so = (uint64_t)(s * (kStageBytes >> 4));
+        mma_ss(tmem, adesc0 + so, bdesc0 + so, idesc, kb != 0);
 #pragma unroll
-        for (int kk = 0; kk < kBK / 16; ++kk) {
-          const uint64_t ad = smem_desc_sw128(sa + kk * 32, 16, 1024);
-          const uint64_t bd = smem_desc_sw128(sa + kABytes + kk * 32, 16, 1024);
-          mma_ss(tmem, ad, bd, idesc, (kb | kk) != 0);
-        }
+        for (int kk = 1; kk < kBK / 16; ++kk) mma_ss_c<true>(tmem, adesc0 + so + 2 * kk, bdesc0 + so + 2 * kk, idesc);
         mma_commit(empty + s);
       }
       mma_commit(acc_full);
