@@ -45,25 +45,31 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint64_t *full = reinterpret_cast<uint64_t *>(smem + kStages * kStageBytes);
   uint64_t *empty = full + kStages;
-  uint64_t *acc_full = empty + kStages;
-  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_full + 1);
+  uint64_t *acc_full = empty + kStages;   // [2]: accumulator buffer ready for the epilogue
+  uint64_t *acc_empty = acc_full + 2;     // [2]: accumulator buffer drained
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_empty + 2);
   volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int n_tile = blockIdx.x, m_tile = blockIdx.y;
   const int nkb = P.K / kBK;
+  const int tile_cols = P.epi == 2 ? 128 : kBN;
+  const int m_tiles = (P.M + kBM - 1) / kBM, n_tiles = (P.N + tile_cols - 1) / tile_cols;
+  const int total_tiles = m_tiles * n_tiles;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
       mbar_init(full + s, 1);
       mbar_init(empty + s, 1);
     }
-    mbar_init(acc_full, 1);
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(acc_full + b, 1);
+      mbar_init(acc_empty + b, 4);
+    }
     *abort_flag = 0;
     fence_barrier_init();
   }
   if (warp == 5) {
-    tmem_alloc(tmem_slot, 256);
+    tmem_alloc(tmem_slot, 512);
     tmem_relinquish();
   }
   tc_fence_before();
@@ -71,21 +77,30 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
 
+  // Persistent: CTA c computes tiles c, c + gridDim.x, ...; tile id = n_tile * m_tiles + m_tile, so the CTAs
+  // running together cover all M rows of a few weight tiles (A stays in L2, each weight tile is read once).
+  // Two accumulator buffers in TMEM let the epilogue of one tile overlap the main loop of the next.
   if (warp == 4) {
     if (lane == 0) {
       prefetch_tensormap(&P.map_a);
       prefetch_tensormap(&P.map_b);
-      const int brow0 = P.epi == 2 ? n_tile * 128 : n_tile * kBN;
-      const int brow1 = P.epi == 2 ? P.up_row_offset + n_tile * 128 : n_tile * kBN + 128;
-      for (int kb = 0; kb < nkb; ++kb) {
-        const int s = kb % kStages;
-        const uint32_t ph = (kb / kStages) & 1;
-        if (!mbar_wait(empty + s, ph ^ 1u, abort_flag)) break;
-        uint8_t *sa = smem + s * kStageBytes;
-        mbar_arrive_expect_tx(full + s, kStageBytes);
-        tma_load_2d(sa, &P.map_a, full + s, kb * kBK, m_tile * kBM);
-        tma_load_2d(sa + kABytes, &P.map_b, full + s, kb * kBK, brow0);
-        tma_load_2d(sa + kABytes + 128 * kBK * 2, &P.map_b, full + s, kb * kBK, brow1);
+      int stage = 0;
+      uint32_t ph = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        const int m_tile = tile % m_tiles, n_tile = tile / m_tiles;
+        const int brow0 = P.epi == 2 ? n_tile * 128 : n_tile * kBN;
+        const int brow1 = P.epi == 2 ? P.up_row_offset + n_tile * 128 : n_tile * kBN + 128;
+        for (int kb = 0; kb < nkb; ++kb) {
+          ok = mbar_wait(empty + stage, ph ^ 1u, abort_flag);
+          if (!ok) break;
+          uint8_t *sa = smem + stage * kStageBytes;
+          mbar_arrive_expect_tx(full + stage, kStageBytes);
+          tma_load_2d(sa, &P.map_a, full + stage, kb * kBK, m_tile * kBM);
+          tma_load_2d(sa + kABytes, &P.map_b, full + stage, kb * kBK, brow0);
+          tma_load_2d(sa + kABytes + 128 * kBK * 2, &P.map_b, full + stage, kb * kBK, brow1);
+          if (++stage == kStages) { stage = 0; ph ^= 1u; }
+        }
       }
     }
   } else if (warp == 5) {
@@ -94,27 +109,41 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
       // descriptors are built once; stage and K-step offsets are added in 16-byte units
       const uint64_t adesc0 = smem_desc_sw128(smem_u32(smem), 16, 1024);
       const uint64_t bdesc0 = smem_desc_sw128(smem_u32(smem) + kABytes, 16, 1024);
+      int stage = 0, k = 0;
+      uint32_t ph = 0;
       bool ok = true;
-      for (int kb = 0; kb < nkb && ok; ++kb) {
-        const int s = kb % kStages;
-        const uint32_t ph = (kb / kStages) & 1;
-        ok = mbar_wait(full + s, ph, abort_flag);
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++k) {
+        const int buf = k & 1;
+        ok = mbar_wait(acc_empty + buf, ((k >> 1) & 1) ^ 1u, abort_flag);  // epilogue of tile k - 2 has drained this buffer
         if (!ok) break;
         tc_fence_after();
-        const uint64_t so = (uint64_t)(s * (kStageBytes >> 4));
-        mma_ss(tmem, adesc0 + so, bdesc0 + so, idesc, kb != 0);
+        const uint32_t acc = tmem + buf * kBN;
+        for (int kb = 0; kb < nkb; ++kb) {
+          ok = mbar_wait(full + stage, ph, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          const uint64_t so = (uint64_t)(stage * (kStageBytes >> 4));
+          mma_ss(acc, adesc0 + so, bdesc0 + so, idesc, kb != 0);
 #pragma unroll
-        for (int kk = 1; kk < kBK / 16; ++kk) mma_ss_c<true>(tmem, adesc0 + so + 2 * kk, bdesc0 + so + 2 * kk, idesc);
-        mma_commit(empty + s);
+          for (int kk = 1; kk < kBK / 16; ++kk) mma_ss_c<true>(acc, adesc0 + so + 2 * kk, bdesc0 + so + 2 * kk, idesc);
+          mma_commit(empty + stage);
+          if (++stage == kStages) { stage = 0; ph ^= 1u; }
+        }
+        if (ok) mma_commit(acc_full + buf);
       }
-      mma_commit(acc_full);
     }
   } else {
+   int k = 0;
+   bool live = true;
+   for (int tile = blockIdx.x; tile < total_tiles && live; tile += gridDim.x, ++k) {
+    const int m_tile = tile % m_tiles, n_tile = tile / m_tiles;
+    const int buf = k & 1;
     // ---------------- epilogue: thread = one accumulator row
-    const bool ok = __all_sync(0xffffffffu, mbar_wait(acc_full, 0, abort_flag));  // warp-uniform: tcgen05.ld is warp-wide
+    const bool ok = __all_sync(0xffffffffu, mbar_wait(acc_full + buf, (k >> 1) & 1, abort_flag));  // warp-uniform: tcgen05.ld is warp-wide
     tc_fence_after();
     const int row = m_tile * kBM + warp * 32 + lane;
-    const uint32_t taddr = tmem + ((uint32_t)(warp * 32) << 16);
+    const uint32_t taddr = tmem + buf * kBN + ((uint32_t)(warp * 32) << 16);
+    live = ok;
     if (ok) {
       if (P.epi == 2) {
         const int col0 = n_tile * 128;
@@ -189,12 +218,17 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
         }
       }
     }
+    // this warp has read its part of the accumulator: hand the buffer back to the MMA issuer
+    tc_fence_before();
+    __syncwarp();
+    if (lane == 0) mbar_arrive(acc_empty + buf);
+   }
   }
   // ---------------- teardown
   if (threadIdx.x == 0 && *abort_flag && P.status) atomicOr(reinterpret_cast<unsigned int *>(P.status), DPARA_STATUS_TIMEOUT);
   tc_fence_before();
   __syncthreads();
-  if (warp == 5) tmem_dealloc(tmem, 256);
+  if (warp == 5) tmem_dealloc(tmem, 512);
 }
 
 dpara_status launch_gemm_tc(const GemmArgs &g, int32_t *status, cudaStream_t st) {
@@ -210,8 +244,10 @@ dpara_status launch_gemm_tc(const GemmArgs &g, int32_t *status, cudaStream_t st)
   P.out = g.out; P.resid = g.resid; P.resid_bf16 = g.resid_bf16; P.out_bf16 = g.out_bf16; P.status = status;
   if (cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess) return DPARA_ERR_CUDA;
   const int tile_cols = g.epi == 2 ? 128 : kBN;
-  dim3 grid((g.N + tile_cols - 1) / tile_cols, (g.M + kBM - 1) / kBM);
-  gemm_tc_kernel<<<grid, kThreads, kSmemBytes, st>>>(P);
+  const int tiles = ((g.N + tile_cols - 1) / tile_cols) * ((g.M + kBM - 1) / kBM);
+  int dev = 0, sms = kNumSM;
+  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  gemm_tc_kernel<<<tiles < sms ? tiles : sms, kThreads, kSmemBytes, st>>>(P);
   DPARA_CHECK_LAUNCH();
   count_launches(1);
   return DPARA_OK;
