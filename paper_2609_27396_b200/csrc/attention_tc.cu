@@ -35,8 +35,8 @@ struct TcParams {
   CUtensorMap map_q, map_kc, map_vc, map_ks, map_vs, map_kb, map_vb;
   AttnParams a;
   int JI_T, n_ji, n_tiles, n_pairs, nsplit, S8, R_blk, has_blk, has_tail, n_items;
-  float *part_o;   // [item][2][128][D]
-  float *part_ml;  // [item][2][128][2]
+  float *part_o;   // split-KV partials [item slot][2][128][D] fp32 (unnormalised rows)
+  float2 *part_ml; // [item slot][2][128] (row max in raw-score units, row sum)
   float c_log2;    // softmax scale * log2(e)
   // requests in order of decreasing context length: the block scheduler hands out CTAs in grid order, so
   // launching the long requests first leaves the short ones to fill the tail of a ragged batch
@@ -105,7 +105,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
   volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  if (A.status_word && (*reinterpret_cast<volatile int32_t *>(A.status_word) & (int32_t)DPARA_STATUS_TIMEOUT)) return;
+  // (a CTA of a cluster must not leave early: its peers meet it at the cluster barriers below)
+  if (P.nsplit == 1 && A.status_word && (*reinterpret_cast<volatile int32_t *>(A.status_word) & (int32_t)DPARA_STATUS_TIMEOUT)) return;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kSlots; ++s) { mbar_init(kv_full + s, 1); mbar_init(kv_empty + s, 1); }
@@ -277,12 +278,12 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
       const bool valid = (t < I.ntq) && (r < P.JI_T * A.G) && (ji < P.n_ji);
       const int j = A.lo + ji / A.Bq, i = ji % A.Bq, h = I.g * A.G + r % A.G;
       const size_t orow = (((size_t)I.n * A.J + j) * A.Bq + i) * A.Hq + h;
-      const size_t pslot = (((size_t)I.slot * 2 + t) * 128 + r);
+      // split-KV: this CTA's partial rows go to an L2-resident scratch slot and are merged after a cluster barrier
+      const size_t pslot = ((size_t)I.slot * 2 + t) * 128 + r;
       if (I.n_iter == 0 || t >= I.ntq) {
         // nothing visible to this work item, or no second tile in the last pair
         if (P.nsplit > 1) {
-          P.part_ml[pslot * 2] = -INFINITY;
-          P.part_ml[pslot * 2 + 1] = 0.f;
+          __stcg(P.part_ml + pslot, make_float2(-INFINITY, 0.f));
         } else if (valid) {
           for (int d = 0; d < D; ++d) {
             if (A.out_f32) static_cast<float *>(A.out)[orow * D + d] = 0.f;
@@ -380,8 +381,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
           float4 *dst = reinterpret_cast<float4 *>(P.part_o + pslot * D + cc * 32);
 #pragma unroll
           for (int v = 0; v < 8; ++v)
-            dst[v] = make_float4(__uint_as_float(o[4 * v]), __uint_as_float(o[4 * v + 1]), __uint_as_float(o[4 * v + 2]),
-                                 __uint_as_float(o[4 * v + 3]));
+            __stcg(dst + v, make_float4(__uint_as_float(o[4 * v]), __uint_as_float(o[4 * v + 1]), __uint_as_float(o[4 * v + 2]),
+                                        __uint_as_float(o[4 * v + 3])));
         } else if (valid) {
           if (A.out_f32) {
             float4 *dst = reinterpret_cast<float4 *>(static_cast<float *>(A.out) + orow * D + cc * 32);
@@ -404,12 +405,87 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
       }
       tc_fence_before();  // the O_t reads above are ordered before this warp's next p_full arrive
       if (P.nsplit > 1) {
-        P.part_ml[pslot * 2] = m_used;
-        P.part_ml[pslot * 2 + 1] = l;
+        __stcg(P.part_ml + pslot, make_float2(m_used, l));
       } else if (valid && A.out_lse) {
         A.out_lse[orow] = l > 0.f ? (m_used * c + log2f(l)) * 0.6931471805599453f : -INFINITY;
       }
       cnt += n_iter;
+    }
+  }
+
+  // ------------------------------------------------------------------ split-KV merge across the cluster
+  // The nsplit CTAs that share (request, KV head, tile pair) form one thread-block cluster.  Each has written
+  // its unnormalised rows and (max, sum) to its scratch slot (which stays in L2); after a cluster barrier CTA
+  // `rank` merges 256 / nsplit of the rows from all peers' slots and writes the final output.  No second launch.
+  if (P.nsplit > 1) {
+    __threadfence();
+    __syncwarp();
+    cluster_sync_all();
+    if (warp < 8 && !*abort_flag) {
+      const Item I = decode_item(P, blockIdx.x);
+      const uint32_t rank = cluster_ctarank();
+      const int rows_per = 256 / P.nsplit;
+      const float c = P.c_log2;
+      const size_t slot0 = (size_t)(I.slot - I.split);  // scratch slot of split 0 of this item
+      // unit of work: 16 output elements of one row; all loads of a step are issued before their first use
+      constexpr int kParts = D / 16;
+      for (int u = threadIdx.x; u < rows_per * kParts; u += 256) {
+        const int R = (int)rank * rows_per + u / kParts, part = u % kParts;
+        const int t = R >> 7, r = R & 127;
+        const int ji = (I.pair * 2 + t) * P.JI_T + r / A.G;
+        if (t >= I.ntq || r >= P.JI_T * A.G || ji >= P.n_ji) continue;
+        const int j = A.lo + ji / A.Bq, i = ji % A.Bq, h = I.g * A.G + r % A.G;
+        const size_t orow = (((size_t)I.n * A.J + j) * A.Bq + i) * A.Hq + h;
+        float2 ml[8];
+#pragma unroll
+        for (int sp = 0; sp < 8; ++sp)
+          ml[sp] = sp < P.nsplit ? __ldcg(P.part_ml + ((slot0 + sp) * 2 + t) * 128 + r) : make_float2(-INFINITY, 0.f);
+        float mmax = -INFINITY;
+#pragma unroll
+        for (int sp = 0; sp < 8; ++sp) if (ml[sp].y > 0.f) mmax = fmaxf(mmax, ml[sp].x);
+        float acc[16], lsum = 0.f;
+#pragma unroll
+        for (int e = 0; e < 16; ++e) acc[e] = 0.f;
+#pragma unroll
+        for (int sp0 = 0; sp0 < 8; sp0 += 2) {
+          if (sp0 >= P.nsplit) break;
+          float4 x[2][4];
+#pragma unroll
+          for (int q = 0; q < 2; ++q) {
+            const float4 *src = reinterpret_cast<const float4 *>(P.part_o + (((slot0 + sp0 + q) * 2 + t) * 128 + r) * D + part * 16);
+#pragma unroll
+            for (int v = 0; v < 4; ++v) x[q][v] = __ldcg(src + v);
+          }
+#pragma unroll
+          for (int q = 0; q < 2; ++q) {
+            // a peer without visible keys wrote no rows (its slot may hold anything): weight 0 skips it
+            const float wgt = ml[sp0 + q].y > 0.f ? ex2((ml[sp0 + q].x - mmax) * c) : 0.f;
+            lsum = fmaf(wgt, ml[sp0 + q].y, lsum);
+            if (wgt > 0.f) {
+#pragma unroll
+              for (int v = 0; v < 4; ++v) {
+                acc[4 * v] = fmaf(wgt, x[q][v].x, acc[4 * v]);
+                acc[4 * v + 1] = fmaf(wgt, x[q][v].y, acc[4 * v + 1]);
+                acc[4 * v + 2] = fmaf(wgt, x[q][v].z, acc[4 * v + 2]);
+                acc[4 * v + 3] = fmaf(wgt, x[q][v].w, acc[4 * v + 3]);
+              }
+            }
+          }
+        }
+        const float inv = lsum > 0.f ? 1.0f / lsum : 0.f;
+        if (A.out_f32) {
+          float4 *dst = reinterpret_cast<float4 *>(static_cast<float *>(A.out) + orow * D + part * 16);
+#pragma unroll
+          for (int v = 0; v < 4; ++v) dst[v] = make_float4(acc[4 * v] * inv, acc[4 * v + 1] * inv, acc[4 * v + 2] * inv, acc[4 * v + 3] * inv);
+        } else {
+          uint4 *dst = reinterpret_cast<uint4 *>(static_cast<uint16_t *>(A.out) + orow * D + part * 16);
+#pragma unroll
+          for (int v = 0; v < 2; ++v)
+            dst[v] = make_uint4(pack_bf16(acc[8 * v] * inv, acc[8 * v + 1] * inv), pack_bf16(acc[8 * v + 2] * inv, acc[8 * v + 3] * inv),
+                                pack_bf16(acc[8 * v + 4] * inv, acc[8 * v + 5] * inv), pack_bf16(acc[8 * v + 6] * inv, acc[8 * v + 7] * inv));
+        }
+        if (A.out_lse && part == 0) A.out_lse[orow] = lsum > 0.f ? (mmax * c + log2f(lsum)) * 0.6931471805599453f : -INFINITY;
+      }
     }
   }
 
@@ -427,52 +503,6 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
     __syncthreads();
   }
   if (warp == 9) tmem_dealloc(tmem, 512);
-}
-
-// ------------------------------------------------------------------------------------------------ split-KV combine
-// One warp per (item pair, tile, row): merges the nsplit partial (m, l, O) triples of a query row.
-template <int D>
-__global__ void __launch_bounds__(128) attn_tc_combine_kernel(const TcParams P) {
-  const AttnParams &A = P.a;
-  const int lane = threadIdx.x & 31;
-  const long long w = (long long)blockIdx.x * 4 + (threadIdx.x >> 5);
-  const long long total = (long long)A.b * A.Hkv * P.n_pairs * 256;
-  if (w >= total) return;
-  const int r = (int)(w & 127), t = (int)((w >> 7) & 1);
-  const long long base_item = (w >> 8);  // (n * Hkv + g) * n_pairs + pair
-  const int pair = (int)(base_item % P.n_pairs);
-  const int g = (int)((base_item / P.n_pairs) % A.Hkv), n = (int)(base_item / P.n_pairs / A.Hkv);
-  const int ji = (pair * 2 + t) * P.JI_T + r / A.G;
-  if (pair * 2 + t >= P.n_tiles || r >= P.JI_T * A.G || ji >= P.n_ji) return;
-  const int j = A.lo + ji / A.Bq, i = ji % A.Bq, h = g * A.G + r % A.G;
-  constexpr int E = D / 32;
-  float mmax = -INFINITY;
-  for (int s = 0; s < P.nsplit; ++s) mmax = fmaxf(mmax, P.part_ml[((((size_t)base_item * P.nsplit + s) * 2 + t) * 128 + r) * 2]);
-  float l = 0.f, o[E];
-#pragma unroll
-  for (int e = 0; e < E; ++e) o[e] = 0.f;
-  for (int s = 0; s < P.nsplit; ++s) {
-    const size_t slot = (((size_t)base_item * P.nsplit + s) * 2 + t) * 128 + r;
-    const float ms = P.part_ml[slot * 2], ls = P.part_ml[slot * 2 + 1];
-    if (!(ls > 0.f)) continue;
-    const float wgt = ptx::ex2((ms - mmax) * P.c_log2);
-    l += wgt * ls;
-    const float *po = P.part_o + slot * D + lane * E;
-#pragma unroll
-    for (int e = 0; e < E; ++e) o[e] = fmaf(wgt, po[e], o[e]);
-  }
-  const float inv = l > 0.f ? 1.0f / l : 0.f;
-  const size_t orow = (((size_t)n * A.J + j) * A.Bq + i) * A.Hq + h;
-  if (A.out_f32) {
-    float *dst = static_cast<float *>(A.out) + orow * D + lane * E;
-#pragma unroll
-    for (int e = 0; e < E; ++e) dst[e] = o[e] * inv;
-  } else {
-    uint16_t *dst = static_cast<uint16_t *>(A.out) + orow * D + lane * E;
-#pragma unroll
-    for (int e = 0; e < E; e += 2) *reinterpret_cast<uint32_t *>(dst + e) = pack_bf16(o[e] * inv, o[e + 1] * inv);
-  }
-  if (A.out_lse && lane == 0) A.out_lse[orow] = l > 0.f ? (mmax * P.c_log2 + log2f(l)) * 0.6931471805599453f : -INFINITY;
 }
 
 // ------------------------------------------------------------------------------------------------ host
@@ -495,12 +525,12 @@ TcPlan plan_attention_tc(const dpara_shape *s, const int64_t *host_off) {
   if (tot + 128 >= (1ll << 31) || (long long)s->batch * s->n_boundaries * s->block >= (1ll << 31)) return p;
   const long long items = (long long)s->batch * s->n_kv_heads * p.n_pairs;
   const int max_tiles = (int)((max_l + 127) / 128);
+  // split the KV range over a cluster of 2, 4 or 8 CTAs when the batch alone cannot fill the GPU
   int nsplit = 1;
   if (items < 96 && max_tiles > 1) {
-    nsplit = (int)((kNumSM + items - 1) / items);
-    if (nsplit > max_tiles) nsplit = max_tiles;
-    if (nsplit > 32) nsplit = 32;
-    if (nsplit < 1) nsplit = 1;
+    const long long want = (kNumSM + items - 1) / items;
+    for (int c = 8; c >= 2; c >>= 1)
+      if (c <= want && c <= max_tiles) { nsplit = c; break; }
   }
   p.nsplit = nsplit;
   p.items = items;
@@ -515,16 +545,28 @@ static dpara_status launch_tc_d(const TcParams &P, const TcPlan &plan, cudaStrea
   if (cudaFuncSetAttribute(attn_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes) != cudaSuccess) return DPARA_ERR_CUDA;
   int dev = 0, sms = kNumSM;
   if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  const int grid = P.n_items < sms ? P.n_items : sms;  // persistent: at most one CTA per SM
-  attn_tc_kernel<D><<<grid, kThreads, Cfg::kSmemBytes, st>>>(P);
-  DPARA_CHECK_LAUNCH();
-  count_launches(1);
+  cudaLaunchConfig_t cfg = {};
+  cudaLaunchAttribute attr[1];
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = Cfg::kSmemBytes;
+  cfg.stream = st;
   if (P.nsplit > 1) {
-    const long long rows = plan.items * 256;
-    attn_tc_combine_kernel<D><<<(unsigned)((rows + 3) / 4), 128, 0, st>>>(P);
-    DPARA_CHECK_LAUNCH();
-    count_launches(1);
+    // one CTA per (item, split); the splits of an item are consecutive CTAs = one cluster
+    cfg.gridDim = dim3(P.n_items);
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = P.nsplit;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+  } else {
+    cfg.gridDim = dim3(P.n_items < sms ? P.n_items : sms);  // persistent: at most one CTA per SM
   }
+  if (cudaLaunchKernelEx(&cfg, attn_tc_kernel<D>, P) != cudaSuccess) {
+    cudaGetLastError();
+    return DPARA_ERR_CUDA;
+  }
+  count_launches(1);
   return DPARA_OK;
 }
 
@@ -570,7 +612,7 @@ dpara_status launch_attention_tc(const AttnParams &A, const TcPlan &plan, const 
   }
   if (plan.nsplit > 1) {
     P.part_o = static_cast<float *>(workspace);
-    P.part_ml = P.part_o + (size_t)plan.items * plan.nsplit * 256 * D;
+    P.part_ml = reinterpret_cast<float2 *>(P.part_o + (size_t)plan.items * plan.nsplit * 256 * D);
   }
   return D == 128 ? launch_tc_d<128>(P, plan, st) : launch_tc_d<64>(P, plan, st);
 }
