@@ -180,8 +180,8 @@ dpara_status dpara_verify_select(const dpara_verify_io *io, void *workspace, siz
  *    that device.
  *  - Requests whose scratch need (dpara_verify_workspace_bytes) exceeds the fixed size are refused
  *    with DPARA_ERR_STATIC_LIMIT and nothing is launched.  For scale: greedy mode with 16 requests
- *    x 16 boundaries needs 2.3 KB, sampling mode with 8 requests over a 151 936-token vocabulary
- *    5 KB; the need grows with batch * n_boundaries (greedy) or batch * ceil(vocab / 4096) (sampling).
+ *    x 16 boundaries needs 3.3 KB, sampling mode with 8 requests over a 151 936-token vocabulary
+ *    5.3 KB; the need grows with batch * n_boundaries (greedy) or batch * ceil(vocab / 4096) (sampling).
  *  - All calls on a device share the one array and it keeps whatever the previous call left; the
  *    call itself clears the parts that must start at zero.  Two calls that overlap on the same GPU
  *    (different streams, or different host threads without ordering) race on it and give undefined

@@ -10,7 +10,11 @@
 namespace dpara {
 
 constexpr int kVsThreads = 256;
-constexpr int kGreedyChunk = 8192;  // floats per CTA: 8 x 16 B in flight per thread
+#ifndef DPARA_GREEDY_LOADS
+#define DPARA_GREEDY_LOADS 16
+#endif
+constexpr int kGreedyLoads = DPARA_GREEDY_LOADS;             // 16-byte loads in flight per thread
+constexpr int kGreedyChunk = kGreedyLoads * 1024;  // floats per CTA
 constexpr int kSampChunk = 4096;    // floats per CTA and per row
 constexpr int kMaxJ = 64;
 
@@ -46,14 +50,14 @@ __device__ __forceinline__ void gather_branch(const uint8_t *__restrict__ reps, 
     const uint4 *s = reinterpret_cast<const uint4 *>(src);
     uint4 *d = reinterpret_cast<uint4 *>(dst);
     const size_t nv = bytes >> 4;
-    // 8 independent 16-byte loads in flight per thread: the copy is one CTA's job, so latency matters
+    // 16 independent 16-byte loads in flight per thread: the copy is one CTA's job, so latency matters
     size_t i = tid;
-    for (; i + 7 * (size_t)nthreads < nv; i += 8 * (size_t)nthreads) {
-      uint4 v[8];
+    for (; i + 15 * (size_t)nthreads < nv; i += 16 * (size_t)nthreads) {
+      uint4 v[16];
 #pragma unroll
-      for (int k = 0; k < 8; ++k) v[k] = __ldcs(s + i + k * (size_t)nthreads);
+      for (int k = 0; k < 16; ++k) v[k] = __ldcs(s + i + k * (size_t)nthreads);
 #pragma unroll
-      for (int k = 0; k < 8; ++k) d[i + k * (size_t)nthreads] = v[k];
+      for (int k = 0; k < 16; ++k) d[i + k * (size_t)nthreads] = v[k];
     }
     for (; i < nv; i += nthreads) d[i] = __ldcs(s + i);
   } else {
@@ -71,8 +75,9 @@ struct VerifyParams {
   uint8_t *selected;
   int32_t *status_word;
   unsigned long long *ws64;  // greedy: keys[b*J]; sampling: chunk sums [b][nchunks][2]
-  unsigned int *counters;    // [b], zeroed before the launch
-  int J, V, nchunks, vec_ok;
+  unsigned int *counters;    // greedy: [b*J] row counters; sampling: [b]; zeroed before the launch
+  unsigned long long *masks; // greedy: [b] completed-row masks, zeroed before the launch
+  int b, J, V, nchunks, vec_ok;
   size_t rep_bytes;  // Bq * hidden * 2
 };
 
@@ -91,8 +96,10 @@ __device__ __forceinline__ void write_result(const VerifyParams &P, int n, int r
 // ------------------------------------------------------------------------------------------ greedy
 __global__ void __launch_bounds__(kVsThreads) verify_greedy_kernel(const VerifyParams P) {
   const int tid = threadIdx.x;
-  const int row = blockIdx.y;  // n * J + i
-  const int n = row / P.J;
+  // rows are handed out position-major (every request's row 0 first, then every row 1, ...): the early rows,
+  // which decide the accepted length, finish early for ALL requests
+  const int n = blockIdx.y % P.b;
+  const int row = n * P.J + blockIdx.y / P.b;
   const float *__restrict__ p = P.target + (size_t)row * P.V;
   const int base = blockIdx.x * kGreedyChunk;
   const int end = min(P.V, base + kGreedyChunk);
@@ -106,14 +113,14 @@ __global__ void __launch_bounds__(kVsThreads) verify_greedy_kernel(const VerifyP
   float bv = -INFINITY;
   uint32_t bi = 0xffffffffu;
   if (P.vec_ok) {
-    float4 v[8];
+    float4 v[kGreedyLoads];
 #pragma unroll
-    for (int it = 0; it < 8; ++it) {
+    for (int it = 0; it < kGreedyLoads; ++it) {
       int idx = base + (it * kVsThreads + tid) * 4;
       v[it] = idx < end ? __ldcs(reinterpret_cast<const float4 *>(p + idx)) : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
     }
 #pragma unroll
-    for (int it = 0; it < 8; ++it) {
+    for (int it = 0; it < kGreedyLoads; ++it) {
       const uint32_t idx = base + (it * kVsThreads + tid) * 4;
       if (v[it].x > bv) { bv = v[it].x; bi = idx; }
       if (v[it].y > bv) { bv = v[it].y; bi = idx + 1; }
@@ -147,41 +154,71 @@ __global__ void __launch_bounds__(kVsThreads) verify_greedy_kernel(const VerifyP
       __syncthreads();
     }
   }
+  // Completion protocol (no CTA waits for another):
+  //   row counter   -- the CTA that brings a row's counter to nchunks has completed that row;
+  //   request mask  -- it then ORs the row's bit into the request's mask.  The accepted length is decided
+  //                    as soon as rows 0..k are complete and either draft k+1 disagrees with row k's maximum or
+  //                    k is the last row.  Exactly one CTA sees the mask go from "undecided" to "decided"
+  //                    (the atomic OR serialises them); it writes the results and gathers the branch -- usually
+  //                    while most of the request's later rows are still streaming, so the gather is hidden.
+  __shared__ unsigned long long s_old, s_new;
   if (tid == 0) {
     unsigned long long m = s_k[0];
 #pragma unroll
     for (int w = 1; w < kVsThreads / 32; ++w) m = s_k[w] > m ? s_k[w] : m;
     if (m) atomicMax(P.ws64 + row, m);
     __threadfence();
-    unsigned int t = atomicAdd(P.counters + n, 1u);
-    s_flag = (t == (unsigned int)(P.J * P.nchunks) - 1u);
+    s_flag = 0;
+    if (atomicAdd(P.counters + row, 1u) == (unsigned int)P.nchunks - 1u) {
+      __threadfence();
+      const unsigned long long bit = 1ull << (row - n * P.J);
+      const unsigned long long old = atomicOr(P.masks + n, bit);
+      s_old = old;
+      s_new = old | bit;
+      s_flag = 1;
+    }
   }
   __syncthreads();
   if (!s_flag) return;
 
-  // ---- last CTA of request n: position scan, outputs, gather
+  // ---- this CTA completed a row: is the request's outcome decided now, and was it not before?
   __threadfence();
   __shared__ int s_a[kMaxJ], s_t[kMaxJ];
-  __shared__ int s_r, s_bad;
+  __shared__ int s_r, s_bad, s_act;
+  const unsigned long long mask_new = s_new, mask_old = s_old;
   if (tid < P.J) {
-    unsigned long long k = __ldcg(P.ws64 + (size_t)n * P.J + tid);
+    const bool done = (mask_new >> tid) & 1ull;
+    unsigned long long k = done ? __ldcg(P.ws64 + (size_t)n * P.J + tid) : 0ull;
     s_a[tid] = k == 0ull ? 0 : (int)(0xffffffffu - (uint32_t)(k & 0xffffffffull));  // all-NaN row -> 0
     s_t[tid] = tid < P.J - 1 ? P.tokens[(size_t)n * (P.J - 1) + tid] : -1;           // all tokens in one round trip
   }
   __syncthreads();
   if (tid == 0) {
-    int r = 0;
-    bool bad = false;
-    while (r < P.J - 1) {
-      const int t = s_t[r];
-      if (t < 0 || t >= P.V) { bad = true; break; }
-      if (t != s_a[r]) break;
-      ++r;
+    // scan with the new mask; remember how far the OLD mask would have allowed the same scan to go
+    int r = -1;
+    bool bad = false, decided_before = false;
+    for (int k = 0; k < P.J; ++k) {
+      if (!((mask_new >> k) & 1ull)) break;  // row k not complete yet: undecided
+      bool stop = (k == P.J - 1);
+      if (!stop) {
+        const int t = s_t[k];
+        if (t < 0 || t >= P.V) { bad = true; stop = true; }
+        else if (t != s_a[k]) stop = true;
+      }
+      if (stop) {
+        r = k;
+        // decided before iff rows 0..k were all complete in the old mask as well
+        const unsigned long long need = (k == 63) ? ~0ull : ((1ull << (k + 1)) - 1ull);
+        decided_before = (mask_old & need) == need;
+        break;
+      }
     }
+    s_act = (r >= 0) && !decided_before;
     s_r = r;
     s_bad = bad;
   }
   __syncthreads();
+  if (!s_act) return;
   const int r = s_r;
   if (tid == 0) {
     P.accept_len[n] = r;
@@ -423,7 +460,8 @@ using namespace dpara;
 
 extern "C" size_t dpara_verify_workspace_bytes(const dpara_verify_io *io) {
   if (validate_dims(io) != DPARA_OK) return 0;
-  return align_up(ws64_count(io) * 8, 256) + align_up((size_t)io->batch * 4, 256);
+  const size_t ncnt = io->mode == 0 ? (size_t)io->batch * io->n_boundaries : (size_t)io->batch;
+  return align_up(ws64_count(io) * 8, 256) + align_up((size_t)io->batch * 8, 256) + align_up(ncnt * 4, 256);
 }
 
 namespace dpara {
@@ -441,23 +479,27 @@ dpara_status launch_verify(const dpara_verify_io *io, void *ws, int32_t *status_
   P.out_tokens = io->out_tokens;
   P.selected = static_cast<uint8_t *>(io->selected);
   P.status_word = status_word;
+  P.b = io->batch;
   P.J = io->n_boundaries;
   P.V = io->vocab;
   P.nchunks = chunks_of(io);
   P.rep_bytes = (size_t)io->block * io->hidden * 2;
   size_t n64 = ws64_count(io);
-  size_t cnt_off = align_up(n64 * 8, 256);
+  const size_t mask_off = align_up(n64 * 8, 256);
+  const size_t cnt_off = mask_off + align_up((size_t)io->batch * 8, 256);
+  const size_t ncnt = io->mode == 0 ? (size_t)io->batch * io->n_boundaries : (size_t)io->batch;
   P.ws64 = static_cast<unsigned long long *>(ws);
+  P.masks = reinterpret_cast<unsigned long long *>(static_cast<uint8_t *>(ws) + mask_off);
   P.counters = reinterpret_cast<unsigned int *>(static_cast<uint8_t *>(ws) + cnt_off);
   bool vec = (io->vocab % 4 == 0) && aligned16(io->target) && (io->mode == 0 || io->n_boundaries == 1 || aligned16(io->draft_probs));
   P.vec_ok = vec ? 1 : 0;
   // greedy needs keys and counters at zero; sampling only the counters
   if (io->mode == 0) {
-    if (cudaMemsetAsync(ws, 0, cnt_off + (size_t)io->batch * 4, st) != cudaSuccess) return DPARA_ERR_CUDA;
+    if (cudaMemsetAsync(ws, 0, cnt_off + ncnt * 4, st) != cudaSuccess) return DPARA_ERR_CUDA;  // keys, masks, counters
     dim3 grid(P.nchunks, io->batch * io->n_boundaries);
     verify_greedy_kernel<<<grid, kVsThreads, 0, st>>>(P);
   } else {
-    if (cudaMemsetAsync(P.counters, 0, (size_t)io->batch * 4, st) != cudaSuccess) return DPARA_ERR_CUDA;
+    if (cudaMemsetAsync(P.counters, 0, ncnt * 4, st) != cudaSuccess) return DPARA_ERR_CUDA;
     dim3 grid(P.nchunks, io->batch);
     verify_sampling_kernel<<<grid, kVsThreads, 0, st>>>(P);
   }
