@@ -215,6 +215,13 @@ typedef struct {
 } dpara_gemm_io;
 dpara_status dpara_gemm_bf16(const dpara_gemm_io *io, int32_t *status_word, void *stream);
 
+/* Failure-detection self-test (the paper has no counterpart): launches one CTA that waits, with the
+ * same bounded wait all kernels here use, on a barrier nothing arrives at.  After `limit_us`
+ * microseconds (1 .. 1 000 000) the wait gives up, DPARA_STATUS_TIMEOUT is OR-ed into *status_word
+ * (device, required), the time actually waited is stored in *waited_ns (device, optional) and the kernel
+ * ends normally; the CUDA context stays usable.  Errors: INVALID_ARG, CUDA. */
+dpara_status dpara_selftest_bounded_wait(int32_t *status_word, uint32_t limit_us, uint64_t *waited_ns, void *stream);
+
 /* Number of kernels this library has launched in this process so far (all calls, all streams).
  * Bookkeeping for benchmarks; the paper has no counterpart. */
 int64_t dpara_kernel_launches(void);

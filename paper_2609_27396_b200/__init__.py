@@ -101,6 +101,22 @@ def gemm_bf16(a, w, *, epilogue: int = 0, resid=None, want_bf16_copy: bool = Fal
     return (out, out16, st) if out16 is not None else (out, st)
 
 
+lib.dpara_selftest_bounded_wait.restype = C.c_int
+lib.dpara_selftest_bounded_wait.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p]
+EXPORTED.append("dpara_selftest_bounded_wait")
+
+
+def selftest_bounded_wait(limit_us: int = 1000, stream=None):
+    """dpara_selftest_bounded_wait: returns (status_word, waited_ns) after the stream has drained."""
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    waited = torch.zeros(1, dtype=torch.int64, device="cuda")
+    rc = lib.dpara_selftest_bounded_wait(st.data_ptr(), limit_us, waited.data_ptr(), _stream_ptr(stream))
+    if rc != OK:
+        raise DparaError(rc)
+    torch.cuda.synchronize()
+    return int(st.item()), int(waited.item())
+
+
 class DparaError(RuntimeError):
     def __init__(self, code: int):
         self.code = code
