@@ -33,7 +33,7 @@ METRIC = "all_boundary_draft_step_us"
 L2_FLUSH_BYTES = 256 << 20
 # dram__bytes_read.sum + dram__bytes_write.sum of one attention launch, from the ncu capture summarised in
 # profiles/attention_tc_cfg3_b16.md (bytes per launch; None where no capture exists)
-NCU_DRAM_TRAFFIC = {"cfg3": 269349120, "cfg2": None}
+NCU_DRAM_TRAFFIC = {"cfg3": 266551296, "cfg2": None}
 
 
 # ----------------------------------------------------------------------------- algorithmic work
