@@ -40,8 +40,14 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
 }
 // Bounded wait: gives up after kWaitLimitNs of wall time (or as soon as another thread of the CTA has
 // given up), sets *abort_flag and returns false.  Never waits forever.
-constexpr uint64_t kWaitLimitNs = 200ull * 1000 * 1000;
-__device__ __forceinline__ bool mbar_wait_limit(uint64_t *bar, uint32_t parity, volatile int *abort_flag, uint64_t limit_ns) {
+#ifndef DPARA_WAIT_LIMIT_NS
+#define DPARA_WAIT_LIMIT_NS (200ull * 1000 * 1000)
+#endif
+constexpr uint64_t kWaitLimitNs = DPARA_WAIT_LIMIT_NS;
+// `site` (1..255) identifies the wait: the first one to give up in a CTA leaves its site in *abort_flag (a
+// diagnostic for whoever reads the flag; any non-zero value means "give up").
+__device__ __forceinline__ bool mbar_wait_limit(uint64_t *bar, uint32_t parity, volatile int *abort_flag, uint64_t limit_ns,
+                                                int site = 1) {
   if (mbar_try(bar, parity)) return true;
   const uint64_t t0 = global_timer_ns();
   for (;;) {
@@ -49,11 +55,11 @@ __device__ __forceinline__ bool mbar_wait_limit(uint64_t *bar, uint32_t parity, 
     if (*abort_flag) return false;
     if (global_timer_ns() - t0 > limit_ns) break;
   }
-  *abort_flag = 1;
+  if (*abort_flag == 0) *abort_flag = site;
   return false;
 }
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag) {
-  return mbar_wait_limit(bar, parity, abort_flag, kWaitLimitNs);
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag, int site = 1) {
+  return mbar_wait_limit(bar, parity, abort_flag, kWaitLimitNs, site);
 }
 
 __device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
