@@ -5,17 +5,22 @@
 // of all G query heads that share the KV head, and every K/V byte streamed from HBM serves all
 // boundaries and all heads of the group at once.
 //
-//   warp 8      TMA producer: Q tiles once, then K and V tiles of 128 keys through one ring of tile slots.
-//               The context needs no mask at all (every row sees the whole cache); the spine prefix
-//               and the boundaries' own blocks are packed into ONE extra "tail" tile per CTA.
-//   warp 9      one thread issues tcgen05.mma:  S_t = Q_t K^T  (A, B from shared memory) and
-//               O_t += P_t V  (A = P_t from tensor memory, B = V, MN-major), t = 0, 1 ping-pong so the
-//               tensor pipe works on one tile while the other tile's softmax runs.
-//   warps 0-3   softmax of tile 0, warps 4-7 softmax of tile 1: thread = row.  tcgen05.ld the S row,
-//               mask (tail tile only: anchor prefix of the row's boundary + its own block), online
-//               max/sum in registers with LAZY rescaling (O in TMEM is rescaled only when a row's max
-//               grows by more than 2^8), P written back over S as bf16 with tcgen05.st.
-// TMEM: S0 | S1 (128 fp32 columns each, P aliases the first 64) | O0 | O1 (D columns each).
+//   warp 8      TMA producer: Q tiles once, then K and V tiles of 128 keys through one ring of tile slots
+//               (order K0 K1 V0 K2 V1 ...).  The context needs no mask at all (every row sees the whole
+//               cache); the spine prefix and the boundaries' own blocks are packed into ONE extra "tail"
+//               tile per CTA.
+//   warp 9      one thread issues tcgen05.mma:  S = Q_t K^T  (A, B from shared memory) and
+//               O_t += P_t V  (A = P_t from tensor memory, B = V, MN-major).
+//   warps 0-3   softmax of tile 0, warps 4-7 softmax of tile 1: thread = row.  tcgen05.ld the S row into
+//               registers and hand the S buffer back at once; mask (tail tile only: anchor prefix of the
+//               row's boundary + its own block), online max/sum in registers with LAZY rescaling (O in
+//               TMEM is rescaled only when a row's max grows by more than 2^8), P_t written as bf16 with
+//               tcgen05.st to its own columns.
+// TMEM: O0 | O1 (128 columns reserved each) | S (128 fp32 columns, ONE buffer that the two tiles take in
+// turns) | P0 | P1 (64 columns each).  S lives only from its QK to the softmax warps' load, and P_t does not
+// alias it, so QK(t, i+1) never waits for softmax(t, i): a tile's softmax finds its next scores ready, and
+// the tensor pipe and the softmax warps are coupled only through buffer hand-offs, not through a
+// score -> probability -> score chain.
 // Every mbarrier wait is bounded; on expiry the CTA sets DPARA_STATUS_TIMEOUT and drains.
 #include <math.h>
 
@@ -49,11 +54,11 @@ struct TcCfg {
   static constexpr int kSlabs = D / 64;
   static constexpr int kSlabBytes = 128 * 128;         // 128 rows x 64 bf16
   static constexpr int kTileBytes = kSlabs * kSlabBytes;  // Q, K or V tile
-  // K and V tiles travel through ONE ring of tile-sized slots (K0 V0 K1 V1 ...), as deep as shared memory
+  // K and V tiles travel through ONE ring of tile-sized slots (K0 K1 V0 K2 V1 ...), as deep as shared memory
   // allows next to the two Q tiles: the producer runs ~1.5 iterations ahead of the MMA issuer
   static constexpr int kSlots = (227 * 1024 - 2 * kTileBytes - 2048) / kTileBytes > 8 ? 8 : (227 * 1024 - 2 * kTileBytes - 2048) / kTileBytes;
   static constexpr int kSmemBytes = 2 * kTileBytes + kSlots * kTileBytes + 1024 + 512;
-  static constexpr int kOBase = 256;                    // TMEM column of O0
+  static constexpr int kColO = 0, kColS = 256, kColP = 384;  // TMEM columns: O_t at kColO + 128 t, S, P_t at kColP + 64 t
 };
 
 // One unit of work of a persistent CTA.
@@ -100,8 +105,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
   constexpr int kSlots = Cfg::kSlots;
   uint64_t *bars = reinterpret_cast<uint64_t *>(sKV + kSlots * Cfg::kTileBytes);
   uint64_t *kv_full = bars, *kv_empty = bars + kSlots, *q_full = bars + 2 * kSlots, *q_empty = q_full + 1, *s_full = q_full + 2,
-           *p_full = q_full + 4, *pv_done = q_full + 6;
-  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(q_full + 8);
+           *p_full = q_full + 4, *pv_done = q_full + 6, *s_free = q_full + 8;
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(q_full + 9);
   volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -113,6 +118,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
     mbar_init(q_full, 1);
     mbar_init(q_empty, 1);
     for (int t = 0; t < 2; ++t) { mbar_init(s_full + t, 1); mbar_init(p_full + t, 4); mbar_init(pv_done + t, 1); }
+    mbar_init(s_free, 4);
     *abort_flag = 0;
     fence_barrier_init();
   }
@@ -146,9 +152,11 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
           for (int sb = 0; sb < Cfg::kSlabs; ++sb)
             tma_load_3d(sQ + t * Cfg::kTileBytes + sb * Cfg::kSlabBytes, &P.map_q, q_full, sb * 64, I.g * A.G, qrow0 + t * P.JI_T);
       }
-      // load q = 2 it is the K tile of iteration it, load 2 it + 1 its V tile; slot = (ld + q) % kSlots
+      // load order K0 K1 V0 K2 V1 ... K(n-1) V(n-2) V(n-1): the order the MMA issuer consumes them in
+      // (the scores of iteration it + 1 are issued before the PV product of iteration it); slot = (ld + q) % kSlots
       for (int q = 0; q < 2 * I.n_iter; ++q) {
-        const int it = q >> 1, is_v = q & 1;
+        const bool is_v = q > 0 && (((q & 1) == 0) || ((q + 1) >> 1) >= I.n_iter);
+        const int it = q == 0 ? 0 : (is_v ? ((q & 1) ? I.n_iter - 1 : (q >> 1) - 1) : (q + 1) >> 1);
         const int sl = (ld + q) % kSlots;
         const uint32_t ph = ((ld + q) / kSlots) & 1;
         ok = __all_sync(0xffffffffu, mbar_wait(kv_empty + sl, ph ^ 1u, abort_flag));
@@ -198,12 +206,20 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
       const uint64_t kdesc0 = smem_desc_sw128(smem_u32(sKV), 16, 1024);                 // K tile: K-major operand
       const uint64_t vdesc0 = smem_desc_sw128(smem_u32(sKV), Cfg::kSlabBytes, 1024);    // V tile: MN-major operand
       int ring_slot = 0, k = 0;
-      uint32_t ring_phase = 0, ph_p[2] = {0, 0};
-      bool ok = true;
+      uint32_t ring_phase = 0, ph_p[2] = {0, 0}, ph_sf = 0;
+      bool ok = true, first_qk = true;
       auto next_load = [&](int &slot_out) {  // wait for the next tile of the K/V ring (loads are consumed in order)
         slot_out = ring_slot;
         const bool r = mbar_wait(kv_full + ring_slot, ring_phase, abort_flag);
         if (++ring_slot == kSlots) { ring_slot = 0; ring_phase ^= 1u; }
+        return r;
+      };
+      // The single S buffer is handed back by the softmax warps of whichever tile read it last (also across
+      // items): every QK but the kernel's first waits for one phase of s_free.
+      auto wait_s_free = [&]() {
+        if (first_qk) { first_qk = false; return true; }
+        const bool r = mbar_wait(s_free, ph_sf, abort_flag, 3);
+        ph_sf ^= 1u;
         return r;
       };
       for (int id = blockIdx.x; id < P.n_items && ok; id += gridDim.x) {
@@ -215,8 +231,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
 #pragma unroll
           for (int kk = 0; kk < D / 16; ++kk) {
             const uint32_t off = ((kk >> 2) * Cfg::kSlabBytes + (kk & 3) * 32) >> 4;
-            if (kk == 0) mma_ss_c<false>(tmem + t * 128, qa + off, ka + off, idesc_qk);
-            else mma_ss_c<true>(tmem + t * 128, qa + off, ka + off, idesc_qk);
+            if (kk == 0) mma_ss_c<false>(tmem + Cfg::kColS, qa + off, ka + off, idesc_qk);
+            else mma_ss_c<true>(tmem + Cfg::kColS, qa + off, ka + off, idesc_qk);
           }
           mma_commit(s_full + t);
           if (t == ntq - 1) {
@@ -226,35 +242,40 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
         };
         auto issue_pv = [&](int t, int vslot, bool acc) {
           const uint64_t va = vdesc0 + (uint64_t)(vslot * kTile16);
-          const uint32_t o_t = tmem + Cfg::kOBase + t * D, p_t = tmem + t * 128;
+          const uint32_t o_t = tmem + Cfg::kColO + t * 128, p_t = tmem + Cfg::kColP + t * 64;
           mma_ts(o_t, p_t, va, idesc_pv, acc);
 #pragma unroll
           for (int kk = 1; kk < 8; ++kk) mma_ts_c<true>(o_t, p_t + kk * 8, va + (uint64_t)(kk * (2048 >> 4)), idesc_pv);
           mma_commit(pv_done + t);
           if (t == ntq - 1) mma_commit(kv_empty + vslot);  // V tile consumed
         };
+        // issue order per iteration: QK(0, it+1)  PV(0, it)  QK(1, it+1)  PV(1, it) -- each operation right
+        // where its inputs become ready in steady state (the S buffer comes back when the OTHER tile has
+        // loaded its scores; P_t arrives when tile t's softmax ends)
         int kslot = 0, vslot = 0;
-        ok = mbar_wait(q_full, k & 1, abort_flag) && next_load(kslot);
-        if (!ok) break;
-        tc_fence_after();
-        for (int t = 0; t < ntq; ++t) issue_qk(t, kslot, n_iter == 1);
+        ok = mbar_wait(q_full, k & 1, abort_flag, 4) && next_load(kslot);
+        for (int t = 0; t < ntq && ok; ++t) {
+          ok = wait_s_free();
+          if (!ok) break;
+          tc_fence_after();
+          issue_qk(t, kslot, n_iter == 1);
+        }
         for (int it = 0; it < n_iter && ok; ++it) {
           const bool more = it + 1 < n_iter;
           for (int t = 0; t < ntq && ok; ++t) {
-            ok = mbar_wait(p_full + t, ph_p[t], abort_flag);
+            if (more) {
+              if (t == 0) ok = next_load(kslot);
+              ok = ok && wait_s_free();
+              if (!ok) break;
+              tc_fence_after();
+              issue_qk(t, kslot, it + 2 == n_iter);
+            }
+            if (t == 0) ok = next_load(vslot);
+            ok = ok && mbar_wait(p_full + t, ph_p[t], abort_flag, 5);
             ph_p[t] ^= 1u;
-            if (ok && t == 0) ok = next_load(vslot);
             if (!ok) break;
             tc_fence_after();
             issue_pv(t, vslot, it > 0);
-            if (more) {
-              if (t == 0) {
-                ok = next_load(kslot);
-                if (!ok) break;
-                tc_fence_after();
-              }
-              issue_qk(t, kslot, it + 2 == n_iter);
-            }
           }
         }
         ++k;
@@ -271,6 +292,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
     const float c = P.c_log2;
     const float thr = kRescaleLog2 / c;
     int cnt = 0;  // iterations this tile's barriers have been through
+    uint32_t ph_pv = 0;  // pv_done[t] completes once per (item, iteration); every phase is waited for exactly once, in order
     bool ok = true;
     for (int id = blockIdx.x; id < P.n_items && ok; id += gridDim.x) {
       const Item I = decode_item(P, id);
@@ -299,13 +321,18 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
       float m_used = -INFINITY, l = 0.f;
 
       for (int it = 0; it < n_iter; ++it) {
-        ok = __all_sync(0xffffffffu, mbar_wait(s_full + t, (cnt + it) & 1, abort_flag));
+        ok = __all_sync(0xffffffffu, mbar_wait(s_full + t, (cnt + it) & 1, abort_flag, 6));
         if (!ok) break;
         tc_fence_after();
         uint32_t su[128];
 #pragma unroll
-        for (int cc = 0; cc < 4; ++cc) tmem_ld32(lane_addr + t * 128 + cc * 32, su + cc * 32);
+        for (int cc = 0; cc < 4; ++cc) tmem_ld32(lane_addr + Cfg::kColS + cc * 32, su + cc * 32);
         tmem_wait_ld();
+        // the scores are in registers: hand the S buffer to the next QK product
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(s_free);
+        bool pv_waited = (it == 0);  // PV(t, it-1) must be complete before O_t is rescaled or P_t overwritten
         float s[128];
 #pragma unroll
         for (int kx = 0; kx < 128; ++kx) s[kx] = __uint_as_float(su[kx]);
@@ -317,25 +344,33 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
 #pragma unroll
           for (int kx = 0; kx < 128; ++kx) s[kx] = kx < nv ? s[kx] : -INFINITY;
         }
-        float mx = fmaxf(s[0], s[1]);
+        float mxa = fmaxf(s[0], s[1]), mxb = fmaxf(s[2], s[3]), mxc = fmaxf(s[4], s[5]), mxd = fmaxf(s[6], s[7]);
 #pragma unroll
-        for (int kx = 2; kx < 128; kx += 2) mx = max3(mx, s[kx], s[kx + 1]);
+        for (int kx = 8; kx < 128; kx += 8) {  // four independent chains
+          mxa = max3(mxa, s[kx], s[kx + 1]);
+          mxb = max3(mxb, s[kx + 2], s[kx + 3]);
+          mxc = max3(mxc, s[kx + 4], s[kx + 5]);
+          mxd = max3(mxd, s[kx + 6], s[kx + 7]);
+        }
+        const float mx = fmaxf(fmaxf(mxa, mxb), fmaxf(mxc, mxd));
         const bool need = mx > m_used + thr;  // also true when m_used = -inf and the tile has a visible key
         if (it == 0) {
           if (need) m_used = mx;
         } else if (__any_sync(0xffffffffu, need)) {
-          ok = __all_sync(0xffffffffu, mbar_wait(pv_done + t, (cnt + it - 1) & 1, abort_flag));
+          ok = __all_sync(0xffffffffu, mbar_wait(pv_done + t, ph_pv, abort_flag, 7));
+          ph_pv ^= 1u;
+          pv_waited = true;
           if (!ok) break;
           tc_fence_after();
           const float f = need ? ex2((m_used - mx) * c) : 1.0f;
 #pragma unroll 1
           for (int cc = 0; cc < D / 32; ++cc) {
             uint32_t o[32];
-            tmem_ld32(lane_addr + Cfg::kOBase + t * D + cc * 32, o);
+            tmem_ld32(lane_addr + Cfg::kColO + t * 128 + cc * 32, o);
             tmem_wait_ld();
 #pragma unroll
             for (int kx = 0; kx < 32; ++kx) o[kx] = __float_as_uint(__uint_as_float(o[kx]) * f);
-            tmem_st32(lane_addr + Cfg::kOBase + t * D + cc * 32, o);
+            tmem_st32(lane_addr + Cfg::kColO + t * 128 + cc * 32, o);
           }
           tmem_wait_st();
           l *= f;
@@ -359,8 +394,14 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
           unpack2(l2, la, lb);
           l += la + lb;
         }
-        tmem_st32(lane_addr + t * 128, pk);
-        tmem_st32(lane_addr + t * 128 + 32, pk + 32);
+        if (!pv_waited) {
+          ok = __all_sync(0xffffffffu, mbar_wait(pv_done + t, ph_pv, abort_flag, 8));
+          ph_pv ^= 1u;
+          if (!ok) break;
+          tc_fence_after();
+        }
+        tmem_st32(lane_addr + Cfg::kColP + t * 64, pk);
+        tmem_st32(lane_addr + Cfg::kColP + t * 64 + 32, pk + 32);
         tmem_wait_st();
         tc_fence_before();
         __syncwarp();
@@ -368,14 +409,17 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
       }
 
       // ---- epilogue of this item (the MMA issuer cannot touch O_t again before this tile's next p_full arrive)
-      if (ok) ok = __all_sync(0xffffffffu, mbar_wait(pv_done + t, (cnt + n_iter - 1) & 1, abort_flag));
+      if (ok) {
+        ok = __all_sync(0xffffffffu, mbar_wait(pv_done + t, ph_pv, abort_flag, 9));
+        ph_pv ^= 1u;
+      }
       if (!ok) break;
       tc_fence_after();
       const float inv = l > 0.f ? 1.0f / l : 0.f;
 #pragma unroll 1
       for (int cc = 0; cc < D / 32; ++cc) {
         uint32_t o[32];
-        tmem_ld32(lane_addr + Cfg::kOBase + t * D + cc * 32, o);
+        tmem_ld32(lane_addr + Cfg::kColO + t * 128 + cc * 32, o);
         tmem_wait_ld();
         if (P.nsplit > 1) {
           float4 *dst = reinterpret_cast<float4 *>(P.part_o + pslot * D + cc * 32);
