@@ -36,6 +36,14 @@ constexpr float kRescaleLog2 = 8.0f;
 constexpr int kMaxOrdered = 128;
 }  // namespace
 
+// Optional clock trace of CTA 0 (build with -DDPARA_TRACE): g_trace[slot][n] = clock64() at trace point `slot`, n-th visit.
+#ifdef DPARA_TRACE
+__device__ long long g_trace[32 * 64];
+#define TRACE(slot, n) do { if (blockIdx.x == 0 && (n) < 64) g_trace[(slot) * 64 + (n)] = clock64(); } while (0)
+#else
+#define TRACE(slot, n) do {} while (0)
+#endif
+
 struct TcParams {
   CUtensorMap map_q, map_kc, map_vc, map_ks, map_vs, map_kb, map_vb;
   AttnParams a;
@@ -105,8 +113,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
   constexpr int kSlots = Cfg::kSlots;
   uint64_t *bars = reinterpret_cast<uint64_t *>(sKV + kSlots * Cfg::kTileBytes);
   uint64_t *kv_full = bars, *kv_empty = bars + kSlots, *q_full = bars + 2 * kSlots, *q_empty = q_full + 1, *s_full = q_full + 2,
-           *p_full = q_full + 4, *pv_done = q_full + 6, *s_free = q_full + 8;
-  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(q_full + 9);
+           *p_full = q_full + 4, *pv_done = q_full + 6, *sf_a = q_full + 8, *sf_b = q_full + 9;
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(q_full + 10);
   volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -114,11 +122,15 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
   if (P.nsplit == 1 && A.status_word && (*reinterpret_cast<volatile int32_t *>(A.status_word) & (int32_t)DPARA_STATUS_TIMEOUT)) return;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kSlots; ++s) { mbar_init(kv_full + s, 1); mbar_init(kv_empty + s, 1); }
+    // K/V slots and the Q buffer are released by BOTH MMA issuers
+    for (int s = 0; s < kSlots; ++s) { mbar_init(kv_full + s, 1); mbar_init(kv_empty + s, 2); }
     mbar_init(q_full, 1);
-    mbar_init(q_empty, 1);
+    mbar_init(q_empty, 2);
     for (int t = 0; t < 2; ++t) { mbar_init(s_full + t, 1); mbar_init(p_full + t, 4); mbar_init(pv_done + t, 1); }
-    mbar_init(s_free, 4);
+    // S hand-off: sf_a is waited for by tile 0's issuer only, sf_b by tile 1's only (one waiter per barrier, so
+    // every phase is consumed in order); the softmax warps arrive on the one the NEXT user of S waits for
+    mbar_init(sf_a, 4);
+    mbar_init(sf_b, 4);
     *abort_flag = 0;
     fence_barrier_init();
   }
@@ -193,92 +205,99 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
       ld += 2 * I.n_iter;
       ++k;
     }
-  } else if (warp == 9) {
-    // ------------------------------------------------------------------ MMA issuer
+  } else if (warp == 9 || warp == 10) {
+    // ------------------------------------------------------------------ MMA issuers: warp 9 for tile 0, warp 10 for tile 1
+    // One issuing thread per query tile.  A tcgen05.mma block issued into a drained pipe pays a start-up latency
+    // and the issuing thread spends the block's whole execution time issuing it (the queue is shallow); with
+    // one thread per tile, one tile's waits and commits overlap the other tile's products and the tensor pipe
+    // stays fed.  The two threads meet only through barriers (the S hand-off below, the K/V ring).
     if (lane == 0) {
-      // The issuing thread is on the critical path of every tile, so its instruction count matters:
-      // descriptors are built once and advanced with plain adds (the address field counts 16-byte units),
-      // ring slots and phases are tracked incrementally (no divisions).
+      const int ti = warp - 9;
       constexpr uint32_t idesc_qk = idesc_bf16_f32(128, 128, false, false);
       constexpr uint32_t idesc_pv = idesc_bf16_f32(128, D, false, true);
       constexpr uint32_t kTile16 = Cfg::kTileBytes >> 4;
-      const uint64_t qdesc[2] = {smem_desc_sw128(smem_u32(sQ), 16, 1024), smem_desc_sw128(smem_u32(sQ) + Cfg::kTileBytes, 16, 1024)};
+      const uint64_t qdesc = smem_desc_sw128(smem_u32(sQ) + ti * Cfg::kTileBytes, 16, 1024);
       const uint64_t kdesc0 = smem_desc_sw128(smem_u32(sKV), 16, 1024);                 // K tile: K-major operand
       const uint64_t vdesc0 = smem_desc_sw128(smem_u32(sKV), Cfg::kSlabBytes, 1024);    // V tile: MN-major operand
+      const uint32_t s_t = tmem + Cfg::kColS, o_t = tmem + Cfg::kColO + ti * 128, p_t = tmem + Cfg::kColP + ti * 64;
+      uint64_t *sf = ti == 0 ? sf_a : sf_b;
       int ring_slot = 0, k = 0;
-      uint32_t ring_phase = 0, ph_p[2] = {0, 0}, ph_sf = 0;
-      bool ok = true, first_qk = true;
-      auto next_load = [&](int &slot_out) {  // wait for the next tile of the K/V ring (loads are consumed in order)
+      uint32_t ring_phase = 0, ph_p = 0, ph_sf = 0;
+      bool ok = true, first_qk = (ti == 0);
+      auto next_load = [&](int &slot_out) {  // wait for the next tile of the K/V ring (both issuers take every tile, in order)
         slot_out = ring_slot;
-        const bool r = mbar_wait(kv_full + ring_slot, ring_phase, abort_flag);
+        const bool r = mbar_wait(kv_full + ring_slot, ring_phase, abort_flag, 2);
         if (++ring_slot == kSlots) { ring_slot = 0; ring_phase ^= 1u; }
         return r;
       };
-      // The single S buffer is handed back by the softmax warps of whichever tile read it last (also across
-      // items): every QK but the kernel's first waits for one phase of s_free.
+      // The S buffer comes back from whichever tile's softmax warps loaded it last (also across items).
       auto wait_s_free = [&]() {
         if (first_qk) { first_qk = false; return true; }
-        const bool r = mbar_wait(s_free, ph_sf, abort_flag, 3);
+        const bool r = mbar_wait(sf, ph_sf, abort_flag, 3);
         ph_sf ^= 1u;
         return r;
+      };
+      auto issue_qk = [&](int kslot, bool last_it) {
+        const uint64_t ka = kdesc0 + (uint64_t)(kslot * kTile16);
+#pragma unroll
+        for (int kk = 0; kk < D / 16; ++kk) {
+          const uint32_t off = ((kk >> 2) * Cfg::kSlabBytes + (kk & 3) * 32) >> 4;
+          if (kk == 0) mma_ss_c<false>(s_t, qdesc + off, ka + off, idesc_qk);
+          else mma_ss_c<true>(s_t, qdesc + off, ka + off, idesc_qk);
+        }
+        mma_commit(s_full + ti);
+        mma_commit(kv_empty + kslot);        // this tile is done with the K tile
+        if (last_it) mma_commit(q_empty);    // ... and with its Q tile
+      };
+      auto issue_pv = [&](int vslot, bool acc) {
+        const uint64_t va = vdesc0 + (uint64_t)(vslot * kTile16);
+        mma_ts(o_t, p_t, va, idesc_pv, acc);
+#pragma unroll
+        for (int kk = 1; kk < 8; ++kk) mma_ts_c<true>(o_t, p_t + kk * 8, va + (uint64_t)(kk * (2048 >> 4)), idesc_pv);
+        mma_commit(pv_done + ti);
+        mma_commit(kv_empty + vslot);
       };
       for (int id = blockIdx.x; id < P.n_items && ok; id += gridDim.x) {
         const Item I = decode_item(P, id);
         if (I.n_iter == 0) continue;
-        const int ntq = I.ntq, n_iter = I.n_iter;
-        auto issue_qk = [&](int t, int kslot, bool last_it) {
-          const uint64_t qa = qdesc[t], ka = kdesc0 + (uint64_t)(kslot * kTile16);
-#pragma unroll
-          for (int kk = 0; kk < D / 16; ++kk) {
-            const uint32_t off = ((kk >> 2) * Cfg::kSlabBytes + (kk & 3) * 32) >> 4;
-            if (kk == 0) mma_ss_c<false>(tmem + Cfg::kColS, qa + off, ka + off, idesc_qk);
-            else mma_ss_c<true>(tmem + Cfg::kColS, qa + off, ka + off, idesc_qk);
-          }
-          mma_commit(s_full + t);
-          if (t == ntq - 1) {
-            mma_commit(kv_empty + kslot);           // K tile consumed by every query tile
-            if (last_it) mma_commit(q_empty);       // last use of this item's Q tiles
-          }
-        };
-        auto issue_pv = [&](int t, int vslot, bool acc) {
-          const uint64_t va = vdesc0 + (uint64_t)(vslot * kTile16);
-          const uint32_t o_t = tmem + Cfg::kColO + t * 128, p_t = tmem + Cfg::kColP + t * 64;
-          mma_ts(o_t, p_t, va, idesc_pv, acc);
-#pragma unroll
-          for (int kk = 1; kk < 8; ++kk) mma_ts_c<true>(o_t, p_t + kk * 8, va + (uint64_t)(kk * (2048 >> 4)), idesc_pv);
-          mma_commit(pv_done + t);
-          if (t == ntq - 1) mma_commit(kv_empty + vslot);  // V tile consumed
-        };
-        // issue order per iteration: QK(0, it+1)  PV(0, it)  QK(1, it+1)  PV(1, it) -- each operation right
-        // where its inputs become ready in steady state (the S buffer comes back when the OTHER tile has
-        // loaded its scores; P_t arrives when tile t's softmax ends)
+        const int n_iter = I.n_iter;
         int kslot = 0, vslot = 0;
-        ok = mbar_wait(q_full, k & 1, abort_flag, 4) && next_load(kslot);
-        for (int t = 0; t < ntq && ok; ++t) {
-          ok = wait_s_free();
-          if (!ok) break;
-          tc_fence_after();
-          issue_qk(t, kslot, n_iter == 1);
+        ok = mbar_wait(q_full, k & 1, abort_flag, 4);
+        ++k;
+        if (!ok) break;
+        if (ti >= I.ntq) {
+          // no second tile in this item: keep the ring and Q-buffer protocols in step (a slot is released only
+          // after its load has landed, so this thread cannot run ahead of the other issuer by a ring cycle)
+          for (int q = 0; q < 2 * n_iter && ok; ++q) {
+            ok = next_load(kslot);
+            if (ok) mbar_arrive(kv_empty + kslot);
+          }
+          if (ok) mbar_arrive(q_empty);
+          continue;
         }
+        // per iteration: QK(it + 1), then PV(it) -- the scores of the next iteration are issued as soon as
+        // the S buffer and the K tile are there, the PV product when this tile's softmax has written P
+        ok = next_load(kslot) && wait_s_free();
+        if (!ok) break;
+        tc_fence_after();
+        issue_qk(kslot, n_iter == 1);
         for (int it = 0; it < n_iter && ok; ++it) {
-          const bool more = it + 1 < n_iter;
-          for (int t = 0; t < ntq && ok; ++t) {
-            if (more) {
-              if (t == 0) ok = next_load(kslot);
-              ok = ok && wait_s_free();
-              if (!ok) break;
-              tc_fence_after();
-              issue_qk(t, kslot, it + 2 == n_iter);
-            }
-            if (t == 0) ok = next_load(vslot);
-            ok = ok && mbar_wait(p_full + t, ph_p[t], abort_flag, 5);
-            ph_p[t] ^= 1u;
+          if (it + 1 < n_iter) {
+            TRACE(0 + 4 * ti, it);
+            ok = next_load(kslot) && wait_s_free();
             if (!ok) break;
             tc_fence_after();
-            issue_pv(t, vslot, it > 0);
+            TRACE(1 + 4 * ti, it);
+            issue_qk(kslot, it + 2 == n_iter);
           }
+          TRACE(2 + 4 * ti, it);
+          ok = next_load(vslot) && mbar_wait(p_full + ti, ph_p, abort_flag, 5);
+          ph_p ^= 1u;
+          if (!ok) break;
+          tc_fence_after();
+          TRACE(3 + 4 * ti, it);
+          issue_pv(vslot, it > 0);
         }
-        ++k;
       }
     }
   }
@@ -316,14 +335,21 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
         continue;
       }
       const int n_iter = I.n_iter;
+#ifdef DPARA_TRACE
+      const int kitem = (id - (int)blockIdx.x) / (int)gridDim.x;
+      if (warp == 0 && lane == 0) { TRACE(24, kitem); if (blockIdx.x == 0 && kitem < 64) g_trace[28 * 64 + kitem] = n_iter * 10 + I.ntq; }
+#endif
       const int na = max(0, min(j + A.pb, A.S));
       const int b0 = P.has_blk ? P.S8 + (j - I.jb0) * A.Bq : 0, b1 = P.has_blk ? b0 + A.Bq : 0;
       float m_used = -INFINITY, l = 0.f;
 
       for (int it = 0; it < n_iter; ++it) {
+        const bool tr = (wq == 0 && lane == 0);
+        if (tr) TRACE(8 + 8 * t, it);
         ok = __all_sync(0xffffffffu, mbar_wait(s_full + t, (cnt + it) & 1, abort_flag, 6));
         if (!ok) break;
         tc_fence_after();
+        if (tr) TRACE(9 + 8 * t, it);
         uint32_t su[128];
 #pragma unroll
         for (int cc = 0; cc < 4; ++cc) tmem_ld32(lane_addr + Cfg::kColS + cc * 32, su + cc * 32);
@@ -331,7 +357,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
         // the scores are in registers: hand the S buffer to the next QK product
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(s_free);
+        if (lane == 0) mbar_arrive((t == 0 && I.ntq == 2) ? sf_b : sf_a);  // next user: tile 1 of this iteration, else tile 0
+        if (tr) TRACE(10 + 8 * t, it);
         bool pv_waited = (it == 0);  // PV(t, it-1) must be complete before O_t is rescaled or P_t overwritten
         float s[128];
 #pragma unroll
@@ -376,6 +403,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
           l *= f;
           if (need) m_used = mx;
         }
+        if (tr) TRACE(11 + 8 * t, it);
         const float mc = (m_used == -INFINITY ? 0.f : m_used) * c;
         uint32_t pk[64];
         {
@@ -394,6 +422,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
           unpack2(l2, la, lb);
           l += la + lb;
         }
+        if (tr) TRACE(12 + 8 * t, it);
         if (!pv_waited) {
           ok = __all_sync(0xffffffffu, mbar_wait(pv_done + t, ph_pv, abort_flag, 8));
           ph_pv ^= 1u;
@@ -406,9 +435,13 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(p_full + t);
+        if (tr) TRACE(13 + 8 * t, it);
       }
 
       // ---- epilogue of this item (the MMA issuer cannot touch O_t again before this tile's next p_full arrive)
+#ifdef DPARA_TRACE
+      if (warp == 0 && lane == 0) TRACE(25, kitem);
+#endif
       if (ok) {
         ok = __all_sync(0xffffffffu, mbar_wait(pv_done + t, ph_pv, abort_flag, 9));
         ph_pv ^= 1u;
@@ -454,6 +487,9 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
         A.out_lse[orow] = l > 0.f ? (m_used * c + log2f(l)) * 0.6931471805599453f : -INFINITY;
       }
       cnt += n_iter;
+#ifdef DPARA_TRACE
+      if (warp == 0 && lane == 0) TRACE(26, kitem);
+#endif
     }
   }
 
@@ -662,3 +698,7 @@ dpara_status launch_attention_tc(const AttnParams &A, const TcPlan &plan, const 
 }
 
 }  // namespace dpara
+
+#ifdef DPARA_TRACE
+extern "C" int dpara_debug_read_trace(long long *host, int n) { return (int)cudaMemcpyFromSymbol(host, dpara::g_trace, sizeof(long long) * n); }
+#endif
