@@ -24,6 +24,11 @@
 // Every mbarrier wait is bounded; on expiry the CTA sets DPARA_STATUS_TIMEOUT and drains.
 #include <math.h>
 
+#include <algorithm>
+#include <queue>
+#include <utility>
+#include <vector>
+
 #include "attention_tc.cuh"
 #include "sm100_ptx.cuh"
 
@@ -34,6 +39,7 @@ namespace {
 constexpr int kThreads = 384;  // warps 0-7 softmax, 8 TMA producer, 9 MMA issuer, 10-11 idle (complete the third warpgroup)
 constexpr float kRescaleLog2 = 8.0f;
 constexpr int kMaxOrdered = 128;
+constexpr int kMaxSched = 3072;  // items a host-built schedule can hold (kernel parameter space)
 }  // namespace
 
 // Optional clock trace of CTA 0 (build with -DDPARA_TRACE): g_trace[slot][n] = clock64() at trace point `slot`, n-th visit.
@@ -55,6 +61,13 @@ struct TcParams {
   // launching the long requests first leaves the short ones to fill the tail of a ragged batch
   uint8_t req_order[kMaxOrdered];
   int use_order;
+  // Work schedule of the persistent CTAs (no KV split, more items than CTAs): CTA c runs items
+  // sched[cta_first[c]] .. sched[cta_first[c + 1] - 1].  The host balances the CTAs' loads (longest processing
+  // time first, each item to the least loaded CTA); a ragged batch has few items per CTA (about five at the
+  // benchmark shape), so handing them out round-robin leaves the most loaded CTA ~20 % above the mean.
+  int use_sched;
+  uint16_t cta_first[kNumSM + 1];
+  uint16_t sched[kMaxSched];
 };
 
 template <int D>
@@ -118,6 +131,10 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
   volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  // this CTA's items: its slice of the host-built schedule, else items blockIdx.x, blockIdx.x + gridDim.x, ...
+  const int q_begin = P.use_sched ? (int)P.cta_first[blockIdx.x] : (int)blockIdx.x;
+  const int q_end = P.use_sched ? (int)P.cta_first[blockIdx.x + 1] : P.n_items;
+  const int q_step = P.use_sched ? 1 : (int)gridDim.x;
   // (a CTA of a cluster must not leave early: its peers meet it at the cluster barriers below)
   if (P.nsplit == 1 && A.status_word && (*reinterpret_cast<volatile int32_t *>(A.status_word) & (int32_t)DPARA_STATUS_TIMEOUT)) return;
 
@@ -151,7 +168,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
     }
     int ld = 0, k = 0;  // running K/V load counter, processed-item counter
     bool ok = true;
-    for (int id = blockIdx.x; id < P.n_items && ok; id += gridDim.x) {
+    for (int qi = q_begin; qi < q_end && ok; qi += q_step) {
+      const int id = P.use_sched ? (int)P.sched[qi] : qi;
       const Item I = decode_item(P, id);
       if (I.n_iter == 0) continue;
       // the Q buffer is free once the previous item's last QK has completed
@@ -257,7 +275,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
         mma_commit(pv_done + ti);
         mma_commit(kv_empty + vslot);
       };
-      for (int id = blockIdx.x; id < P.n_items && ok; id += gridDim.x) {
+      for (int qi = q_begin; qi < q_end && ok; qi += q_step) {
+      const int id = P.use_sched ? (int)P.sched[qi] : qi;
         const Item I = decode_item(P, id);
         if (I.n_iter == 0) continue;
         const int n_iter = I.n_iter;
@@ -313,7 +332,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
     int cnt = 0;  // iterations this tile's barriers have been through
     uint32_t ph_pv = 0;  // pv_done[t] completes once per (item, iteration); every phase is waited for exactly once, in order
     bool ok = true;
-    for (int id = blockIdx.x; id < P.n_items && ok; id += gridDim.x) {
+    for (int qi = q_begin; qi < q_end && ok; qi += q_step) {
+      const int id = P.use_sched ? (int)P.sched[qi] : qi;
       const Item I = decode_item(P, id);
       const int ji = (I.pair * 2 + t) * P.JI_T + r / A.G;
       const bool valid = (t < I.ntq) && (r < P.JI_T * A.G) && (ji < P.n_ji);
@@ -336,7 +356,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
       }
       const int n_iter = I.n_iter;
 #ifdef DPARA_TRACE
-      const int kitem = (id - (int)blockIdx.x) / (int)gridDim.x;
+      const int kitem = (qi - q_begin) / q_step;
       if (warp == 0 && lane == 0) { TRACE(24, kitem); if (blockIdx.x == 0 && kitem < 64) g_trace[28 * 64 + kitem] = n_iter * 10 + I.ntq; }
 #endif
       const int na = max(0, min(j + A.pb, A.S));
@@ -689,6 +709,40 @@ dpara_status launch_attention_tc(const AttnParams &A, const TcPlan &plan, const 
       idx[c + 1] = v;
     }
     for (int n = 0; n < A.b; ++n) P.req_order[n] = (uint8_t)idx[n];
+  }
+  int sms = kNumSM, dev = 0;
+  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (plan.nsplit == 1 && P.n_items > sms && P.n_items <= kMaxSched && sms <= kNumSM) {
+    // cost model in SM clocks, from traces of this kernel: an iteration (128 keys) of a two-tile item, of a
+    // one-tile item, and the fixed part of an item (Q load, first scores, epilogue)
+    const int X = plan.n_pairs, per_req = X * A.Hkv;
+    std::vector<std::pair<int, int>> cost(P.n_items);  // (cost, id)
+    for (int id = 0; id < P.n_items; ++id) {
+      const int z = id / per_req, x = id % X;
+      const int n = P.use_order ? (int)P.req_order[z] : z;
+      const long long L = host_off[n + 1] - host_off[n];
+      const int n_iter = (int)((L + 127) >> 7) + (P.has_tail ? 1 : 0);
+      const int ntq = std::min(2, plan.n_tiles - x * 2);
+      cost[id] = {n_iter * (ntq == 2 ? 3200 : 1800) + 6000, id};
+    }
+    std::stable_sort(cost.begin(), cost.end(), [](const std::pair<int, int> &a, const std::pair<int, int> &b) { return a.first > b.first; });
+    typedef std::pair<long long, int> Load;  // (load, CTA): least loaded first, ties to the lower CTA
+    std::priority_queue<Load, std::vector<Load>, std::greater<Load>> heap;
+    for (int c = 0; c < sms; ++c) heap.push({0, c});
+    std::vector<std::vector<uint16_t>> lists(sms);
+    for (const auto &ci : cost) {
+      Load l = heap.top();
+      heap.pop();
+      lists[l.second].push_back((uint16_t)ci.second);
+      heap.push({l.first + ci.first, l.second});
+    }
+    int q = 0;
+    for (int c = 0; c < sms; ++c) {
+      P.cta_first[c] = (uint16_t)q;
+      for (uint16_t id : lists[c]) P.sched[q++] = id;
+    }
+    for (int c = sms; c <= kNumSM; ++c) P.cta_first[c] = (uint16_t)q;
+    P.use_sched = 1;
   }
   if (plan.nsplit > 1) {
     P.part_o = static_cast<float *>(workspace);
