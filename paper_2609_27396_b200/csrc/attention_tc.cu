@@ -723,7 +723,7 @@ dpara_status launch_attention_tc(const AttnParams &A, const TcPlan &plan, const 
       const long long L = host_off[n + 1] - host_off[n];
       const int n_iter = (int)((L + 127) >> 7) + (P.has_tail ? 1 : 0);
       const int ntq = std::min(2, plan.n_tiles - x * 2);
-      cost[id] = {n_iter * (ntq == 2 ? 3200 : 1800) + 6000, id};
+      cost[id] = {n_iter * (ntq == 2 ? 3300 : 2700) + 11000, id};
     }
     std::stable_sort(cost.begin(), cost.end(), [](const std::pair<int, int> &a, const std::pair<int, int> &b) { return a.first > b.first; });
     typedef std::pair<long long, int> Load;  // (load, CTA): least loaded first, ties to the lower CTA
