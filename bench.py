@@ -31,12 +31,12 @@ import workloads as W  # noqa: E402
 
 METRIC = "all_boundary_draft_step_us"
 L2_FLUSH_BYTES = 256 << 20
-# dram__bytes_read.sum + dram__bytes_write.sum of one attention launch, from the ncu capture summarised in
-# profiles/attention_tc_cfg3_b16.md (bytes per launch; None where no capture exists)
-NCU_DRAM_TRAFFIC = {"cfg3": 266551296, "cfg2": None}
+# dram__bytes_read.sum + dram__bytes_write.sum of one attention launch, from an ncu capture of this command's
+# workload (bytes per launch; None where no capture exists)
+NCU_DRAM_TRAFFIC = {"cfg3": 369188608, "cfg2": None}
 
 
-# ----------------------------------------------------------------------------- algorithmic work
+# ----------------------------------------------------------------------------- algorithmic work (flops and bytes every launch must do)
 def attention_flops(sh: W.AttnShape) -> float:
     """4 * D flops per (query row, visible key): QK^T and PV."""
     rows_per_boundary = sh.block * sh.n_q_heads

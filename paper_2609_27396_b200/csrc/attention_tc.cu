@@ -9,7 +9,7 @@
 //               (order K0 K1 V0 K2 V1 ...).  The context needs no mask at all (every row sees the whole
 //               cache); the spine prefix and the boundaries' own blocks are packed into ONE extra "tail"
 //               tile per CTA.
-//   warp 9      one thread issues tcgen05.mma:  S = Q_t K^T  (A, B from shared memory) and
+//   warps 9, 10 one thread per query tile issues tcgen05.mma:  S = Q_t K^T  (A, B from shared memory) and
 //               O_t += P_t V  (A = P_t from tensor memory, B = V, MN-major).
 //   warps 0-3   softmax of tile 0, warps 4-7 softmax of tile 1: thread = row.  tcgen05.ld the S row into
 //               registers and hand the S buffer back at once; mask (tail tile only: anchor prefix of the
@@ -36,7 +36,7 @@ namespace dpara {
 using namespace ptx;
 
 namespace {
-constexpr int kThreads = 384;  // warps 0-7 softmax, 8 TMA producer, 9 MMA issuer, 10-11 idle (complete the third warpgroup)
+constexpr int kThreads = 384;  // warps 0-7 softmax, 8 TMA producer, 9 and 10 MMA issuers, 11 idle (completes the third warpgroup)
 constexpr float kRescaleLog2 = 8.0f;
 constexpr int kMaxOrdered = 128;
 constexpr int kMaxSched = 3072;  // items a host-built schedule can hold (kernel parameter space)
