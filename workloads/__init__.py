@@ -98,6 +98,18 @@ class LayerShape:
 
 
 @dataclass(frozen=True)
+class HeadShape:
+    """Critical-path remainder: LM head on the selected branch + the autoregressive head loop."""
+    batch: int
+    block: int                 # d = draft length = rows per selected branch
+    hidden: int
+    vocab: int
+    rank: int = 256            # width of the head's low-rank token embedding (the paper gives no number)
+    lm_sigma: float = 0.02
+    ar_sigma: float = 0.05
+
+
+@dataclass(frozen=True)
 class Workload:
     name: str
     index: int
@@ -264,6 +276,35 @@ def make_layer_inputs(layer: LayerShape, attn: AttnShape, seed: int) -> LayerInp
     w_down = _normal_bf16(rng, (H, I), s)
     gains = [f32_to_bf16_bits(1.0 + 0.1 * rng.standard_normal(n, dtype=np.float32)) for n in (H, H, D, D)]
     return LayerInputs(layer, x, w_qkv, w_o, w_gate_up, w_down, *gains)
+
+
+@dataclass
+class HeadInputs:
+    shape: HeadShape
+    sel_reps: np.ndarray   # [b][d][hidden] bf16 bits: the selected branches' final hidden states
+    w_lm: np.ndarray       # [V][hidden] bf16 bits
+    ar_w: np.ndarray       # [V][rank] bf16 bits (W)
+    ar_e: np.ndarray       # [V][rank] bf16 bits (E)
+    bonus: np.ndarray      # [b] int32
+
+
+def head_shape(w: Workload, rank: int = 256) -> HeadShape:
+    v = w.verify
+    return HeadShape(v.batch, v.block, v.hidden, v.vocab, rank)
+
+
+def make_head_inputs(shape: HeadShape, seed: int) -> HeadInputs:
+    """Unit-variance hidden states; N(0, lm_sigma^2) head weights (base logits with standard deviation
+    lm_sigma * sqrt(hidden), 1.4 at hidden 5120); W ~ N(0, 1), E ~ N(0, ar_sigma^2), so the correction W E(y) has
+    standard deviation ar_sigma * sqrt(rank) (0.8 at rank 256): comparable to the base logits' spread, the
+    previous token really changes the argmax."""
+    rng = np.random.Generator(np.random.Philox(seed ^ 0x4EAD))
+    reps = _normal_bf16(rng, (shape.batch, shape.block, shape.hidden))
+    w_lm = _normal_bf16(rng, (shape.vocab, shape.hidden), shape.lm_sigma)
+    ar_w = _normal_bf16(rng, (shape.vocab, shape.rank), 1.0)
+    ar_e = _normal_bf16(rng, (shape.vocab, shape.rank), shape.ar_sigma)
+    bonus = rng.integers(0, shape.vocab, size=shape.batch).astype(np.int32)
+    return HeadInputs(shape, reps, w_lm, ar_w, ar_e, bonus)
 
 
 def scaled(w: Workload, **kw) -> Workload:
