@@ -191,6 +191,36 @@ dpara_status dpara_verify_select(const dpara_verify_io *io, void *workspace, siz
 #define DPARA_VERIFY_STATIC_SCRATCH_BYTES (256u * 1024u)
 dpara_status dpara_verify_select_static(const dpara_verify_io *io, int32_t *status_word, void *stream);
 
+/* The critical-path remainder T_Head (Alg. 1, the lines after the barrier: "select precomputed branch r; y_0 = b;
+ * for i = 1..d: z_i = l_i + W E(y_{i-1}), y_i ~ softmax(z_i)"; Sec. 3.2 "Loss" defines the head: E is its own
+ * low-rank token embedding, W projects it to the vocabulary, and it reads only the preceding token).  The base
+ * logits l_i are the language-model head applied to the selected branch's final hidden states (App. D runs the
+ * language-model head on shipped hidden states right before the head loop).  Greedy decoding (Table 1): y_i is the
+ * lowest index holding the maximum of z_i; NaN ranks below every number.
+ *   sel_reps     device [b][block][hidden] bf16: the selected branches (the `selected` output of dpara_verify_select)
+ *   w_lm         device [vocab][hidden] bf16 (weights stored [out][in])
+ *   ar_w, ar_e   device [vocab][rank] bf16: W (one row per vocabulary entry) and E (one row per token)
+ *   bonus        device [b] int32: y_0 of each request; a value outside [0, vocab) sets DPARA_STATUS_BAD_TOKEN in
+ *                *status_word and is treated as token 0
+ *   next_tokens  device [b][block] int32 out: y_1 .. y_d
+ * bf16 products with fp32 accumulation; z_i = (fp32 base logit) + (fp32 correction), compared in fp32.
+ * Workspace: dpara_head_workspace_bytes(b, block, vocab) bytes of device memory, 16-byte aligned, owned by the
+ * caller and private to the call while it runs (it holds the fp32 base logits [b * block][vocab]).
+ * All work is queued on `stream`; nothing is allocated.  Errors: INVALID_ARG (null or misaligned pointer,
+ * non-positive size), UNSUPPORTED (b > 32, block > 64, rank not a multiple of 64 or > 256, hidden % 64 != 0,
+ * vocab % 8 != 0), CUDA.  A device-side wait that runs out sets DPARA_STATUS_TIMEOUT in *status_word. */
+typedef struct {
+  const void *sel_reps;
+  const void *w_lm;
+  const void *ar_w;
+  const void *ar_e;
+  const int32_t *bonus;
+  int32_t *next_tokens;
+  int32_t b, block, hidden, vocab, rank;
+} dpara_head_io;
+size_t dpara_head_workspace_bytes(int32_t b, int32_t block, int32_t vocab);
+dpara_status dpara_draft_head(const dpara_head_io *io, void *workspace, size_t workspace_bytes, int32_t *status_word, void *stream);
+
 const char *dpara_status_string(dpara_status s);
 
 /* Library/ABI version: major * 1000 + minor. */
@@ -201,7 +231,7 @@ int32_t dpara_version(void);
  *   out[M][N] = epilogue( a[M][K] * w[N][K]^T ),  a and w bf16 row-major (weights stored [out][in]).
  * epilogue 0: out bf16.   epilogue 1: out fp32 = resid + product (resid [M][N], bf16 when
  * resid_dtype == DPARA_BF16 else fp32), optional bf16 copy in out_bf16.   epilogue 2: w holds 2N rows,
- * [0,N) gate and [N,2N) up; out bf16 = silu(a Wg^T) * (a Wu^T).
+ * [0,N) gate and [N,2N) up; out bf16 = silu(a Wg^T) * (a Wu^T).   epilogue 3: out fp32 = product.
  * No workspace.  Errors: INVALID_ARG (null/misaligned), UNSUPPORTED (K % 64 != 0 or N % 8 != 0), CUDA. */
 typedef struct {
   const void *a;

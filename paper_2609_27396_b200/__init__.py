@@ -90,7 +90,7 @@ def gemm_bf16(a, w, *, epilogue: int = 0, resid=None, want_bf16_copy: bool = Fal
     """dpara_gemm_bf16: out = epilogue(a @ w.T); a [M][K], w [N][K] (epilogue 2: [2N][K]) bf16 CUDA tensors."""
     M, K = a.shape
     N = w.shape[0] // 2 if epilogue == 2 else w.shape[0]
-    out = torch.empty((M, N), dtype=torch.float32 if epilogue == 1 else torch.bfloat16, device=a.device)
+    out = torch.empty((M, N), dtype=torch.float32 if epilogue in (1, 3) else torch.bfloat16, device=a.device)
     out16 = torch.empty((M, N), dtype=torch.bfloat16, device=a.device) if (want_bf16_copy and epilogue == 1) else None
     st = status if status is not None else torch.zeros(1, dtype=torch.int32, device=a.device)
     io = GemmIO(_ptr(a), _ptr(w), M, N, K, epilogue, _ptr(resid),
@@ -252,3 +252,51 @@ def verify_select(target, draft_tokens, reps=None, *, mode: int = 0, draft_probs
     plan(target=target, draft_tokens=draft_tokens, reps=reps, draft_probs=draft_probs, uniforms=uniforms, stream=stream)
     return dict(accept_len=plan.accept_len, bonus=plan.bonus, gather_idx=plan.gather_idx, out_tokens=plan.out_tokens,
                 selected=plan.selected if reps is not None else None, status=plan.status)
+
+
+# ----------------------------------------------------------------------------- critical-path remainder: LM head + AR head loop
+class HeadIO(C.Structure):
+    _fields_ = [("sel_reps", C.c_void_p), ("w_lm", C.c_void_p), ("ar_w", C.c_void_p), ("ar_e", C.c_void_p),
+                ("bonus", C.c_void_p), ("next_tokens", C.c_void_p), ("b", C.c_int32), ("block", C.c_int32),
+                ("hidden", C.c_int32), ("vocab", C.c_int32), ("rank", C.c_int32)]
+
+
+lib.dpara_head_workspace_bytes.restype = C.c_size_t
+lib.dpara_head_workspace_bytes.argtypes = [C.c_int32, C.c_int32, C.c_int32]
+lib.dpara_draft_head.restype = C.c_int
+lib.dpara_draft_head.argtypes = [C.POINTER(HeadIO), C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
+EXPORTED += ["dpara_head_workspace_bytes", "dpara_draft_head"]
+
+
+class HeadPlan:
+    """Buffers of dpara_draft_head for fixed shapes (allocated once; a call allocates nothing)."""
+
+    def __init__(self, b: int, block: int, hidden: int, vocab: int, rank: int, device="cuda"):
+        self.b, self.block, self.hidden, self.vocab, self.rank = b, block, hidden, vocab, rank
+        self.workspace_bytes = int(lib.dpara_head_workspace_bytes(b, block, vocab))
+        self.workspace = torch.empty(self.workspace_bytes, dtype=torch.uint8, device=device)
+        self.next_tokens = torch.full((b, block), -1, dtype=torch.int32, device=device)
+        self.status = torch.zeros(1, dtype=torch.int32, device=device)
+
+    def base_logits(self) -> torch.Tensor:
+        """View of the fp32 base logits [b * block][vocab] the last call left in the workspace."""
+        n = self.b * self.block * self.vocab
+        return self.workspace[: n * 4].view(torch.float32).view(self.b * self.block, self.vocab)
+
+    def run(self, sel_reps, w_lm, ar_w, ar_e, bonus, stream=None):
+        io = HeadIO(_ptr(sel_reps), _ptr(w_lm), _ptr(ar_w), _ptr(ar_e), _ptr(bonus), _ptr(self.next_tokens),
+                    self.b, self.block, self.hidden, self.vocab, self.rank)
+        rc = lib.dpara_draft_head(C.byref(io), self.workspace.data_ptr(), self.workspace_bytes, self.status.data_ptr(),
+                                  _stream_ptr(stream))
+        if rc != OK:
+            raise DparaError(rc)
+        return self.next_tokens
+
+
+def draft_head(sel_reps, w_lm, ar_w, ar_e, bonus, stream=None):
+    """dpara_draft_head: sel_reps [b][block][hidden], w_lm [vocab][hidden], ar_w / ar_e [vocab][rank] (bf16 CUDA
+    tensors), bonus [b] int32.  Returns (next_tokens [b][block] int32, plan)."""
+    b, block, hidden = sel_reps.shape
+    plan = HeadPlan(b, block, hidden, w_lm.shape[0], ar_w.shape[1], sel_reps.device)
+    plan.run(sel_reps, w_lm, ar_w, ar_e, bonus, stream)
+    return plan.next_tokens, plan

@@ -92,9 +92,25 @@ extern "C" int64_t dpara_kernel_launches(void) { return g_launches.load(std::mem
 
 extern "C" dpara_status dpara_gemm_bf16(const dpara_gemm_io *io, int32_t *status_word, void *stream) {
   if (!io) return DPARA_ERR_INVALID_ARG;
-  if (io->epilogue < 0 || io->epilogue > 2) return DPARA_ERR_INVALID_ARG;
+  if (io->epilogue < 0 || io->epilogue > 3) return DPARA_ERR_INVALID_ARG;
   GemmArgs g;
   g.a = io->a; g.w = io->w; g.M = io->M; g.N = io->N; g.K = io->K; g.epi = io->epilogue;
   g.resid = io->resid; g.resid_bf16 = io->resid_dtype == DPARA_BF16; g.out = io->out; g.out_bf16 = io->out_bf16;
   return launch_gemm_tc(g, status_word, static_cast<cudaStream_t>(stream));
+}
+
+#include "head.cuh"
+
+extern "C" size_t dpara_head_workspace_bytes(int32_t b, int32_t block, int32_t vocab) { return head_workspace_bytes(b, block, vocab); }
+
+extern "C" dpara_status dpara_draft_head(const dpara_head_io *io, void *workspace, size_t workspace_bytes, int32_t *status_word,
+                                         void *stream) {
+  if (!io) return DPARA_ERR_INVALID_ARG;
+  if (io->b <= 0 || io->block <= 0 || io->vocab <= 0) return DPARA_ERR_INVALID_ARG;
+  const size_t need = head_workspace_bytes(io->b, io->block, io->vocab);
+  if (!workspace || workspace_bytes < need || !aligned16(workspace)) return DPARA_ERR_WORKSPACE;
+  HeadArgs h;
+  h.sel_reps = io->sel_reps; h.w_lm = io->w_lm; h.ar_w = io->ar_w; h.ar_e = io->ar_e; h.bonus = io->bonus;
+  h.next_tokens = io->next_tokens; h.b = io->b; h.block = io->block; h.hidden = io->hidden; h.vocab = io->vocab; h.rank = io->rank;
+  return launch_head(h, workspace, status_word, static_cast<cudaStream_t>(stream));
 }

@@ -8,10 +8,10 @@ struct GemmArgs {
   const void *a;      // [M][K] bf16, row-major
   const void *w;      // [N][K] bf16 (epi 2: [2N][K], rows [0,N) gate and [N,2N) up)
   int M, N, K;        // N = output columns
-  int epi;            // 0 bf16 store; 1 fp32 out = resid + acc (+ bf16 copy); 2 bf16 out = silu(gate) * up
+  int epi;            // 0 bf16 store; 1 fp32 out = resid + acc (+ bf16 copy); 2 bf16 out = silu(gate) * up; 3 fp32 store
   const void *resid;  // epi 1: [M][N] bf16 or fp32
   int resid_bf16;
-  void *out;          // [M][N] bf16 (epi 0, 2) or fp32 (epi 1)
+  void *out;          // [M][N] bf16 (epi 0, 2) or fp32 (epi 1, 3)
   void *out_bf16;     // epi 1: optional bf16 copy of out
 };
 

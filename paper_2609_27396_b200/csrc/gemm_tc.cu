@@ -9,6 +9,7 @@
 //   2  bf16 out = silu(gate) * up                   (gate/up projection: the tile's 256 accumulator
 //                                                    columns are 128 gate columns and the matching 128
 //                                                    up columns, so the activation never leaves the SM)
+//   3  fp32 store                                   (LM head: base logits)
 // Every mbarrier wait is bounded; on expiry the CTA sets DPARA_STATUS_TIMEOUT and drains.
 #include "gemm.cuh"
 #include "sm100_ptx.cuh"
@@ -197,7 +198,9 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
               for (int v = 0; v < 8; ++v) {
                 if (cb + v * 4 < P.N) {
                   float x[4];
-                  if (P.resid_bf16) {
+                  if (P.epi == 3) {
+                    x[0] = x[1] = x[2] = x[3] = 0.f;
+                  } else if (P.resid_bf16) {
                     uint2 rr = *reinterpret_cast<const uint2 *>(static_cast<const uint16_t *>(P.resid) + (size_t)row * P.N + cb + v * 4);
                     x[0] = bf16lo(rr.x); x[1] = bf16hi(rr.x); x[2] = bf16lo(rr.y); x[3] = bf16hi(rr.y);
                   } else {
@@ -234,7 +237,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
 dpara_status launch_gemm_tc(const GemmArgs &g, int32_t *status, cudaStream_t st) {
   if (g.M <= 0 || g.N <= 0 || g.K <= 0) return DPARA_ERR_INVALID_ARG;
   if (g.K % kBK != 0 || g.N % 8 != 0) return DPARA_ERR_UNSUPPORTED;
-  if (!g.a || !g.w || !g.out || (g.epi == 1 && !g.resid)) return DPARA_ERR_INVALID_ARG;
+  if (g.epi < 0 || g.epi > 3 || !g.a || !g.w || !g.out || (g.epi == 1 && !g.resid)) return DPARA_ERR_INVALID_ARG;
   if (!aligned16(g.a) || !aligned16(g.w) || !aligned16(g.out) || !aligned16(g.resid) || !aligned16(g.out_bf16)) return DPARA_ERR_INVALID_ARG;
   GemmKernelParams P;
   const int w_rows = g.epi == 2 ? 2 * g.N : g.N;
