@@ -240,6 +240,53 @@ class LayerRunner:
         return [(e[0].elapsed_time(e[2]), e[0].elapsed_time(e[1]), e[1].elapsed_time(e[2])) for e in ev]
 
 
+class HeadRunner:
+    """The critical-path remainder T_Head at the main workload's shape: LM head on the selected branches
+    (b * d rows against the [vocab][hidden] weight) + the autoregressive head loop (d dependent steps)."""
+
+    def __init__(self, wl: W.Workload, seed: int, rank: int = 256):
+        import torch
+        import paper_2609_27396_b200 as dp
+        self.torch, self.dp = torch, dp
+        self.shape = W.head_shape(wl, rank)
+        inp = W.make_head_inputs(self.shape, seed)
+        bf = lambda bits: torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda().view(torch.bfloat16)
+        self.t = [bf(x) for x in (inp.sel_reps, inp.w_lm, inp.ar_w, inp.ar_e)]
+        self.bonus = torch.from_numpy(inp.bonus).cuda()
+        sh = self.shape
+        self.plan = dp.HeadPlan(sh.batch, sh.block, sh.hidden, sh.vocab, sh.rank)
+        self.flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device="cuda")
+
+    def step(self):
+        self.plan.run(*self.t, self.bonus)
+
+    def lm_head_only(self):
+        sh = self.shape
+        return self.dp.gemm_bf16(self.t[0].view(sh.batch * sh.block, sh.hidden), self.t[1], epilogue=3, status=self.plan.status)
+
+    def timed(self, k: int, lm_only: bool = False):
+        torch = self.torch
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(k)]
+        for s in range(k):
+            self.flush.zero_()
+            ev[s][0].record()
+            if lm_only:
+                self.lm_head_only()
+            else:
+                self.step()
+            ev[s][1].record()
+        torch.cuda.synchronize()
+        return [e[0].elapsed_time(e[1]) for e in ev]
+
+
+def head_bytes(sh: W.HeadShape):
+    """Algorithmic HBM bytes of T_Head: LM head = weight once + hidden rows + fp32 logits written; head loop = the
+    logits read back once (each step reads its own rows) + W once (it is re-read every step, from L2) + E rows."""
+    lm = sh.vocab * sh.hidden * 2 + sh.batch * sh.block * sh.hidden * 2 + sh.batch * sh.block * sh.vocab * 4
+    ar = sh.batch * sh.block * sh.vocab * 4 + sh.vocab * sh.rank * 2 + sh.batch * sh.block * sh.rank * 2
+    return lm, ar
+
+
 def layer_gemm_flops(a: W.AttnShape, l: W.LayerShape) -> float:
     M = a.batch * a.n_boundaries * a.block
     qd, kd = a.n_q_heads * a.head_dim, a.n_kv_heads * a.head_dim
@@ -306,6 +353,7 @@ def main():
     ap.add_argument("--workload", default="cfg3", choices=["cfg2", "cfg3"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-layer", action="store_true", help="skip the full-layer (cfg5) leg")
+    ap.add_argument("--no-head", action="store_true", help="skip the LM head + autoregressive head loop (T_Head) leg")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -433,6 +481,22 @@ def main():
                                  "flops": fl5, "tflops": fl5 / (d5 * 1e-6) / 1e12,
                                  "tensor_frac_of_measured_sustained": fl5 / (d5 * 1e-6) / 1e12 / (peaks["bf16_tflops_sustained"] or peaks["bf16_tflops"])}
             del r5
+        if not args.no_head:
+            rh = HeadRunner(wl, wl.seed)
+            for _ in range(3):
+                rh.step()
+            th = statistics.median(rh.timed(max(5, min(args.steps, 10)))) * 1e3
+            tl = statistics.median(rh.timed(max(5, min(args.steps, 10)), lm_only=True)) * 1e3
+            lmb, arb = head_bytes(rh.shape)
+            sh = rh.shape
+            out["head"] = {"workload": "T_Head at %s: b=%d, d=%d, hidden=%d, vocab=%d, head rank=%d (greedy)" % (wl.name, sh.batch, sh.block, sh.hidden, sh.vocab, sh.rank),
+                           "head_us": th, "lm_head_us": tl, "ar_loop_us": th - tl, "ar_step_us": (th - tl) / sh.block,
+                           "lm_head": {"bound": "hbm", "achieved": lmb / (tl * 1e-6) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                       "frac": lmb / (tl * 1e-6) / 1e9 / peaks["hbm_gbs"], "bytes": lmb,
+                                       "tflops": 2.0 * sh.batch * sh.block * sh.hidden * sh.vocab / (tl * 1e-6) / 1e12},
+                           "ar_loop": {"w_bytes_per_step": sh.vocab * sh.rank * 2, "hbm_bytes": arb,
+                                       "w_read_gbs": sh.vocab * sh.rank * 2 * sh.block / ((th - tl) * 1e-6) / 1e9}}
+            del rh
         if not args.no_cpu_baseline:
             t, est, desc = oracle_sample(wl, wl.seed, 0, wl.verify.batch, run.inp, run.ver)
             out["cpu_baseline"] = {"value": est * 1e6, "unit": "us", "cores": oracle_threads(), "kind": "oracle", "sample": desc,

@@ -279,9 +279,11 @@ class HeadPlan:
         self.status = torch.zeros(1, dtype=torch.int32, device=device)
 
     def base_logits(self) -> torch.Tensor:
-        """View of the fp32 base logits [b * block][vocab] the last call left in the workspace."""
+        """The fp32 base logits the last call left in the workspace (stored step-major [block][b][vocab]), as
+        [b * block][vocab] in request-major row order."""
         n = self.b * self.block * self.vocab
-        return self.workspace[: n * 4].view(torch.float32).view(self.b * self.block, self.vocab)
+        return self.workspace[: n * 4].view(torch.float32).view(self.block, self.b, self.vocab).permute(1, 0, 2).reshape(
+            self.b * self.block, self.vocab)
 
     def run(self, sel_reps, w_lm, ar_w, ar_e, bonus, stream=None):
         io = HeadIO(_ptr(sel_reps), _ptr(w_lm), _ptr(ar_w), _ptr(ar_e), _ptr(bonus), _ptr(self.next_tokens),

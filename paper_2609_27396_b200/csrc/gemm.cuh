@@ -13,6 +13,7 @@ struct GemmArgs {
   int resid_bf16;
   void *out;          // [M][N] bf16 (epi 0, 2) or fp32 (epi 1, 3)
   void *out_bf16;     // epi 1: optional bf16 copy of out
+  int perm_block = 0, perm_b = 0;  // epi 3 only, if set: output row (n * perm_block + i) is stored at row (i * perm_b + n)
 };
 
 dpara_status launch_gemm_tc(const GemmArgs &g, int32_t *status, cudaStream_t st);

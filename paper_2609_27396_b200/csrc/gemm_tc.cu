@@ -37,6 +37,7 @@ struct GemmKernelParams {
   int resid_bf16;
   void *out_bf16;
   int32_t *status;
+  int perm_block, perm_b;
 };
 
 __device__ __forceinline__ float silu_f(float g) { return g / (1.0f + __expf(-g)); }
@@ -193,7 +194,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
                 }
               }
             } else {
-              float *o = static_cast<float *>(P.out) + (size_t)row * P.N + cb;
+              const int orow = P.perm_block ? (row % P.perm_block) * P.perm_b + row / P.perm_block : row;
+              float *o = static_cast<float *>(P.out) + (size_t)orow * P.N + cb;
 #pragma unroll
               for (int v = 0; v < 8; ++v) {
                 if (cb + v * 4 < P.N) {
@@ -245,6 +247,7 @@ dpara_status launch_gemm_tc(const GemmArgs &g, int32_t *status, cudaStream_t st)
   if (!make_tmap_bf16_2d(&P.map_b, g.w, g.K, w_rows, (uint64_t)g.K * 2, kBK, 128)) return DPARA_ERR_CUDA;
   P.M = g.M; P.N = g.N; P.K = g.K; P.epi = g.epi; P.up_row_offset = g.N;
   P.out = g.out; P.resid = g.resid; P.resid_bf16 = g.resid_bf16; P.out_bf16 = g.out_bf16; P.status = status;
+  P.perm_block = g.epi == 3 ? g.perm_block : 0; P.perm_b = g.perm_b;
   if (cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess) return DPARA_ERR_CUDA;
   const int tile_cols = g.epi == 2 ? 128 : kBN;
   const int tiles = ((g.N + tile_cols - 1) / tile_cols) * ((g.M + kBM - 1) / kBM);

@@ -6,12 +6,14 @@
 // embedding rows E(y_{i-1}) -- 0.6 GFLOP and one pass over W (78 MB at vocab 151 936, rank 256, which stays in
 // L2) per step.  ONE persistent cooperative kernel runs all d steps:
 //   warp 4      TMA producer: streams this CTA's 128-row tiles of W through a ring of shared-memory stages (the
-//               tiles do not depend on the tokens, so the ring runs ahead across steps);
+//               tiles do not depend on the tokens, so the ring runs ahead across steps), and with each tile the
+//               b x 128 block of base logits it will be added to (plain loads of those from the epilogue queued
+//               behind the deep W stream and cost 1.6 us each; as part of the stage they cost nothing);
 //   warp 5      one thread issues tcgen05.mma: D[128 vocab rows][nb] = W_tile[128][rank] * Ey[nb][rank]^T
 //               (M = 128, N = nb = 16 or 32, both operands K-major in shared memory, 128-byte swizzle);
 //   warps 0-3   build Ey in shared memory at the start of a step (gather of E rows, swizzled by hand), then for
 //               every tile: tcgen05.ld the accumulator (thread = vocab row), add the base logit of each
-//               request (coalesced fp32 loads), keep the running (value, index) maximum per request;
+//               request (from the stage), keep the running (value, index) maximum per request;
 //               at the end of the step a warp reduction and one 64-bit atomicMax per request and warp.
 // Between steps the CTAs meet at a grid barrier (a counter in global memory; the launch is cooperative, so all
 // CTAs are resident; the wait is bounded by wall time and gives up with DPARA_STATUS_TIMEOUT).
@@ -28,6 +30,7 @@ namespace {
 constexpr int kThreads = 192;
 constexpr int kMaxBatch = 32;
 constexpr int kAccCols = 32;  // TMEM columns per accumulator buffer (nb <= 32)
+constexpr int kBestStride = 16;  // 64-bit words between two requests' maxima: one 128-byte line (one L2 atomic unit) each
 
 __device__ __forceinline__ uint32_t head_key(float f) {
   if (f != f) return 0u;                    // NaN below everything
@@ -39,11 +42,12 @@ __device__ __forceinline__ uint32_t head_key(float f) {
 
 struct ArParams {
   CUtensorMap map_w;
-  const float *logits;        // [b * block][vocab]
+  CUtensorMap map_l;          // base logits [block * b][vocab] fp32, box = 128 columns x nb rows
+  const float *logits;        // [block][b][vocab]: the rows one step reads are contiguous
   const uint16_t *ar_e;       // [vocab][rank]
   const int32_t *bonus;       // [b]
   int32_t *next_tokens;       // [b][block]
-  unsigned long long *best;   // [block][kMaxBatch], zeroed before the launch
+  unsigned long long *best;   // [block][kMaxBatch][kBestStride], zeroed before the launch
   unsigned int *barrier;      // zeroed before the launch
   int32_t *status;
   int b, block, vocab, rank, n_tiles, nb, stages;
@@ -53,18 +57,21 @@ __global__ void __launch_bounds__(kThreads, 1) ar_head_kernel(const __grid_const
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int tile_bytes = 128 * P.rank * 2;
+  const int lg_bytes = P.nb * 128 * 4;                   // base logits of one tile: [nb rows][128 vocab entries] fp32
+  const int stage_bytes = tile_bytes + lg_bytes;
   const int slabs = P.rank / 64;
-  uint8_t *sW = smem;                                    // ring of W tiles: [stage][slab][128 rows][128 B]
-  uint8_t *sE = smem + P.stages * tile_bytes;            // Ey: [slab][nb rows][128 B]
+  uint8_t *sW = smem;                                    // ring of stages: W tile [slab][128 rows][128 B], then the logits block
+  uint8_t *sE = smem + P.stages * stage_bytes;           // Ey: [slab][nb rows][128 B]
   uint64_t *bars = reinterpret_cast<uint64_t *>(sE + slabs * P.nb * 128);
   uint64_t *full = bars, *empty = bars + 4, *acc_full = bars + 8, *acc_empty = bars + 10, *e_ready = bars + 12, *epi_bar = bars + 13;
   uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 14);
   volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
   int *s_tok = reinterpret_cast<int *>(tmem_slot + 2);   // [kMaxBatch] previous tokens of this step
+  unsigned long long *s_red = reinterpret_cast<unsigned long long *>(s_tok + kMaxBatch);  // [4 warps][kMaxBatch]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
-    for (int s = 0; s < 4; ++s) { mbar_init(full + s, 1); mbar_init(empty + s, 1); }
+    for (int s = 0; s < 4; ++s) { mbar_init(full + s, 1); mbar_init(empty + s, 5); }  // released by the MMA commit and the four epilogue warps
     for (int a = 0; a < 2; ++a) { mbar_init(acc_full + a, 1); mbar_init(acc_empty + a, 4); }
     mbar_init(e_ready, 4);
     mbar_init(epi_bar, 4);
@@ -91,8 +98,9 @@ __global__ void __launch_bounds__(kThreads, 1) ar_head_kernel(const __grid_const
           ok = mbar_wait(empty + stage, ph ^ 1u, abort_flag, 2);
           if (!ok) break;
           const int row0 = ((int)blockIdx.x + k * (int)gridDim.x) * 128;
-          mbar_arrive_expect_tx(full + stage, (uint32_t)tile_bytes);
-          for (int sb = 0; sb < slabs; ++sb) tma_load_2d(sW + stage * tile_bytes + sb * 16384, &P.map_w, full + stage, sb * 64, row0);
+          mbar_arrive_expect_tx(full + stage, (uint32_t)stage_bytes);
+          for (int sb = 0; sb < slabs; ++sb) tma_load_2d(sW + stage * stage_bytes + sb * 16384, &P.map_w, full + stage, sb * 64, row0);
+          tma_load_2d(sW + stage * stage_bytes + tile_bytes, &P.map_l, full + stage, row0, step * P.b);
           if (++stage == P.stages) { stage = 0; ph ^= 1u; }
         }
       }
@@ -113,7 +121,7 @@ __global__ void __launch_bounds__(kThreads, 1) ar_head_kernel(const __grid_const
           ok = mbar_wait(acc_empty + buf, ((kt >> 1) & 1) ^ 1u, abort_flag, 4) && mbar_wait(full + stage, ph, abort_flag, 5);
           if (!ok) break;
           tc_fence_after();
-          const uint64_t wd = wdesc0 + (uint64_t)((stage * tile_bytes) >> 4);
+          const uint64_t wd = wdesc0 + (uint64_t)((stage * stage_bytes) >> 4);
           for (int kk = 0; kk < P.rank / 16; ++kk) {
             const uint32_t woff = ((kk >> 2) * 16384 + (kk & 3) * 32) >> 4;
             const uint32_t eoff = ((kk >> 2) * (P.nb * 128) + (kk & 3) * 32) >> 4;
@@ -128,9 +136,9 @@ __global__ void __launch_bounds__(kThreads, 1) ar_head_kernel(const __grid_const
   } else {
     // ------------------------------------------------------------------ Ey build + epilogue: thread = vocab row of the tile
     const uint32_t taddr = tmem + ((uint32_t)(warp * 32) << 16);
-    int kt = 0;
+    int kt = 0, stage = 0;
     bool ok = true;
-    uint32_t ph_epi = 0;
+    uint32_t ph_epi = 0, ph_full = 0;
     // barrier of the four epilogue warps (bounded like every other wait; orders their shared-memory writes)
     auto epi_sync = [&]() {
       __syncwarp();
@@ -151,7 +159,7 @@ __global__ void __launch_bounds__(kThreads, 1) ar_head_kernel(const __grid_const
               tok = 0;
             }
           } else {
-            const unsigned long long w = __ldcg(P.best + (size_t)(step - 1) * kMaxBatch + threadIdx.x);
+            const unsigned long long w = __ldcg(P.best + ((size_t)(step - 1) * kMaxBatch + threadIdx.x) * kBestStride);
             tok = (int)(0xffffffffu - (uint32_t)(w & 0xffffffffull));
             if (w == 0ull) tok = 0;  // (all-NaN row)
             if (blockIdx.x == 0) P.next_tokens[(size_t)threadIdx.x * P.block + (step - 1)] = tok;
@@ -190,20 +198,30 @@ __global__ void __launch_bounds__(kThreads, 1) ar_head_kernel(const __grid_const
         __syncwarp();
         if (lane == 0) mbar_arrive(acc_empty + buf);
         const int v = ((int)blockIdx.x + k * (int)gridDim.x) * 128 + warp * 32 + lane;
-        if (v < P.vocab) {
-          const float *lrow = P.logits + (size_t)step * P.vocab + v;
+        {
+          // (acc_full implies the stage's loads have landed: the MMA issuer waited for them; this wait is the
+          //  epilogue threads' own acquire of the TMA-written logits and returns at once)
+          ok = __all_sync(0xffffffffu, mbar_wait(full + stage, ph_full, abort_flag, 9));
+          if (!ok) break;
+          const bool live = v < P.vocab;
+          const float *sl = reinterpret_cast<const float *>(sW + stage * stage_bytes + tile_bytes) + warp * 32 + lane;
+          const unsigned long long lowv = (unsigned long long)(0xffffffffu - (uint32_t)v);
 #pragma unroll
           for (int n = 0; n < kMaxBatch; ++n) {
             if (n < P.b) {
-              const float z = __uint_as_float(acc[n]) + __ldcs(lrow + (size_t)n * P.block * P.vocab);
-              const unsigned long long pk = ((unsigned long long)head_key(z) << 32) | (unsigned long long)(0xffffffffu - (uint32_t)v);
-              bestv[n] = pk > bestv[n] ? pk : bestv[n];
+              const float z = __uint_as_float(acc[n]) + sl[n * 128];
+              const unsigned long long pk = ((unsigned long long)head_key(z) << 32) | lowv;
+              bestv[n] = (live && pk > bestv[n]) ? pk : bestv[n];
             }
           }
+          __syncwarp();
+          if (lane == 0) mbar_arrive(empty + stage);
+          if (++stage == P.stages) { stage = 0; ph_full ^= 1u; }
         }
       }
       if (!ok) break;
-      // step maximum: warp reduction, then one atomic per request and warp
+      // step maximum: warp reduction, CTA reduction through shared memory, then ONE atomic per request and CTA,
+      // each request on its own 128-byte line (atomics on one line are serialised by a single L2 unit)
 #pragma unroll
       for (int n = 0; n < kMaxBatch; ++n) {
         if (n < P.b) {
@@ -213,8 +231,16 @@ __global__ void __launch_bounds__(kThreads, 1) ar_head_kernel(const __grid_const
             const unsigned long long y = __shfl_xor_sync(0xffffffffu, x, o);
             x = y > x ? y : x;
           }
-          if (lane == 0) atomicMax(P.best + (size_t)step * kMaxBatch + n, x);
+          if (lane == 0) s_red[warp * kMaxBatch + n] = x;
         }
+      }
+      ok = epi_sync();
+      if (!ok) break;
+      if ((int)threadIdx.x < P.b) {
+        unsigned long long x = s_red[threadIdx.x];
+#pragma unroll
+        for (int w = 1; w < 4; ++w) x = s_red[w * kMaxBatch + threadIdx.x] > x ? s_red[w * kMaxBatch + threadIdx.x] : x;
+        atomicMax(P.best + ((size_t)step * kMaxBatch + threadIdx.x) * kBestStride, x);
       }
       // ---- grid barrier: every CTA's maxima of this step are in before anyone reads them
       __threadfence();
@@ -233,7 +259,7 @@ __global__ void __launch_bounds__(kThreads, 1) ar_head_kernel(const __grid_const
     }
     // the last step's winners
     if (ok && blockIdx.x == 0 && (int)threadIdx.x < P.b) {
-      const unsigned long long w = __ldcg(P.best + (size_t)(P.block - 1) * kMaxBatch + threadIdx.x);
+      const unsigned long long w = __ldcg(P.best + ((size_t)(P.block - 1) * kMaxBatch + threadIdx.x) * kBestStride);
       P.next_tokens[(size_t)threadIdx.x * P.block + (P.block - 1)] = w == 0ull ? 0 : (int)(0xffffffffu - (uint32_t)(w & 0xffffffffull));
     }
   }
@@ -254,7 +280,7 @@ __global__ void __launch_bounds__(kThreads, 1) ar_head_kernel(const __grid_const
 size_t head_workspace_bytes(int b, int block, int vocab) {
   if (b <= 0 || block <= 0 || vocab <= 0) return 0;
   const size_t logits = (((size_t)b * block * vocab * sizeof(float)) + 255) & ~size_t(255);
-  return logits + (size_t)block * kMaxBatch * sizeof(unsigned long long) + 256;
+  return logits + (size_t)block * kMaxBatch * kBestStride * sizeof(unsigned long long) + 256;
 }
 
 dpara_status launch_head(const HeadArgs &h, void *workspace, int32_t *status, cudaStream_t st) {
@@ -266,27 +292,31 @@ dpara_status launch_head(const HeadArgs &h, void *workspace, int32_t *status, cu
   float *logits = reinterpret_cast<float *>(ws);
   const size_t logits_bytes = (((size_t)h.b * h.block * h.vocab * sizeof(float)) + 255) & ~size_t(255);
   unsigned long long *best = reinterpret_cast<unsigned long long *>(ws + logits_bytes);
-  unsigned int *barrier = reinterpret_cast<unsigned int *>(best + (size_t)h.block * kMaxBatch);
-  if (cudaMemsetAsync(best, 0, (size_t)h.block * kMaxBatch * sizeof(unsigned long long) + 256, st) != cudaSuccess) return DPARA_ERR_CUDA;
+  unsigned int *barrier = reinterpret_cast<unsigned int *>(best + (size_t)h.block * kMaxBatch * kBestStride);
+  if (cudaMemsetAsync(best, 0, (size_t)h.block * kMaxBatch * kBestStride * sizeof(unsigned long long) + 256, st) != cudaSuccess) return DPARA_ERR_CUDA;
 
-  // base logits of the selected branches: [b * block][vocab] fp32
+  // base logits of the selected branches, fp32, stored step-major [block][b][vocab] (GEMM row n * block + i goes
+  // to row i * b + n): the b rows a step reads then lie in one contiguous range instead of b ranges
+  // block * vocab * 4 bytes apart
   GemmArgs g;
   g.a = h.sel_reps; g.w = h.w_lm; g.M = h.b * h.block; g.N = h.vocab; g.K = h.hidden; g.epi = 3;
-  g.resid = nullptr; g.resid_bf16 = 0; g.out = logits; g.out_bf16 = nullptr;
+  g.resid = nullptr; g.resid_bf16 = 0; g.out = logits; g.out_bf16 = nullptr; g.perm_block = h.block; g.perm_b = h.b;
   dpara_status rc = launch_gemm_tc(g, status, st);
   if (rc != DPARA_OK) return rc;
 
   ArParams P;
   memset(&P, 0, sizeof(P));
   if (!make_tmap_bf16_2d(&P.map_w, h.ar_w, h.rank, h.vocab, (uint64_t)h.rank * 2, 64, 128)) return DPARA_ERR_CUDA;
+  if (!make_tmap_f32_2d(&P.map_l, logits, h.vocab, (uint64_t)h.block * h.b, (uint64_t)h.vocab * 4, 128, h.b <= 16 ? 16 : 32)) return DPARA_ERR_CUDA;
   P.logits = logits; P.ar_e = static_cast<const uint16_t *>(h.ar_e); P.bonus = h.bonus; P.next_tokens = h.next_tokens;
   P.best = best; P.barrier = barrier; P.status = status;
   P.b = h.b; P.block = h.block; P.vocab = h.vocab; P.rank = h.rank;
   P.n_tiles = (h.vocab + 127) / 128;
   P.nb = h.b <= 16 ? 16 : 32;
-  const int tile_bytes = 128 * h.rank * 2;
-  P.stages = (200 * 1024) / tile_bytes > 4 ? 4 : (200 * 1024) / tile_bytes;
-  const int smem = P.stages * tile_bytes + (h.rank / 64) * P.nb * 128 + 1024 + 512;
+  const int stage_bytes = 128 * h.rank * 2 + P.nb * 128 * 4;
+  const int fixed = (h.rank / 64) * P.nb * 128 + 1024 + 2048;   // Ey, alignment slack, barriers and reduction scratch
+  P.stages = (227 * 1024 - fixed) / stage_bytes > 4 ? 4 : (227 * 1024 - fixed) / stage_bytes;
+  const int smem = P.stages * stage_bytes + fixed;
   if (cudaFuncSetAttribute(ar_head_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return DPARA_ERR_CUDA;
   int dev = 0, sms = kNumSM;
   if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);

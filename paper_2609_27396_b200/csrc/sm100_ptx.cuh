@@ -255,5 +255,8 @@ bool make_tmap_bf16_3d(CUtensorMap *m, const void *base, uint64_t d0, uint64_t d
 // bf16 matrix [rows][cols] (cols contiguous), row stride in bytes; box (64 cols, box_rows); 128-byte swizzle.
 bool make_tmap_bf16_2d(CUtensorMap *m, const void *base, uint64_t cols, uint64_t rows, uint64_t row_stride, uint32_t box_cols,
                        uint32_t box_rows);
+// fp32, 2-D, no swizzle (rows of the box land back to back in shared memory)
+bool make_tmap_f32_2d(CUtensorMap *m, const void *base, uint64_t cols, uint64_t rows, uint64_t row_stride, uint32_t box_cols,
+                      uint32_t box_rows);
 
 }  // namespace dpara

@@ -47,4 +47,18 @@ bool make_tmap_bf16_2d(CUtensorMap *m, const void *base, uint64_t cols, uint64_t
   return r == CUDA_SUCCESS;
 }
 
+bool make_tmap_f32_2d(CUtensorMap *m, const void *base, uint64_t cols, uint64_t rows, uint64_t row_stride, uint32_t box_cols,
+                      uint32_t box_rows) {
+  EncodeTiledFn enc = get_encode_tiled();
+  if (!enc) return false;
+  cuuint64_t dims[2] = {cols, rows ? rows : 1};
+  cuuint64_t strides[1] = {row_stride};
+  cuuint32_t box[2] = {box_cols, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void *>(base), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
 }  // namespace dpara

@@ -107,3 +107,23 @@ def test_head_rejects_bad_arguments():
     plan.run(t[0], t[1], t[2], t[3], bad)
     torch.cuda.synchronize()
     assert plan.status.item() & 1
+
+
+def test_head_full_size_sampled():
+    """The benchmark shape (b = 16, d = 16, hidden 5120, vocab 151 936, rank 256) in the launch configuration the
+    bench times; the oracle checks sampled (request, step) pairs one by one, teacher-forced with the kernel's
+    own previous token, and the base logits of those rows element by element."""
+    sh = W.head_shape(W.workload(3))
+    inp = W.make_head_inputs(sh, W.workload(3).seed)
+    toks, logits = _run(inp)
+    assert ((toks >= 0) & (toks < sh.vocab)).all()
+    rng = np.random.default_rng(7)
+    for n, i in [(0, 0), (15, 15)] + [(int(rng.integers(sh.batch)), int(rng.integers(1, sh.block))) for _ in range(2)]:
+        row = np.concatenate([H.lm_head(inp.sel_reps[n, i][None], inp.w_lm, cols=range(c, min(c + 16384, sh.vocab)))[0]
+                              for c in range(0, sh.vocab, 16384)])
+        scale = max(1.0, float(np.abs(row).max()))
+        assert np.abs(logits[n * sh.block + i] - row).max() <= TIE * scale
+        y_prev = int(inp.bonus[n]) if i == 0 else int(toks[n, i - 1])
+        z = H.ar_logits(row, inp.ar_w, inp.ar_e, y_prev)
+        want, got = int(np.argmax(z)), int(toks[n, i])
+        assert got == want or z[got] >= z[want] - TIE * max(1.0, float(np.abs(z).max())), (n, i, got, want)
