@@ -5,16 +5,18 @@
 // The loop is d dependent steps, each a skinny product: all vocab rows of W (vocab x rank, bf16) against the b
 // embedding rows E(y_{i-1}) -- 0.6 GFLOP and one pass over W (78 MB at vocab 151 936, rank 256, which stays in
 // L2) per step.  ONE persistent cooperative kernel runs all d steps:
-//   warp 4      TMA producer: streams this CTA's 128-row tiles of W through a ring of shared-memory stages (the
+//   warp 8      TMA producer: streams this CTA's 128-row tiles of W through a ring of shared-memory stages (the
 //               tiles do not depend on the tokens, so the ring runs ahead across steps), and with each tile the
 //               b x 128 block of base logits it will be added to (plain loads of those from the epilogue queued
 //               behind the deep W stream and cost 1.6 us each; as part of the stage they cost nothing);
-//   warp 5      one thread issues tcgen05.mma: D[128 vocab rows][nb] = W_tile[128][rank] * Ey[nb][rank]^T
+//   warp 9      one thread issues tcgen05.mma: D[128 vocab rows][nb] = W_tile[128][rank] * Ey[nb][rank]^T
 //               (M = 128, N = nb = 16 or 32, both operands K-major in shared memory, 128-byte swizzle);
-//   warps 0-3   build Ey in shared memory at the start of a step (gather of E rows, swizzled by hand), then for
-//               every tile: tcgen05.ld the accumulator (thread = vocab row), add the base logit of each
-//               request (from the stage), keep the running (value, index) maximum per request;
-//               at the end of the step a warp reduction and one 64-bit atomicMax per request and warp.
+//   warps 0-7   build Ey in shared memory at the start of a step (gather of E rows, swizzled by hand), then for
+//               every tile: tcgen05.ld the accumulator (thread = vocab row; warps w and w + 4 share the 32 rows
+//               of a TMEM lane quarter and take the even / odd requests), add the base logit of each request
+//               (from the stage), keep the running (value, index) maximum per request -- a thread meets its
+//               rows in increasing order, so a strict compare keeps the lowest index; at the end of the step a
+//               warp reduction, a CTA reduction and one 64-bit atomicMax per request and CTA.
 // Between steps the CTAs meet at a grid barrier (a counter in global memory; the launch is cooperative, so all
 // CTAs are resident; the wait is bounded by wall time and gives up with DPARA_STATUS_TIMEOUT).
 // A maximum is carried as (order-preserving key of z) << 32 | ~index: the largest packed value is the largest
@@ -27,7 +29,8 @@ namespace dpara {
 using namespace ptx;
 
 namespace {
-constexpr int kThreads = 192;
+constexpr int kThreads = 320;  // warps 0-7 epilogue, 8 TMA producer, 9 MMA issuer
+constexpr int kEpiWarps = 8, kProducerWarp = 8, kMmaWarp = 9;
 constexpr int kMaxBatch = 32;
 constexpr int kAccCols = 32;  // TMEM columns per accumulator buffer (nb <= 32)
 constexpr int kBestStride = 16;  // 64-bit words between two requests' maxima: one 128-byte line (one L2 atomic unit) each
@@ -71,14 +74,14 @@ __global__ void __launch_bounds__(kThreads, 1) ar_head_kernel(const __grid_const
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
-    for (int s = 0; s < 4; ++s) { mbar_init(full + s, 1); mbar_init(empty + s, 5); }  // released by the MMA commit and the four epilogue warps
-    for (int a = 0; a < 2; ++a) { mbar_init(acc_full + a, 1); mbar_init(acc_empty + a, 4); }
-    mbar_init(e_ready, 4);
-    mbar_init(epi_bar, 4);
+    for (int s = 0; s < 4; ++s) { mbar_init(full + s, 1); mbar_init(empty + s, 1 + kEpiWarps); }  // released by the MMA commit and the epilogue warps
+    for (int a = 0; a < 2; ++a) { mbar_init(acc_full + a, 1); mbar_init(acc_empty + a, kEpiWarps); }
+    mbar_init(e_ready, kEpiWarps);
+    mbar_init(epi_bar, kEpiWarps);
     *abort_flag = 0;
     fence_barrier_init();
   }
-  if (warp == 5) { tmem_alloc(tmem_slot, 64); tmem_relinquish(); }
+  if (warp == kMmaWarp) { tmem_alloc(tmem_slot, 64); tmem_relinquish(); }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -86,7 +89,7 @@ __global__ void __launch_bounds__(kThreads, 1) ar_head_kernel(const __grid_const
   // this CTA's tiles: blockIdx.x, blockIdx.x + gridDim.x, ... (the same in every step)
   const int my_tiles = (P.n_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
 
-  if (warp == 4) {
+  if (warp == kProducerWarp) {
     // ------------------------------------------------------------------ producer
     if (lane == 0) {
       prefetch_tensormap(&P.map_w);
@@ -105,7 +108,7 @@ __global__ void __launch_bounds__(kThreads, 1) ar_head_kernel(const __grid_const
         }
       }
     }
-  } else if (warp == 5) {
+  } else if (warp == kMmaWarp) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       const uint32_t idesc = idesc_bf16_f32(128, P.nb, false, false);
@@ -135,11 +138,12 @@ __global__ void __launch_bounds__(kThreads, 1) ar_head_kernel(const __grid_const
     }
   } else {
     // ------------------------------------------------------------------ Ey build + epilogue: thread = vocab row of the tile
-    const uint32_t taddr = tmem + ((uint32_t)(warp * 32) << 16);
+    const int quarter = warp & 3, nh = warp >> 2;  // TMEM lane quarter; this warp takes requests n = 2 j + nh
+    const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16);
     int kt = 0, stage = 0;
     bool ok = true;
     uint32_t ph_epi = 0, ph_full = 0;
-    // barrier of the four epilogue warps (bounded like every other wait; orders their shared-memory writes)
+    // barrier of the epilogue warps (bounded like every other wait; orders their shared-memory writes)
     auto epi_sync = [&]() {
       __syncwarp();
       if (lane == 0) mbar_arrive(epi_bar);
@@ -172,7 +176,7 @@ __global__ void __launch_bounds__(kThreads, 1) ar_head_kernel(const __grid_const
       // Ey[n][k] = E[tok_n][k] in the K-major 128-byte-swizzle layout the MMA reads: slab = k / 64, row n at
       // 128 B pitch, 16-byte chunk c of the row stored at chunk position c ^ (n & 7); rows n >= b are zero
       const int chunks_per_row = P.rank / 8;
-      for (int q = threadIdx.x; q < P.nb * chunks_per_row; q += 128) {
+      for (int q = threadIdx.x; q < P.nb * chunks_per_row; q += kEpiWarps * 32) {
         const int n = q / chunks_per_row, c = q % chunks_per_row;
         uint4 v = make_uint4(0, 0, 0, 0);
         if (n < P.b) v = *reinterpret_cast<const uint4 *>(P.ar_e + (size_t)s_tok[n] * P.rank + c * 8);
@@ -183,9 +187,10 @@ __global__ void __launch_bounds__(kThreads, 1) ar_head_kernel(const __grid_const
       __syncwarp();
       if (lane == 0) mbar_arrive(e_ready);
 
-      unsigned long long bestv[kMaxBatch];
+      float bz[kMaxBatch / 2];
+      int bv[kMaxBatch / 2];
 #pragma unroll
-      for (int n = 0; n < kMaxBatch; ++n) bestv[n] = 0ull;
+      for (int j = 0; j < kMaxBatch / 2; ++j) { bz[j] = -INFINITY; bv[j] = -1; }
       for (int k = 0; k < my_tiles; ++k, ++kt) {
         const int buf = kt & 1;
         ok = __all_sync(0xffffffffu, mbar_wait(acc_full + buf, (kt >> 1) & 1, abort_flag, 6));
@@ -197,41 +202,40 @@ __global__ void __launch_bounds__(kThreads, 1) ar_head_kernel(const __grid_const
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(acc_empty + buf);
-        const int v = ((int)blockIdx.x + k * (int)gridDim.x) * 128 + warp * 32 + lane;
-        {
-          // (acc_full implies the stage's loads have landed: the MMA issuer waited for them; this wait is the
-          //  epilogue threads' own acquire of the TMA-written logits and returns at once)
-          ok = __all_sync(0xffffffffu, mbar_wait(full + stage, ph_full, abort_flag, 9));
-          if (!ok) break;
-          const bool live = v < P.vocab;
-          const float *sl = reinterpret_cast<const float *>(sW + stage * stage_bytes + tile_bytes) + warp * 32 + lane;
-          const unsigned long long lowv = (unsigned long long)(0xffffffffu - (uint32_t)v);
+        const int v = ((int)blockIdx.x + k * (int)gridDim.x) * 128 + quarter * 32 + lane;
+        // (acc_full implies the stage's loads have landed: the MMA issuer waited for them; this wait is the
+        //  epilogue threads' own acquire of the TMA-written logits and returns at once)
+        ok = __all_sync(0xffffffffu, mbar_wait(full + stage, ph_full, abort_flag, 9));
+        if (!ok) break;
+        const bool live = v < P.vocab;
+        const float *sl = reinterpret_cast<const float *>(sW + stage * stage_bytes + tile_bytes) + quarter * 32 + lane;
 #pragma unroll
-          for (int n = 0; n < kMaxBatch; ++n) {
-            if (n < P.b) {
-              const float z = __uint_as_float(acc[n]) + sl[n * 128];
-              const unsigned long long pk = ((unsigned long long)head_key(z) << 32) | lowv;
-              bestv[n] = (live && pk > bestv[n]) ? pk : bestv[n];
-            }
+        for (int j = 0; j < kMaxBatch / 2; ++j) {
+          const int n = 2 * j + nh;
+          if (n < P.b) {
+            const float z = __uint_as_float(nh ? acc[2 * j + 1] : acc[2 * j]) + sl[n * 128];
+            // larger, or the first number this thread sees (NaN never wins; -inf can, at the lowest index)
+            if (live && (z > bz[j] || (bv[j] < 0 && z == z))) { bz[j] = z; bv[j] = v; }
           }
-          __syncwarp();
-          if (lane == 0) mbar_arrive(empty + stage);
-          if (++stage == P.stages) { stage = 0; ph_full ^= 1u; }
         }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(empty + stage);
+        if (++stage == P.stages) { stage = 0; ph_full ^= 1u; }
       }
       if (!ok) break;
       // step maximum: warp reduction, CTA reduction through shared memory, then ONE atomic per request and CTA,
       // each request on its own 128-byte line (atomics on one line are serialised by a single L2 unit)
 #pragma unroll
-      for (int n = 0; n < kMaxBatch; ++n) {
+      for (int j = 0; j < kMaxBatch / 2; ++j) {
+        const int n = 2 * j + nh;
         if (n < P.b) {
-          unsigned long long x = bestv[n];
+          unsigned long long x = bv[j] < 0 ? 0ull : (((unsigned long long)head_key(bz[j]) << 32) | (unsigned long long)(0xffffffffu - (uint32_t)bv[j]));
 #pragma unroll
           for (int o = 16; o > 0; o >>= 1) {
             const unsigned long long y = __shfl_xor_sync(0xffffffffu, x, o);
             x = y > x ? y : x;
           }
-          if (lane == 0) s_red[warp * kMaxBatch + n] = x;
+          if (lane == 0) s_red[quarter * kMaxBatch + n] = x;
         }
       }
       ok = epi_sync();
@@ -274,7 +278,7 @@ __global__ void __launch_bounds__(kThreads, 1) ar_head_kernel(const __grid_const
     }
     __syncthreads();
   }
-  if (warp == 5) tmem_dealloc(tmem, 64);
+  if (warp == kMmaWarp) tmem_dealloc(tmem, 64);
 }
 
 size_t head_workspace_bytes(int b, int block, int vocab) {
