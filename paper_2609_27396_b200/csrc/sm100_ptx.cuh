@@ -219,6 +219,60 @@ __device__ __forceinline__ float2 ld_dsmem_f2(uint32_t addr) {
   return v;
 }
 
+// ---------------------------------------------------------------------------------------------- CTA pairs (cta_group::2)
+// A pair of CTAs (cluster ranks 2k, 2k+1) shares one MMA: M = 256 rows, the even CTA ("leader") issues.
+// Each CTA holds its own 128 rows of A and D and HALF of the B operand at the same shared-memory offsets.
+constexpr uint32_t kPeerBitMask = 0xFEFFFFFFu;  // clears the CTA-rank bit of a shared::cluster address -> the leader's copy
+__device__ __forceinline__ uint32_t leader_addr(const void *local_smem_ptr) { return smem_u32(local_smem_ptr) & kPeerBitMask; }
+
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t *dst_smem, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_pair() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+// TMA load issued by either CTA of the pair into ITS OWN shared memory; the transaction bytes are counted on
+// the LEADER's mbarrier (no multicast: each CTA fetches only its own operand half).
+__device__ __forceinline__ void tma_load_2d_pair(void *dst, const CUtensorMap *m, uint64_t *bar_local, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(m)), "r"(leader_addr(bar_local)), "r"(c0), "r"(c1)
+      : "memory");
+}
+// Arrive (count 1) on the leader CTA's copy of a barrier, from either CTA.
+__device__ __forceinline__ void mbar_arrive_leader(uint64_t *bar_local) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(leader_addr(bar_local)) : "memory");
+}
+__device__ __forceinline__ void mma2_ss(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, bool accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"((uint32_t)accumulate)
+      : "memory");
+}
+template <bool kAcc>
+__device__ __forceinline__ void mma2_ss_c(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "n"(kAcc ? 1 : 0)
+      : "memory");
+}
+// Arrives on the barrier at this offset in BOTH CTAs of the pair once every tcgen05 operation the thread has
+// issued so far has completed (commit with multicast; not a multicast LOAD).
+__device__ __forceinline__ void mma2_commit_both(uint64_t *bar_local) {
+  const uint16_t mask = 3;
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(smem_u32(bar_local)), "h"(mask) : "memory");
+}
+// Arrives only on the leader's barrier.
+__device__ __forceinline__ void mma2_commit_leader(uint64_t *bar_local) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar_local)) : "memory");
+}
+
 // ---------------------------------------------------------------------------------------------- packed fp32x2 math
 __device__ __forceinline__ uint64_t pack2(float lo, float hi) {
   uint64_t r;
