@@ -248,8 +248,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
 // 128 output rows; the even CTA's thread issues M = 256 products that read both halves.  Per pair and K slab
 // 64 KB enter shared memory instead of the 96 KB two independent 128 x 256 tiles need: these shapes
 // (M = 256..1024 rows against large weights) are bound by the L2 -> shared-memory fill rate, not by the tensor
-// pipe.  Each CTA's producer fetches its own halves (no multicast) and counts the bytes on the LEADER's
-// barrier; stage and accumulator hand-offs from the MMA thread reach both CTAs through a multicast commit;
+// pipe.  Each CTA's producer fetches its own halves with ordinary tiled copies and counts the bytes on the LEADER's
+// barrier; stage and accumulator hand-offs from the MMA thread reach both CTAs through one tcgen05.commit;
 // the epilogue warps of both CTAs arrive on the leader's accumulator-empty barrier.
 namespace {
 constexpr int kStages2 = 6;

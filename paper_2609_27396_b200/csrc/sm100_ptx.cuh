@@ -235,7 +235,7 @@ __device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols
   asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
 }
 // TMA load issued by either CTA of the pair into ITS OWN shared memory; the transaction bytes are counted on
-// the LEADER's mbarrier (no multicast: each CTA fetches only its own operand half).
+// the LEADER's mbarrier (an ordinary tiled copy: each CTA fetches only its own operand half).
 __device__ __forceinline__ void tma_load_2d_pair(void *dst, const CUtensorMap *m, uint64_t *bar_local, int c0, int c1) {
   asm volatile(
       "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
@@ -262,7 +262,7 @@ __device__ __forceinline__ void mma2_ss_c(uint32_t d_tmem, uint64_t adesc, uint6
       : "memory");
 }
 // Arrives on the barrier at this offset in BOTH CTAs of the pair once every tcgen05 operation the thread has
-// issued so far has completed (commit with multicast; not a multicast LOAD).
+// issued so far has completed (a tcgen05.commit that signals both CTAs; no data moves).
 __device__ __forceinline__ void mma2_commit_both(uint64_t *bar_local) {
   const uint16_t mask = 3;
   asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
