@@ -54,13 +54,19 @@ struct TcParams {
   CUtensorMap map_q, map_kc, map_vc, map_ks, map_vs, map_kb, map_vb;
   AttnParams a;
   int JI_T, n_ji, n_tiles, n_pairs, nsplit, S8, R_blk, has_blk, has_tail, n_items;
-  float *part_o;   // split-KV partials [item slot][2][128][D] fp32 (unnormalised rows)
+  float *part_o;   // split-KV partials [item slot][2][D / 4][128 rows] float4 (unnormalised rows; a warp's lanes are
+                   // consecutive rows, so its stores and the merge's loads are contiguous 512-byte runs)
   float2 *part_ml; // [item slot][2][128] (row max in raw-score units, row sum)
   float c_log2;    // softmax scale * log2(e)
   // requests in order of decreasing context length: the block scheduler hands out CTAs in grid order, so
   // launching the long requests first leaves the short ones to fill the tail of a ragged batch
   uint8_t req_order[kMaxOrdered];
   int use_order;
+  // context offsets and lengths of small batches travel in the parameters (saves every CTA two dependent global
+  // loads, ~1 us, before it can start)
+  int use_ctx_p;
+  int ctx_len_p[kMaxOrdered];
+  long long ctx_off_p[kMaxOrdered];
   // Work schedule of the persistent CTAs (no KV split, more items than CTAs): CTA c runs items
   // sched[cta_first[c]] .. sched[cta_first[c + 1] - 1].  The host balances the CTAs' loads (longest processing
   // time first, each item to the least loaded CTA); a ragged batch has few items per CTA (about five at the
@@ -99,8 +105,13 @@ __device__ __forceinline__ Item decode_item(const TcParams &P, int id) {
   I.pair = x / P.nsplit;
   I.split = x % P.nsplit;
   I.ntq = min(2, P.n_tiles - I.pair * 2);
-  I.c0 = A.ctx_offsets[I.n];
-  I.L = (int)(A.ctx_offsets[I.n + 1] - I.c0);
+  if (P.use_ctx_p) {
+    I.c0 = P.ctx_off_p[I.n];
+    I.L = P.ctx_len_p[I.n];
+  } else {
+    I.c0 = A.ctx_offsets[I.n];
+    I.L = (int)(A.ctx_offsets[I.n + 1] - I.c0);
+  }
   I.nctx = (I.L + 127) >> 7;
   I.t0 = (int)((long long)I.split * I.nctx / P.nsplit);
   I.t1 = (int)((long long)(I.split + 1) * I.nctx / P.nsplit);
@@ -475,10 +486,10 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
         tmem_ld32(lane_addr + Cfg::kColO + t * 128 + cc * 32, o);
         tmem_wait_ld();
         if (P.nsplit > 1) {
-          float4 *dst = reinterpret_cast<float4 *>(P.part_o + pslot * D + cc * 32);
+          float4 *dst = reinterpret_cast<float4 *>(P.part_o) + (((size_t)I.slot * 2 + t) * (D / 4) + cc * 8) * 128 + r;
 #pragma unroll
           for (int v = 0; v < 8; ++v)
-            __stcg(dst + v, make_float4(__uint_as_float(o[4 * v]), __uint_as_float(o[4 * v + 1]), __uint_as_float(o[4 * v + 2]),
+            __stcg(dst + v * 128, make_float4(__uint_as_float(o[4 * v]), __uint_as_float(o[4 * v + 1]), __uint_as_float(o[4 * v + 2]),
                                         __uint_as_float(o[4 * v + 3])));
         } else if (valid) {
           if (A.out_f32) {
@@ -527,10 +538,11 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
       const int rows_per = 256 / P.nsplit;
       const float c = P.c_log2;
       const size_t slot0 = (size_t)(I.slot - I.split);  // scratch slot of split 0 of this item
-      // unit of work: 16 output elements of one row; all loads of a step are issued before their first use
+      // unit of work: 16 output elements of one row; a warp's lanes take consecutive rows (contiguous loads);
+      // the loads of four splits are issued before their first use
       constexpr int kParts = D / 16;
       for (int u = threadIdx.x; u < rows_per * kParts; u += 256) {
-        const int R = (int)rank * rows_per + u / kParts, part = u % kParts;
+        const int R = (int)rank * rows_per + u % rows_per, part = u / rows_per;
         const int t = R >> 7, r = R & 127;
         const int ji = (I.pair * 2 + t) * P.JI_T + r / A.G;
         if (t >= I.ntq || r >= P.JI_T * A.G || ji >= P.n_ji) continue;
@@ -540,26 +552,32 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
 #pragma unroll
         for (int sp = 0; sp < 8; ++sp)
           ml[sp] = sp < P.nsplit ? __ldcg(P.part_ml + ((slot0 + sp) * 2 + t) * 128 + r) : make_float2(-INFINITY, 0.f);
-        float mmax = -INFINITY;
-#pragma unroll
-        for (int sp = 0; sp < 8; ++sp) if (ml[sp].y > 0.f) mmax = fmaxf(mmax, ml[sp].x);
         float acc[16], lsum = 0.f;
 #pragma unroll
         for (int e = 0; e < 16; ++e) acc[e] = 0.f;
+        float mmax = -INFINITY;
+        bool have_max = false;
 #pragma unroll
-        for (int sp0 = 0; sp0 < 8; sp0 += 2) {
+        for (int sp0 = 0; sp0 < 8; sp0 += 4) {
           if (sp0 >= P.nsplit) break;
-          float4 x[2][4];
+          float4 x[4][4];
 #pragma unroll
-          for (int q = 0; q < 2; ++q) {
-            const float4 *src = reinterpret_cast<const float4 *>(P.part_o + (((slot0 + sp0 + q) * 2 + t) * 128 + r) * D + part * 16);
+          for (int q = 0; q < 4; ++q) {
+            if (sp0 + q < P.nsplit) {
+              const float4 *src = reinterpret_cast<const float4 *>(P.part_o) + (((slot0 + sp0 + q) * 2 + t) * (D / 4) + part * 4) * 128 + r;
 #pragma unroll
-            for (int v = 0; v < 4; ++v) x[q][v] = __ldcg(src + v);
+              for (int v = 0; v < 4; ++v) x[q][v] = __ldcg(src + v * 128);
+            }
+          }
+          if (!have_max) {
+#pragma unroll
+            for (int sp = 0; sp < 8; ++sp) if (ml[sp].y > 0.f) mmax = fmaxf(mmax, ml[sp].x);
+            have_max = true;
           }
 #pragma unroll
-          for (int q = 0; q < 2; ++q) {
+          for (int q = 0; q < 4; ++q) {
             // a peer without visible keys wrote no rows (its slot may hold anything): weight 0 skips it
-            const float wgt = ml[sp0 + q].y > 0.f ? ex2((ml[sp0 + q].x - mmax) * c) : 0.f;
+            const float wgt = (sp0 + q < P.nsplit && ml[sp0 + q].y > 0.f) ? ex2((ml[sp0 + q].x - mmax) * c) : 0.f;
             lsum = fmaf(wgt, ml[sp0 + q].y, lsum);
             if (wgt > 0.f) {
 #pragma unroll
@@ -697,6 +715,9 @@ dpara_status launch_attention_tc(const AttnParams &A, const TcPlan &plan, const 
     ok = ok && make_tmap_bf16_3d(&P.map_vb, A.v_blk, D, A.Hkv, nq, rs, rs * A.Hkv, 64, 1, plan.R_blk);
   }
   if (!ok) return DPARA_ERR_CUDA;
+  P.use_ctx_p = A.b <= kMaxOrdered;
+  if (P.use_ctx_p)
+    for (int n = 0; n < A.b; ++n) { P.ctx_off_p[n] = host_off[n]; P.ctx_len_p[n] = (int)(host_off[n + 1] - host_off[n]); }
   P.use_order = A.b <= kMaxOrdered && A.b > 1;
   if (P.use_order) {
     int idx[kMaxOrdered];
