@@ -142,6 +142,9 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
   volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+#ifdef DPARA_TRACE  // kernel phases of CTA 0: g_trace[29][0..4] clocks, [8..9] wall time
+  if (threadIdx.x == 0 && blockIdx.x == 0) { g_trace[29 * 64 + 0] = clock64(); g_trace[29 * 64 + 8] = (long long)global_timer_ns(); }
+#endif
   // this CTA's items: its slice of the host-built schedule, else items blockIdx.x, blockIdx.x + gridDim.x, ...
   const int q_begin = P.use_sched ? (int)P.cta_first[blockIdx.x] : (int)blockIdx.x;
   const int q_end = P.use_sched ? (int)P.cta_first[blockIdx.x + 1] : P.n_items;
@@ -167,6 +170,9 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
+#ifdef DPARA_TRACE
+  if (threadIdx.x == 0 && blockIdx.x == 0) g_trace[29 * 64 + 1] = clock64();
+#endif
 
   // register budget: the softmax warpgroups need the registers (a 128-wide score row per thread), the
   // producer / MMA warpgroup almost none
@@ -532,6 +538,9 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
     __threadfence();
     __syncwarp();
     cluster_sync_all();
+#ifdef DPARA_TRACE
+    if (threadIdx.x == 0 && blockIdx.x == 0) g_trace[29 * 64 + 2] = clock64();
+#endif
     if (warp < 8 && !*abort_flag) {
       const Item I = decode_item(P, blockIdx.x);
       const uint32_t rank = cluster_ctarank();
@@ -607,6 +616,9 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
     }
   }
 
+#ifdef DPARA_TRACE
+  if (threadIdx.x == 0 && blockIdx.x == 0) g_trace[29 * 64 + 3] = clock64();
+#endif
   // ------------------------------------------------------------------ teardown
   __syncwarp();
   tc_fence_before();
@@ -621,6 +633,9 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
     __syncthreads();
   }
   if (warp == 9) tmem_dealloc(tmem, 512);
+#ifdef DPARA_TRACE
+  if (threadIdx.x == 0 && blockIdx.x == 0) { g_trace[29 * 64 + 4] = clock64(); g_trace[29 * 64 + 9] = (long long)global_timer_ns(); }
+#endif
 }
 
 // ------------------------------------------------------------------------------------------------ host
