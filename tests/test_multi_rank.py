@@ -10,6 +10,7 @@ import torch.distributed as dist
 import torch.multiprocessing as mp
 
 import workloads as W
+from oracle import head as OH
 from oracle import verify as OV
 from paper_2609_27396_b200 import dist_util as DU
 
@@ -37,7 +38,10 @@ def _worker(rank, world, port, q):
     res = OV.verify_greedy(v.target[mine], v.draft_tokens[mine], v.reps[mine])
     a, b = DU.gather_results(res["accept_len"].tolist(), res["bonus"].tolist())
     t = DU.max_over_ranks(1.0 + rank)
-    q.put((rank, mine, a, b, t))
+    # the head loop shards the same way: each request's chain depends on its own rows and bonus only
+    hin = W.make_head_inputs(W.HeadShape(6, 3, 16, 64, 8), 13)
+    toks = OH.draft_head_greedy(hin.sel_reps[mine], hin.w_lm, hin.ar_w, hin.ar_e, hin.bonus[mine])
+    q.put((rank, mine, a, b, t, toks.tolist()))
     dist.destroy_process_group()
 
 
@@ -55,8 +59,11 @@ def test_two_gloo_ranks_shard_and_reduce():
     sh = W.VerifyShape(6, 5, 300, 2, 8, "greedy", 0.7, 1.0)
     v = W.make_verify_inputs(sh, 11)
     full = OV.verify_greedy(v.target, v.draft_tokens, v.reps)
-    for rank, mine, a, b, t in got:
+    hin = W.make_head_inputs(W.HeadShape(6, 3, 16, 64, 8), 13)
+    htoks = OH.draft_head_greedy(hin.sel_reps, hin.w_lm, hin.ar_w, hin.ar_e, hin.bonus)
+    for rank, mine, a, b, t, toks in got:
         assert t == 2.0                                    # max over ranks of (1 + rank)
+        assert toks == htoks[mine].tolist()                # a shard's head tokens = the same rows of the whole batch
         parts = DU.shard_requests([40, 10, 30, 20, 50, 60], world)
         for r in range(world):                             # every rank sees every shard's outcome
             assert a[r] == full["accept_len"][parts[r]].tolist() and b[r] == full["bonus"][parts[r]].tolist()
