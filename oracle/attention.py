@@ -110,6 +110,29 @@ def draft_rows(q, k_ctx, v_ctx, ctx_offsets, k_spine, v_spine, k_blk, v_blk,
     return np.stack(res) if res else np.zeros((0, D))
 
 
+def spine_rows(q_spine, k_ctx, v_ctx, ctx_offsets, k_spine, v_spine, scale: Optional[float] = None):
+    """The spine tokens as query rows (Sec. 3.2, Fig. 4: the anchors run causally among themselves and see the
+    whole cached context): anchor a of request n attends the context and spine rows 0..a, itself included.
+    q_spine [b][S][Hq][D], k_spine / v_spine [b][S][Hkv][D] (bf16 bit patterns).  Returns float64 [b][S][Hq][D].
+    Not part of the call that is built so far (there the spine's K/V are inputs); kept here, pinned, for the
+    backbone pass that produces them itself."""
+    b, S, Hq, D = q_spine.shape
+    G = Hq // k_spine.shape[2]
+    if scale is None or scale == 0:
+        scale = 1.0 / math.sqrt(D)
+    out = np.zeros((b, S, Hq, D))
+    for n in range(b):
+        lo, hi = int(ctx_offsets[n]), int(ctx_offsets[n + 1])
+        for a in range(S):
+            for h in range(Hq):
+                g = h // G
+                keys = np.concatenate([bf16_bits_to_f64(k_ctx[lo:hi, g]), bf16_bits_to_f64(k_spine[n, :a + 1, g])], axis=0)
+                vals = np.concatenate([bf16_bits_to_f64(v_ctx[lo:hi, g]), bf16_bits_to_f64(v_spine[n, :a + 1, g])], axis=0)
+                o, _ = softmax_attention(bf16_bits_to_f64(q_spine[n, a:a + 1, h]), keys, vals, scale)
+                out[n, a, h] = o[0]
+    return out
+
+
 def tree_mask(d: int, n_slots: int, prefix_base: int = 1) -> np.ndarray:
     """Visibility among the non-context tokens for draft length d: rows/cols ordered as the d+1 spine
     tokens followed by d+1 branches of n_slots mask tokens (Fig. 4 uses n_slots = d).  True = visible.

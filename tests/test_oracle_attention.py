@@ -224,3 +224,52 @@ def test_bf16_rounding_helper():
     t = torch.from_numpy(x).to(torch.bfloat16).to(torch.float32).numpy()
     assert np.array_equal(r, t)
     assert np.array_equal(OA.bf16_bits_to_f64(W.f32_to_bf16_bits(x)), t.astype(np.float64))
+
+
+# ----------------------------------------------------------------------------- spine tokens as query rows (next scope row)
+def _spine_q(inp, seed):
+    rng = np.random.Generator(np.random.Philox(seed))
+    b, S, Hkv, D = inp.k_spine.shape
+    Hq = inp.q.shape[3]
+    return W.f32_to_bf16_bits(rng.standard_normal((b, S, Hq, D), dtype=np.float32))
+
+
+def test_spine_rows_match_the_figures_mask():
+    """Library attention over [context | spine] under the SPINE rows of the figure's mask (from the fixture)."""
+    d = 3
+    L, Hq, Hkv, D = 5, 4, 2, 16
+    inp = _inputs((L,), Hq, Hkv, D, J=d + 1, Bq=d, seed=21)
+    qs = _spine_q(inp, 5)
+    got = OA.spine_rows(qs, inp.k_ctx, inp.v_ctx, inp.ctx_offsets, inp.k_spine, inp.v_spine)
+    S = d + 1
+    mask = _gold_mask()[:S, :S]                            # spine rows x spine columns of the figure
+    dec = lambda a: torch.from_numpy(OA.bf16_bits_to_f64(a))
+    K = torch.cat([dec(inp.k_ctx), dec(inp.k_spine[0])], 0)
+    V = torch.cat([dec(inp.v_ctx), dec(inp.v_spine[0])], 0)
+    full = torch.cat([torch.ones(S, L, dtype=torch.bool), torch.from_numpy(mask)], 1)
+    o = torch.nn.functional.scaled_dot_product_attention(
+        dec(qs[0]).permute(1, 0, 2)[None], K.permute(1, 0, 2)[None], V.permute(1, 0, 2)[None],
+        attn_mask=full[None, None], enable_gqa=True)[0]
+    assert np.abs(o.permute(1, 0, 2).numpy() - got[0]).max() < 1e-12
+
+
+def test_spine_row_equals_boundary_row_with_the_same_query_and_no_block():
+    """Anchor a reads exactly the key set of boundary j = a (prefix_base 1) without its block: putting the
+    anchor's query into slot 0 of that boundary must give the same row from the pinned boundary function."""
+    inp = _inputs((9, 0), 4, 2, 16, J=4, Bq=2, seed=8)
+    qs = _spine_q(inp, 6)
+    got = OA.spine_rows(qs, inp.k_ctx, inp.v_ctx, inp.ctx_offsets, inp.k_spine, inp.v_spine)
+    q = inp.q.copy()
+    q[:, :, 0] = qs                                        # [b][J = S][slot 0][Hq][D]
+    ref, _ = OA.draft_all_boundaries(q, inp.k_ctx, inp.v_ctx, inp.ctx_offsets, inp.k_spine, inp.v_spine, None, None,
+                                     prefix_base=1)
+    assert np.abs(ref[:, :, 0] - got).max() < 1e-12
+
+
+def test_first_anchor_without_context_returns_its_own_value():
+    inp = _inputs((0,), 2, 1, 8, J=3, Bq=2, seed=4)
+    qs = _spine_q(inp, 7)
+    got = OA.spine_rows(qs, inp.k_ctx, inp.v_ctx, inp.ctx_offsets, inp.k_spine, inp.v_spine)
+    v0 = OA.bf16_bits_to_f64(inp.v_spine[0, 0, 0])
+    assert np.array_equal(got[0, 0, 0], v0) and np.array_equal(got[0, 0, 1], v0)
+
