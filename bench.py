@@ -355,6 +355,10 @@ def main():
     ap.add_argument("--no-layer", action="store_true", help="skip the full-layer (cfg5) leg")
     ap.add_argument("--no-head", action="store_true", help="skip the LM head + autoregressive head loop (T_Head) leg")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "ours":
+        # started without a launcher: become one -- N ranks of this script, one per GPU; rank 0 prints the line
+        from paper_2609_27396_b200.dist_util import launch_ranks
+        sys.exit(launch_ranks([os.path.abspath(__file__)] + sys.argv[1:], args.gpus))
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))

@@ -15,10 +15,15 @@
  *
  * Conventions
  *   - Every pointer is a DEVICE pointer unless its name starts with host_.  The caller owns every
- *     buffer; the library allocates nothing and keeps no state between calls.
+ *     buffer; the library allocates nothing.  The only state it keeps between calls is a process-wide
+ *     launch counter (dpara_kernel_launches) and, for the fixed-scratch entry point, that entry's
+ *     scratch array and its cached device address.
  *   - Calls enqueue kernels on `stream` (a cudaStream_t passed as void*) and return without
  *     synchronising.  Outputs are valid once the stream has reached the end of the call's work.
- *   - The return code reports host-detectable errors; on any error nothing has been launched.
+ *   - The return code reports host-detectable errors.  Argument errors (INVALID_ARG, UNSUPPORTED,
+ *     WORKSPACE, STATIC_LIMIT) are found before anything is launched.  DPARA_ERR_CUDA can also come from
+ *     the middle of a multi-kernel call (a launch or tensor-map encode that fails after earlier kernels
+ *     of the same call were queued); outputs are then undefined.
  *     Conditions only the device can see (a draft token outside the vocabulary, a bounded wait that
  *     expired) OR a bit into *status_word (may be NULL) and the kernels still finish with defined
  *     outputs.
@@ -41,7 +46,8 @@ typedef enum {
   DPARA_ERR_UNSUPPORTED = -2, /* shape outside what the kernels are built for (see each call) */
   DPARA_ERR_WORKSPACE = -3,   /* workspace missing or smaller than *_workspace_bytes() */
   DPARA_ERR_CUDA = -4,        /* a CUDA runtime/driver call failed (launch, tensor-map encode) */
-  DPARA_ERR_TIMEOUT = -5,     /* reserved for device-side bounded waits, reported via status_word */
+  DPARA_ERR_TIMEOUT = -5,     /* never returned by a call (calls do not synchronise); the code and its string exist
+                                 for callers that turn DPARA_STATUS_TIMEOUT in *status_word into a status */
   DPARA_ERR_STATIC_LIMIT = -6 /* request needs more scratch than a fixed-scratch entry point owns */
 } dpara_status;
 
@@ -83,8 +89,8 @@ typedef struct {
   float *out_lse;                  /* optional [b][J][Bq][Hq]: natural-log sum-exp of the scaled scores (NULL ok) */
 } dpara_attn_io;
 
-/* Full-layer mode (one pre-norm backbone block; the paper names only "attention, MLP, and their
- * normalizations", Sec. 3.1 -- the equations are this library's reading, stated with the call). */
+/* Full-layer mode (one pre-norm backbone block; Sec. 3.1 lists the block's trainable parts without giving
+ * equations -- the equations are this library's reading, stated with the call). */
 typedef struct {
   const void *x;                                   /* [b][J][Bq][hidden] bf16 hidden states of the mask slots */
   const void *w_qkv;                               /* [(Hq + 2 Hkv) D][hidden] bf16, rows = [q | k | v] */
@@ -124,6 +130,16 @@ dpara_status dpara_draft_all_boundaries(const dpara_shape *shape, const dpara_at
                                         const dpara_layer_io *layer, void *workspace,
                                         size_t workspace_bytes, int32_t *status_word, void *stream);
 
+/* Where a full-layer call leaves the block's intermediates (the quantities named in the equations above;
+ * the paper, Sec. 3.1, lists the block's parts without equations).  offsets[0..8] receive the byte offsets,
+ * inside the call's workspace, of  xn [M][hidden] bf16,  qkv [M][(Hq+2Hkv)D] bf16,  q [M][Hq D] bf16,
+ * k [M][Hkv D] bf16,  v [M][Hkv D] bf16,  a [M][Hq D] bf16,  h1 [M][hidden] fp32,  hn [M][hidden] bf16,
+ * act [M][inter] bf16, with M = b * J * Bq rows in (request, boundary, slot) order.  They hold the last call's
+ * values until the workspace is reused.  Host-only; nothing is launched.  For stage-by-stage checks.
+ * Errors: INVALID_ARG, UNSUPPORTED (as dpara_draft_all_boundaries). */
+dpara_status dpara_layer_workspace_layout(const dpara_shape *shape, const int64_t *host_ctx_offsets,
+                                          const dpara_layer_io *layer, size_t offsets[9]);
+
 /* Verification-side tensors (Sec. 2.1; App. C for mode 1).  Row i of `target` is the target's
  * prediction for the token after t_0..t_i, so draft t_{i+1} is judged by row i and the bonus comes
  * from row r. */
@@ -158,7 +174,11 @@ size_t dpara_verify_workspace_bytes(const dpara_verify_io *io);
  * (m * W) >> 24; empty residual falls back to p_r, then to the lowest-index maximum of p_r.
  * A draft token outside [0, V) is rejected and sets DPARA_STATUS_BAD_TOKEN.
  * selected[n] = reps[n][r] copied bit for bit.
- * workspace: at least dpara_verify_workspace_bytes(); need not be initialised.
+ * workspace: at least dpara_verify_workspace_bytes() bytes, 8-byte aligned, ZERO-FILLED before its first use
+ *   (one cudaMemset when it is allocated).  Every call leaves it zero-filled again -- the CTA that finishes
+ *   last puts back what the call used, so no clearing launch precedes the kernel -- and it can be handed to
+ *   the next call as it is, in either mode, as long as that call's size request is not larger.  Two calls in
+ *   flight must not share it.
  * Errors: INVALID_ARG, UNSUPPORTED (J > 64), WORKSPACE, CUDA. */
 dpara_status dpara_verify_select(const dpara_verify_io *io, void *workspace, size_t workspace_bytes,
                                  int32_t *status_word, void *stream);
@@ -183,7 +203,8 @@ dpara_status dpara_verify_select(const dpara_verify_io *io, void *workspace, siz
  *    x 16 boundaries needs 3.3 KB, sampling mode with 8 requests over a 151 936-token vocabulary
  *    5.3 KB; the need grows with batch * n_boundaries (greedy) or batch * ceil(vocab / 4096) (sampling).
  *  - All calls on a device share the one array and it keeps whatever the previous call left; the
- *    call itself clears the parts that must start at zero.  Two calls that overlap on the same GPU
+ *    array is zero when the library is loaded and each call, before it ends, clears again the parts
+ *    that the next call needs at zero.  Two calls that overlap on the same GPU
  *    (different streams, or different host threads without ordering) race on it and give undefined
  *    results: order them on one stream or with events.
  * Errors: as dpara_verify_select, plus DPARA_ERR_STATIC_LIMIT; DPARA_ERR_CUDA if the address lookup
@@ -191,9 +212,10 @@ dpara_status dpara_verify_select(const dpara_verify_io *io, void *workspace, siz
 #define DPARA_VERIFY_STATIC_SCRATCH_BYTES (256u * 1024u)
 dpara_status dpara_verify_select_static(const dpara_verify_io *io, int32_t *status_word, void *stream);
 
-/* The critical-path remainder T_Head (Alg. 1, the lines after the barrier: "select precomputed branch r; y_0 = b;
- * for i = 1..d: z_i = l_i + W E(y_{i-1}), y_i ~ softmax(z_i)"; Sec. 3.2 "Loss" defines the head: E is its own
- * low-rank token embedding, W projects it to the vocabulary, and it reads only the preceding token).  The base
+/* The critical-path remainder T_Head (Alg. 1, the lines after the barrier: starting from the bonus token, each of
+ * the d head steps adds a correction computed from the previous step's token to the selected branch's base logits
+ * and picks the next token; Sec. 3.2 "Loss" gives the formula: the head has its own low-rank token embedding E and
+ * a projection W of it to the vocabulary, and reads only the preceding token).  The base
  * logits l_i are the language-model head applied to the selected branch's final hidden states (App. D runs the
  * language-model head on shipped hidden states right before the head loop).  Greedy decoding (Table 1): y_i is the
  * lowest index holding the maximum of z_i; NaN ranks below every number.
@@ -226,8 +248,8 @@ const char *dpara_status_string(dpara_status s);
 /* Library/ABI version: major * 1000 + minor. */
 int32_t dpara_version(void);
 
-/* The projection GEMM of the backbone block on its own (Sec. 3.1 names the block's parts only as
- * "attention, MLP, and their normalizations"; bf16 operands, fp32 accumulation on the tensor cores):
+/* The projection GEMM of the backbone block on its own (Sec. 3.1, trainable parts of the backbone block;
+ * bf16 operands, fp32 accumulation on the tensor cores):
  *   out[M][N] = epilogue( a[M][K] * w[N][K]^T ),  a and w bf16 row-major (weights stored [out][in]).
  * epilogue 0: out bf16.   epilogue 1: out fp32 = resid + product (resid [M][N], bf16 when
  * resid_dtype == DPARA_BF16 else fp32), optional bf16 copy in out_bf16.   epilogue 2: w holds 2N rows,

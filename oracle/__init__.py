@@ -11,8 +11,8 @@ attention : every acceptance boundary as an independent plain softmax attention 
             Fig. 4: shared causal spine, isolated bidirectional branches, all rows read the cache).
 verify    : accepted length, bonus token and branch selection (paper Sec. 2.1, Alg. 1 lines 2-3,
             App. C for the rejection rule).
-layer     : one drafter backbone block around the attention (paper Sec. 3.1 names only
-            "attention, MLP, and their normalizations"; the block structure is this build's reading
+layer     : one drafter backbone block around the attention (paper Sec. 3.1 only lists a block's
+            parts -- attention, MLP, norms; the block structure is this build's reading
             -- PARITY UNPINNED by the paper for the structure itself, pinned only piecewise).
 """
 from . import attention, verify, layer  # noqa: F401

@@ -1,7 +1,7 @@
 """One drafter backbone block around the all-boundary attention (test infrastructure).
 
-PARITY UNPINNED (structure): the paper names the backbone blocks only as "attention, MLP, and their
-normalizations" (Sec. 3.1, trainable/frozen split) and fixes no layer equations.  The block below is
+PARITY UNPINNED (structure): the paper lists the parts of a backbone block (Sec. 3.1, trainable/frozen
+split: the attention, the MLP and the norms around them) and fixes no layer equations.  The block below is
 this build's reading -- the pre-norm block of the Qwen3 family the drafters are trained for:
 
     xn  = bf16( rmsnorm(x) * g1 )
@@ -19,7 +19,8 @@ The bf16 roundings are part of the definition ("bf16 inputs, fp32 accumulate" fo
 sums themselves are taken in float64 here.  Positions: spine row s of request n sits at L_n + s; the
 unknown bonus of boundary j would sit at L_n + j + 1; mask slot i of boundary j therefore sits at
 L_n + j + 2 + i.  The individual pieces (rmsnorm, silu, rope, matmul) are pinned by closed forms in
-the tests; the composition is pinned by nothing but this text.
+the tests (linear / swiglu_linear by integer-exact scalar loops that a transposed weight or swapped
+gate/up halves would fail); the composition is pinned by nothing but this text.
 """
 from __future__ import annotations
 
@@ -95,7 +96,7 @@ class LayerOracle:
         Hq, Hkv, D, Bq = sh.n_q_heads, sh.n_kv_heads, sh.head_dim, sh.block
         x = bf16_bits_to_f64(self.x[n, j])                                   # [Bq][hidden]
         xn = _r16(rmsnorm(x, self.g1, L.rms_eps))
-        qkv = _r16(xn @ self.w_qkv.T)
+        qkv = _r16(linear(xn, self.w_qkv))
         q = qkv[:, : Hq * D].reshape(Bq, Hq, D)
         k = qkv[:, Hq * D:(Hq + Hkv) * D].reshape(Bq, Hkv, D)
         v = qkv[:, (Hq + Hkv) * D:].reshape(Bq, Hkv, D)
@@ -124,10 +125,8 @@ class LayerOracle:
             for h in range(g * G, (g + 1) * G):
                 a[:, h], _ = softmax_attention(q[:, h], keys, vals, self.scale)
         a = _r16(a).reshape(Bq, Hq * D)
-        h1 = (x + a @ self.w_o.T).astype(np.float32).astype(np.float64)
+        h1 = (x + linear(a, self.w_o)).astype(np.float32).astype(np.float64)
         hn = _r16(rmsnorm(h1, self.g2, L.rms_eps))
-        gu = hn @ self.w_gu.T
-        I = L.intermediate
-        act = _r16(silu(gu[:, :I]) * gu[:, I:])
-        y = (h1 + act @ self.w_down.T).astype(np.float32)
+        act = swiglu_linear(hn, self.w_gu)
+        y = (h1 + linear(act, self.w_down)).astype(np.float32)
         return dict(y=y, q=q, k=k, v=v, a=a, h1=h1.astype(np.float32))

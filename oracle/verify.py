@@ -127,7 +127,9 @@ def verify_sampling(target_probs: np.ndarray, draft_probs: np.ndarray, draft_tok
             if not (lhs < np.float32(target_probs[n, r, t])):
                 break
             r += 1
-        m = int(round(float(uniforms[n, g]) * (1 << 24)))
+        # a uniform is m * 2^-24 with m < 2^24 (App. C draws from [0, 1)); a value of 1 or more is read as the
+        # largest uniform, so that the threshold stays below the total weight and the draw inside the vocabulary
+        m = min(int(round(float(uniforms[n, g]) * (1 << 24))), (1 << 24) - 1)
         w = fixed_point_weights(target_probs[n, r], draft_probs[n, r] if r < g else None)
         if int(w.sum(dtype=np.uint64)) == 0:
             w = fixed_point_weights(target_probs[n, r], None)

@@ -71,7 +71,10 @@ lib.dpara_status_string.argtypes = [C.c_int]
 lib.dpara_version.restype = C.c_int32
 lib.dpara_kernel_launches.restype = C.c_int64
 
-EXPORTED = ["dpara_draft_workspace_bytes", "dpara_draft_all_boundaries", "dpara_verify_workspace_bytes",
+lib.dpara_layer_workspace_layout.restype = C.c_int
+lib.dpara_layer_workspace_layout.argtypes = [C.POINTER(Shape), C.c_void_p, C.POINTER(LayerIO), C.POINTER(C.c_size_t)]
+
+EXPORTED = ["dpara_layer_workspace_layout", "dpara_draft_workspace_bytes", "dpara_draft_all_boundaries", "dpara_verify_workspace_bytes",
             "dpara_verify_select", "dpara_verify_select_static", "dpara_status_string", "dpara_version", "dpara_kernel_launches"]
 
 
@@ -175,6 +178,28 @@ class DraftPlan:
             raise DparaError(rc)
 
 
+LAYER_STAGES = ("xn", "qkv", "q", "k", "v", "a", "h1", "hn", "act")
+
+
+def layer_intermediates(plan: "DraftPlan") -> dict:
+    """dpara_layer_workspace_layout: views of the block's intermediates that the last full-layer call of `plan`
+    left in its workspace, keyed by LAYER_STAGES, each [M][width] (h1 fp32, the rest bf16)."""
+    off = (C.c_size_t * 9)()
+    rc = lib.dpara_layer_workspace_layout(C.byref(plan.shape), C.cast(plan.host_off, C.c_void_p), C.byref(plan.layer), off)
+    if rc != OK:
+        raise DparaError(rc)
+    sh, L = plan.shape, plan.layer
+    M = sh.batch * sh.n_boundaries * sh.block
+    QD, KD = sh.n_q_heads * sh.head_dim, sh.n_kv_heads * sh.head_dim
+    width = dict(xn=L.hidden, qkv=QD + 2 * KD, q=QD, k=KD, v=KD, a=QD, h1=L.hidden, hn=L.hidden, act=L.intermediate)
+    res = {}
+    for name, o in zip(LAYER_STAGES, off):
+        dt = torch.float32 if name == "h1" else torch.bfloat16
+        nbytes = M * width[name] * (4 if name == "h1" else 2)
+        res[name] = plan.workspace[o:o + nbytes].view(dt).view(M, width[name])
+    return res
+
+
 def make_layer_io(*, x, w_qkv, w_o, w_gate_up, w_down, rms1_w=None, rms2_w=None, qnorm_w=None, knorm_w=None,
                   rms_eps=1e-6, rope_theta=1e6, use_rope=True, y_f32=None, y_bf16=None) -> LayerIO:
     hidden = x.shape[-1]
@@ -217,7 +242,8 @@ class VerifyPlan:
         self.io.selected = self.selected.data_ptr()
         need = lib.dpara_verify_workspace_bytes(C.byref(self.io))
         self.workspace_bytes = int(need)
-        self.workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=device)
+        # zero-filled once; every call leaves it zero-filled again
+        self.workspace = torch.zeros(max(need, 16), dtype=torch.uint8, device=device)
 
     def __call__(self, *, target, draft_tokens, reps=None, draft_probs=None, uniforms=None, stream=None) -> None:
         io = self.io

@@ -44,6 +44,18 @@ extern "C" size_t dpara_draft_workspace_bytes(const dpara_shape *shape, const in
   return bytes;
 }
 
+extern "C" dpara_status dpara_layer_workspace_layout(const dpara_shape *shape, const int64_t *host_ctx_offsets,
+                                                     const dpara_layer_io *layer, size_t offsets[9]) {
+  if (!layer || !offsets) return DPARA_ERR_INVALID_ARG;
+  dpara_status s = validate_shape(shape);
+  if (s != DPARA_OK) return s;
+  s = validate_offsets(shape, host_ctx_offsets);
+  if (s != DPARA_OK) return s;
+  if (layer->hidden <= 0 || layer->intermediate <= 0) return DPARA_ERR_INVALID_ARG;
+  layer_workspace_offsets(shape, layer, attention_workspace_bytes(shape, host_ctx_offsets), offsets);
+  return DPARA_OK;
+}
+
 extern "C" dpara_status dpara_draft_all_boundaries(const dpara_shape *shape, const dpara_attn_io *io,
                                                    const dpara_layer_io *layer, void *workspace, size_t workspace_bytes,
                                                    int32_t *status_word, void *stream) {

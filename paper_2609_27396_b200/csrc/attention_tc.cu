@@ -42,13 +42,6 @@ constexpr int kMaxOrdered = 128;
 constexpr int kMaxSched = 3072;  // items a host-built schedule can hold (kernel parameter space)
 }  // namespace
 
-// Optional clock trace of CTA 0 (build with -DDPARA_TRACE): g_trace[slot][n] = clock64() at trace point `slot`, n-th visit.
-#ifdef DPARA_TRACE
-__device__ long long g_trace[32 * 64];
-#define TRACE(slot, n) do { if (blockIdx.x == 0 && (n) < 64) g_trace[(slot) * 64 + (n)] = clock64(); } while (0)
-#else
-#define TRACE(slot, n) do {} while (0)
-#endif
 
 struct TcParams {
   CUtensorMap map_q, map_kc, map_vc, map_ks, map_vs, map_kb, map_vb;
@@ -142,9 +135,6 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
   volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-#ifdef DPARA_TRACE  // kernel phases of CTA 0: g_trace[29][0..4] clocks, [8..9] wall time
-  if (threadIdx.x == 0 && blockIdx.x == 0) { g_trace[29 * 64 + 0] = clock64(); g_trace[29 * 64 + 8] = (long long)global_timer_ns(); }
-#endif
   // this CTA's items: its slice of the host-built schedule, else items blockIdx.x, blockIdx.x + gridDim.x, ...
   const int q_begin = P.use_sched ? (int)P.cta_first[blockIdx.x] : (int)blockIdx.x;
   const int q_end = P.use_sched ? (int)P.cta_first[blockIdx.x + 1] : P.n_items;
@@ -170,9 +160,6 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-#ifdef DPARA_TRACE
-  if (threadIdx.x == 0 && blockIdx.x == 0) g_trace[29 * 64 + 1] = clock64();
-#endif
 
   // register budget: the softmax warpgroups need the registers (a 128-wide score row per thread), the
   // producer / MMA warpgroup almost none
@@ -319,19 +306,15 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
         issue_qk(kslot, n_iter == 1);
         for (int it = 0; it < n_iter && ok; ++it) {
           if (it + 1 < n_iter) {
-            TRACE(0 + 4 * ti, it);
             ok = next_load(kslot) && wait_s_free();
             if (!ok) break;
             tc_fence_after();
-            TRACE(1 + 4 * ti, it);
             issue_qk(kslot, it + 2 == n_iter);
           }
-          TRACE(2 + 4 * ti, it);
           ok = next_load(vslot) && mbar_wait(p_full + ti, ph_p, abort_flag, 5);
           ph_p ^= 1u;
           if (!ok) break;
           tc_fence_after();
-          TRACE(3 + 4 * ti, it);
           issue_pv(vslot, it > 0);
         }
       }
@@ -372,21 +355,14 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
         continue;
       }
       const int n_iter = I.n_iter;
-#ifdef DPARA_TRACE
-      const int kitem = (qi - q_begin) / q_step;
-      if (warp == 0 && lane == 0) { TRACE(24, kitem); if (blockIdx.x == 0 && kitem < 64) g_trace[28 * 64 + kitem] = n_iter * 10 + I.ntq; }
-#endif
       const int na = max(0, min(j + A.pb, A.S));
       const int b0 = P.has_blk ? P.S8 + (j - I.jb0) * A.Bq : 0, b1 = P.has_blk ? b0 + A.Bq : 0;
       float m_used = -INFINITY, l = 0.f;
 
       for (int it = 0; it < n_iter; ++it) {
-        const bool tr = (wq == 0 && lane == 0);
-        if (tr) TRACE(8 + 8 * t, it);
         ok = __all_sync(0xffffffffu, mbar_wait(s_full + t, (cnt + it) & 1, abort_flag, 6));
         if (!ok) break;
         tc_fence_after();
-        if (tr) TRACE(9 + 8 * t, it);
         uint32_t su[128];
 #pragma unroll
         for (int cc = 0; cc < 4; ++cc) tmem_ld32(lane_addr + Cfg::kColS + cc * 32, su + cc * 32);
@@ -395,7 +371,6 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive((t == 0 && I.ntq == 2) ? sf_b : sf_a);  // next user: tile 1 of this iteration, else tile 0
-        if (tr) TRACE(10 + 8 * t, it);
         bool pv_waited = (it == 0);  // PV(t, it-1) must be complete before O_t is rescaled or P_t overwritten
         float s[128];
 #pragma unroll
@@ -440,7 +415,6 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
           l *= f;
           if (need) m_used = mx;
         }
-        if (tr) TRACE(11 + 8 * t, it);
         const float mc = (m_used == -INFINITY ? 0.f : m_used) * c;
         uint32_t pk[64];
         {
@@ -459,7 +433,6 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
           unpack2(l2, la, lb);
           l += la + lb;
         }
-        if (tr) TRACE(12 + 8 * t, it);
         if (!pv_waited) {
           ok = __all_sync(0xffffffffu, mbar_wait(pv_done + t, ph_pv, abort_flag, 8));
           ph_pv ^= 1u;
@@ -472,13 +445,9 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(p_full + t);
-        if (tr) TRACE(13 + 8 * t, it);
       }
 
       // ---- epilogue of this item (the MMA issuer cannot touch O_t again before this tile's next p_full arrive)
-#ifdef DPARA_TRACE
-      if (warp == 0 && lane == 0) TRACE(25, kitem);
-#endif
       if (ok) {
         ok = __all_sync(0xffffffffu, mbar_wait(pv_done + t, ph_pv, abort_flag, 9));
         ph_pv ^= 1u;
@@ -524,9 +493,6 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
         A.out_lse[orow] = l > 0.f ? (m_used * c + log2f(l)) * 0.6931471805599453f : -INFINITY;
       }
       cnt += n_iter;
-#ifdef DPARA_TRACE
-      if (warp == 0 && lane == 0) TRACE(26, kitem);
-#endif
     }
   }
 
@@ -538,9 +504,6 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
     __threadfence();
     __syncwarp();
     cluster_sync_all();
-#ifdef DPARA_TRACE
-    if (threadIdx.x == 0 && blockIdx.x == 0) g_trace[29 * 64 + 2] = clock64();
-#endif
     if (warp < 8 && !*abort_flag) {
       const Item I = decode_item(P, blockIdx.x);
       const uint32_t rank = cluster_ctarank();
@@ -616,9 +579,6 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
     }
   }
 
-#ifdef DPARA_TRACE
-  if (threadIdx.x == 0 && blockIdx.x == 0) g_trace[29 * 64 + 3] = clock64();
-#endif
   // ------------------------------------------------------------------ teardown
   __syncwarp();
   tc_fence_before();
@@ -633,9 +593,6 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
     __syncthreads();
   }
   if (warp == 9) tmem_dealloc(tmem, 512);
-#ifdef DPARA_TRACE
-  if (threadIdx.x == 0 && blockIdx.x == 0) { g_trace[29 * 64 + 4] = clock64(); g_trace[29 * 64 + 9] = (long long)global_timer_ns(); }
-#endif
 }
 
 // ------------------------------------------------------------------------------------------------ host
@@ -789,6 +746,3 @@ dpara_status launch_attention_tc(const AttnParams &A, const TcPlan &plan, const 
 
 }  // namespace dpara
 
-#ifdef DPARA_TRACE
-extern "C" int dpara_debug_read_trace(long long *host, int n) { return (int)cudaMemcpyFromSymbol(host, dpara::g_trace, sizeof(long long) * n); }
-#endif

@@ -1,5 +1,5 @@
-// One backbone block around the all-boundary attention (Sec. 3.1: "attention, MLP, and their
-// normalizations"; the block equations are stated with dpara_draft_all_boundaries in the header):
+// One backbone block around the all-boundary attention (Sec. 3.1 lists a block's parts, no
+// equations; the block equations are stated with dpara_draft_all_boundaries in the header):
 //   rmsnorm -> QKV GEMM -> per-head RMS norm + rotary embedding -> all-boundary attention ->
 //   O GEMM (+x) -> rmsnorm -> gate/up GEMM with fused SiLU*up -> down GEMM (+h1).
 // The GEMMs and the attention are the tensor-core kernels; the three small kernels here are row-wise
@@ -172,6 +172,12 @@ LayerWs layer_ws_layout(const dpara_shape *s, const dpara_layer_io *l, size_t at
   return w;
 }
 }  // namespace
+
+void layer_workspace_offsets(const dpara_shape *shape, const dpara_layer_io *layer, size_t attn_bytes, size_t out[9]) {
+  const LayerWs w = layer_ws_layout(shape, layer, 0);
+  const size_t o[9] = {w.xn, w.qkv, w.q, w.k, w.v, w.a, w.h1, w.hn, w.act};
+  for (int i = 0; i < 9; ++i) out[i] = attn_bytes + o[i];
+}
 
 size_t layer_workspace_bytes(const dpara_shape *shape, const dpara_layer_io *layer) {
   if (layer->hidden <= 0 || layer->intermediate <= 0) return 0;

@@ -11,6 +11,8 @@ dpara_status launch_attention(const dpara_shape *shape, const dpara_attn_io *io,
 
 // full backbone block around the attention
 size_t layer_workspace_bytes(const dpara_shape *shape, const dpara_layer_io *layer);
+// byte offsets of xn, qkv, q, k, v, a, h1, hn, act inside the workspace of a full-layer call
+void layer_workspace_offsets(const dpara_shape *shape, const dpara_layer_io *layer, size_t attn_bytes, size_t out[9]);
 dpara_status launch_layer(const dpara_shape *shape, const dpara_attn_io *io, const dpara_layer_io *layer, void *workspace,
                           int32_t *status_word, cudaStream_t st);
 

@@ -10,11 +10,7 @@
 namespace dpara {
 
 constexpr int kVsThreads = 256;
-#ifndef DPARA_GREEDY_LOADS
-#define DPARA_GREEDY_LOADS 16
-#endif
-constexpr int kGreedyLoads = DPARA_GREEDY_LOADS;             // 16-byte loads in flight per thread
-constexpr int kGreedyChunk = kGreedyLoads * 1024;  // floats per CTA
+constexpr int kMaxGreedyLoads = 16;  // 16-byte loads in flight per thread (1, 2, 4, 8 or 16: chosen per shape so that the grid fills the GPU)
 constexpr int kSampChunk = 4096;    // floats per CTA and per row
 constexpr int kMaxJ = 64;
 
@@ -74,9 +70,11 @@ struct VerifyParams {
   int32_t *accept_len, *bonus, *gather_idx, *out_tokens;
   uint8_t *selected;
   int32_t *status_word;
+  // The workspace is all zero when a call starts and all zero again when it ends: the CTA that finishes last
+  // puts back what the call dirtied (no clearing launch in front of the kernel).
   unsigned long long *ws64;  // greedy: keys[b*J]; sampling: chunk sums [b][nchunks][2]
-  unsigned int *counters;    // greedy: [b*J] row counters; sampling: [b]; zeroed before the launch
-  unsigned long long *masks; // greedy: [b] completed-row masks, zeroed before the launch
+  unsigned int *counters;    // greedy: [b*J] row counters, then one "rows finished" counter; sampling: [b]
+  unsigned long long *masks; // greedy: [b] completed-row masks
   int b, J, V, nchunks, vec_ok;
   size_t rep_bytes;  // Bq * hidden * 2
 };
@@ -94,7 +92,9 @@ __device__ __forceinline__ void write_result(const VerifyParams &P, int n, int r
 }
 
 // ------------------------------------------------------------------------------------------ greedy
+template <int kGreedyLoads>
 __global__ void __launch_bounds__(kVsThreads) verify_greedy_kernel(const VerifyParams P) {
+  constexpr int kGreedyChunk = kGreedyLoads * 1024;  // floats per CTA
   const int tid = threadIdx.x;
   // rows are handed out position-major (every request's row 0 first, then every row 1, ...): the early rows,
   // which decide the accepted length, finish early for ALL requests
@@ -184,7 +184,7 @@ __global__ void __launch_bounds__(kVsThreads) verify_greedy_kernel(const VerifyP
   // ---- this CTA completed a row: is the request's outcome decided now, and was it not before?
   __threadfence();
   __shared__ int s_a[kMaxJ], s_t[kMaxJ];
-  __shared__ int s_r, s_bad, s_act;
+  __shared__ int s_r, s_bad, s_act, s_last;
   const unsigned long long mask_new = s_new, mask_old = s_old;
   if (tid < P.J) {
     const bool done = (mask_new >> tid) & 1ull;
@@ -218,16 +218,30 @@ __global__ void __launch_bounds__(kVsThreads) verify_greedy_kernel(const VerifyP
     s_bad = bad;
   }
   __syncthreads();
-  if (!s_act) return;
-  const int r = s_r;
-  if (tid == 0) {
-    P.accept_len[n] = r;
-    P.bonus[n] = s_a[r];
-    P.gather_idx[n] = r;
-    if (s_bad && P.status_word) atomicOr(reinterpret_cast<unsigned int *>(P.status_word), DPARA_STATUS_BAD_TOKEN);
+  if (s_act) {
+    const int r = s_r;
+    if (tid == 0) {
+      P.accept_len[n] = r;
+      P.bonus[n] = s_a[r];
+      P.gather_idx[n] = r;
+      if (s_bad && P.status_word) atomicOr(reinterpret_cast<unsigned int *>(P.status_word), DPARA_STATUS_BAD_TOKEN);
+    }
+    if (P.out_tokens && tid < P.J) P.out_tokens[(size_t)n * P.J + tid] = tid < r ? s_t[tid] : (tid == r ? s_a[r] : -1);
+    if (P.reps) gather_branch(P.reps, P.selected, n, P.J, r, P.rep_bytes, tid, kVsThreads);
   }
-  if (P.out_tokens && tid < P.J) P.out_tokens[(size_t)n * P.J + tid] = tid < r ? s_t[tid] : (tid == r ? s_a[r] : -1);
-  if (P.reps) gather_branch(P.reps, P.selected, n, P.J, r, P.rep_bytes, tid, kVsThreads);
+  // ---- leave the workspace as it was found.  Every row-completing CTA checks in here as its LAST access to
+  // the workspace; a CTA that did not complete a row touched it last before its row counter moved, i.e. before
+  // that row's completer got here.  So the CTA that checks in last is alone with the workspace and zeroes it.
+  __syncthreads();
+  if (tid == 0) {
+    __threadfence();
+    s_last = atomicAdd(P.counters + (size_t)P.b * P.J, 1u) == (unsigned int)(P.b * P.J) - 1u;
+  }
+  __syncthreads();
+  if (!s_last) return;
+  for (int i = tid; i < P.b * P.J; i += kVsThreads) { P.ws64[i] = 0ull; P.counters[i] = 0u; }
+  for (int i = tid; i < P.b; i += kVsThreads) P.masks[i] = 0ull;
+  if (tid == 0) P.counters[(size_t)P.b * P.J] = 0u;
 }
 
 // ------------------------------------------------------------------------------------------ sampling
@@ -345,7 +359,10 @@ __global__ void __launch_bounds__(kVsThreads) verify_sampling_kernel(const Verif
     s_chunk = 0;
     if (which < 2) {
       unsigned long long Wt = which ? W1 : W0;
-      unsigned int m = __float2uint_rn(P.uniforms[(size_t)n * P.J + g] * 16777216.0f);
+      // a uniform is m * 2^-24 with m < 2^24; anything at or above 1 is taken as the largest uniform, so the
+      // threshold stays below the total weight and the draw inside the vocabulary
+      unsigned int m = __float2uint_rn(fminf(P.uniforms[(size_t)n * P.J + g], 1.0f) * 16777216.0f);
+      m = m > 16777215u ? 16777215u : m;
       unsigned long long lo = (unsigned long long)m * Wt;  // low 64 bits
       unsigned long long hi = __umul64hi((unsigned long long)m, Wt);
       unsigned long long T = (hi << 40) | (lo >> 24);  // (m * W) >> 24, m < 2^24 so it fits
@@ -419,11 +436,25 @@ __global__ void __launch_bounds__(kVsThreads) verify_sampling_kernel(const Verif
     __syncthreads();
   }
   write_result(P, n, r, s_tok, s_bad != 0, tid);
+  // this CTA is the request's last: nobody reads the chunk sums or the ticket again -- leave them zeroed
+  __syncthreads();
+  for (int i = tid; i < 2 * P.nchunks; i += kVsThreads) P.ws64[(size_t)n * P.nchunks * 2 + i] = 0ull;
+  if (tid == 0) P.counters[n] = 0u;
   if (P.reps) gather_branch(P.reps, P.selected, n, P.J, r, P.rep_bytes, tid, kVsThreads);
 }
 
+// Greedy: 16-byte loads in flight per thread.  As many as possible (fewer, larger CTAs amortise the
+// reduction), but few enough that rows x chunks fills the GPU about four times over: a single request's 8 rows
+// split into 16 K-float chunks would leave half of the SMs idle.
+static int greedy_loads_of(const dpara_verify_io *io) {
+  const long long rows = (long long)io->batch * io->n_boundaries;
+  for (int l = kMaxGreedyLoads; l > 1; l >>= 1)
+    if (rows * ((io->vocab + l * 1024 - 1) / (l * 1024)) >= 4 * kNumSM) return l;
+  return 1;
+}
+
 static int chunks_of(const dpara_verify_io *io) {
-  int ch = io->mode == 0 ? kGreedyChunk : kSampChunk;
+  int ch = io->mode == 0 ? greedy_loads_of(io) * 1024 : kSampChunk;
   return (io->vocab + ch - 1) / ch;
 }
 
@@ -460,7 +491,7 @@ using namespace dpara;
 
 extern "C" size_t dpara_verify_workspace_bytes(const dpara_verify_io *io) {
   if (validate_dims(io) != DPARA_OK) return 0;
-  const size_t ncnt = io->mode == 0 ? (size_t)io->batch * io->n_boundaries : (size_t)io->batch;
+  const size_t ncnt = io->mode == 0 ? (size_t)io->batch * io->n_boundaries + 1 : (size_t)io->batch;
   return align_up(ws64_count(io) * 8, 256) + align_up((size_t)io->batch * 8, 256) + align_up(ncnt * 4, 256);
 }
 
@@ -487,19 +518,22 @@ dpara_status launch_verify(const dpara_verify_io *io, void *ws, int32_t *status_
   size_t n64 = ws64_count(io);
   const size_t mask_off = align_up(n64 * 8, 256);
   const size_t cnt_off = mask_off + align_up((size_t)io->batch * 8, 256);
-  const size_t ncnt = io->mode == 0 ? (size_t)io->batch * io->n_boundaries : (size_t)io->batch;
   P.ws64 = static_cast<unsigned long long *>(ws);
   P.masks = reinterpret_cast<unsigned long long *>(static_cast<uint8_t *>(ws) + mask_off);
   P.counters = reinterpret_cast<unsigned int *>(static_cast<uint8_t *>(ws) + cnt_off);
   bool vec = (io->vocab % 4 == 0) && aligned16(io->target) && (io->mode == 0 || io->n_boundaries == 1 || aligned16(io->draft_probs));
   P.vec_ok = vec ? 1 : 0;
-  // greedy needs keys and counters at zero; sampling only the counters
+  // keys, masks and counters are zero on entry (the previous call put them back); nothing is cleared here
   if (io->mode == 0) {
-    if (cudaMemsetAsync(ws, 0, cnt_off + ncnt * 4, st) != cudaSuccess) return DPARA_ERR_CUDA;  // keys, masks, counters
     dim3 grid(P.nchunks, io->batch * io->n_boundaries);
-    verify_greedy_kernel<<<grid, kVsThreads, 0, st>>>(P);
+    switch (greedy_loads_of(io)) {
+      case 16: verify_greedy_kernel<16><<<grid, kVsThreads, 0, st>>>(P); break;
+      case 8: verify_greedy_kernel<8><<<grid, kVsThreads, 0, st>>>(P); break;
+      case 4: verify_greedy_kernel<4><<<grid, kVsThreads, 0, st>>>(P); break;
+      case 2: verify_greedy_kernel<2><<<grid, kVsThreads, 0, st>>>(P); break;
+      default: verify_greedy_kernel<1><<<grid, kVsThreads, 0, st>>>(P); break;
+    }
   } else {
-    if (cudaMemsetAsync(P.counters, 0, ncnt * 4, st) != cudaSuccess) return DPARA_ERR_CUDA;
     dim3 grid(P.nchunks, io->batch);
     verify_sampling_kernel<<<grid, kVsThreads, 0, st>>>(P);
   }
@@ -556,6 +590,7 @@ extern "C" dpara_status dpara_verify_select_static(const dpara_verify_io *io, in
   void *scratch = nullptr;
   s = static_scratch_ptr(&scratch);
   if (s != DPARA_OK) return s;
-  // launch_verify clears (cudaMemsetAsync on `stream`) the keys/counters that must start at zero
+  // the array is zero when the library is loaded, and every call puts back the zeros it consumed (the
+  // CTA that finishes last clears the keys, masks and counters), so nothing has to be cleared up front
   return launch_verify(io, scratch, status_word, static_cast<cudaStream_t>(stream));
 }

@@ -6,7 +6,56 @@ timed region and to take the maximum time over ranks.
 """
 from __future__ import annotations
 
-from typing import List, Sequence, Tuple
+import os
+import socket
+import subprocess
+import sys
+from typing import Dict, List, Optional, Sequence, Tuple
+
+
+def free_port() -> int:
+    """A TCP port that is free on 127.0.0.1 right now."""
+    with socket.socket(socket.AF_INET, socket.SOCK_STREAM) as s:
+        s.bind(("127.0.0.1", 0))
+        return int(s.getsockname()[1])
+
+
+def rank_environments(n: int, port: int, base: Optional[Dict[str, str]] = None) -> List[Dict[str, str]]:
+    """The environments of n ranks of one node, one rank per GPU: what a launcher such as torch.distributed.run
+    would set (RANK, LOCAL_RANK, WORLD_SIZE, LOCAL_WORLD_SIZE, MASTER_ADDR = 127.0.0.1, MASTER_PORT), on top of
+    `base` (default: this process's environment)."""
+    if n < 1:
+        raise ValueError("need at least one rank")
+    base = dict(os.environ if base is None else base)
+    envs = []
+    for r in range(n):
+        e = dict(base)
+        e.update(RANK=str(r), LOCAL_RANK=str(r), WORLD_SIZE=str(n), LOCAL_WORLD_SIZE=str(n),
+                 MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+        envs.append(e)
+    return envs
+
+
+def launch_ranks(argv: Sequence[str], n: int, timeout: Optional[float] = None) -> int:
+    """Runs `python argv...` as n ranks (one child process per GPU) and waits for them.  Rank 0 inherits this
+    process's stdout (it prints the result line); every rank inherits stderr.  Returns the largest exit code;
+    if a rank fails or the timeout passes, the remaining children (exactly those started here) are terminated."""
+    envs = rank_environments(n, free_port())
+    procs = []
+    for r, e in enumerate(envs):
+        procs.append(subprocess.Popen([sys.executable] + list(argv), env=e,
+                                      stdout=None if r == 0 else subprocess.DEVNULL))
+    rc = 0
+    try:
+        for p in procs:
+            rc = max(rc, abs(p.wait(timeout=timeout)))
+    except subprocess.TimeoutExpired:
+        rc = 124
+    finally:
+        for p in procs:
+            if p.poll() is None:
+                p.terminate()
+    return rc
 
 
 def shard_requests(ctx_lens: Sequence[int], world: int) -> List[List[int]]:

@@ -19,8 +19,14 @@ pytestmark = pytest.mark.gpu
 TOL = 1e-2
 
 
-def _tol(ref):
-    return TOL * np.maximum(1.0, np.abs(ref))
+def _tol(ref, ctx_lens):
+    """The plain 1e-2 everywhere, except for requests with a degenerate context (fewer than 16 cached rows),
+    whose outputs can exceed 1 in magnitude: there the two terms that scale with |out| do (see above)."""
+    t = np.full(ref.shape, TOL)
+    for n, L in enumerate(ctx_lens):
+        if L < 16:
+            t[n] = TOL * np.maximum(1.0, np.abs(ref[n]))
+    return t
 
 
 def _oracle(inp, with_blk=True, **kw):
@@ -35,7 +41,7 @@ def _compare(inp, with_blk=True, lo=0, hi=None, scale=0.0):
     out, lse, status = run_attention(inp, out_dtype=torch.float32, want_lse=True, with_blk=with_blk,
                                      boundary_lo=lo, boundary_hi=hi, softmax_scale=scale)
     d = np.abs(out.cpu().numpy().astype(np.float64) - ref)
-    assert np.all(d <= _tol(ref)), d.max()
+    assert np.all(d <= _tol(ref, inp.shape.ctx_lens)), d.max()
     l = lse.cpu().numpy().astype(np.float64)
     fin = np.isfinite(ref_lse)
     assert np.array_equal(np.isfinite(l), fin)
@@ -43,7 +49,7 @@ def _compare(inp, with_blk=True, lo=0, hi=None, scale=0.0):
     out16, status = run_attention(inp, out_dtype=torch.bfloat16, want_lse=False, with_blk=with_blk,
                                   boundary_lo=lo, boundary_hi=hi, softmax_scale=scale)
     d16 = np.abs(out16.float().cpu().numpy().astype(np.float64) - ref)
-    assert np.all(d16 <= _tol(ref)), d16.max()
+    assert np.all(d16 <= _tol(ref, inp.shape.ctx_lens)), d16.max()
     assert int(status.item()) == 0
     return d.max(), d16.max()
 
@@ -97,9 +103,31 @@ def test_cfg2_full_size():
     _compare(W.make_attn_inputs(w.attn, w.seed))
 
 
+def _cfg3_rows(sh, rng):
+    """4096 query rows of the b = 16 workload: 32 for every (request, KV head), i.e. every work unit that shares a
+    K/V stream is covered whatever the kernel's tiling.  Within one (request, KV head) the rows are ordered
+    (boundary, slot, head-in-group); the picks are: all heads of the group at the LAST (boundary, slot) pair of a
+    128-row tile and at the FIRST pair of another tile (tile = 128 // G pairs), six rows of the part-filled last
+    tile, and 16 uniformly drawn rows."""
+    G = sh.n_q_heads // sh.n_kv_heads
+    n_ji = sh.n_boundaries * sh.block
+    per_tile = 128 // G
+    n_full = n_ji // per_tile
+    rows = []
+    for n in range(sh.batch):
+        for g in range(sh.n_kv_heads):
+            ta, tb = int(rng.integers(n_full)), int(rng.integers(n_full))
+            jis = [(ta * per_tile + per_tile - 1, hh) for hh in range(G)] + [(tb * per_tile, hh) for hh in range(G)]
+            tail0 = n_full * per_tile if n_full * per_tile < n_ji else n_ji - 6
+            jis += [(int(ji), int(rng.integers(G))) for ji in rng.choice(np.arange(tail0, n_ji), 6, replace=False)]
+            jis += [(int(rng.integers(n_ji)), int(rng.integers(G))) for _ in range(32 - len(jis))]
+            rows += [(n, ji // sh.block, ji % sh.block, g * G + hh) for (ji, hh) in jis]
+    return rows
+
+
 def test_cfg3_full_size_sampled_rows():
-    """Full b = 16 ragged batch in the launch configuration the benchmark times; the oracle checks a
-    seeded sample of query rows that covers every request and boundary."""
+    """Full b = 16 ragged batch in the launch configuration the benchmark times; the oracle checks 4096 seeded
+    query rows that cover every (request, KV head), every head of a group, tile edges and the part-filled tile."""
     from gpu_util import dev_bf16
     import paper_2609_27396_b200 as dp
     w = W.workload(3)
@@ -109,13 +137,22 @@ def test_cfg3_full_size_sampled_rows():
                                           [int(x) for x in inp.ctx_offsets], dev_bf16(inp.k_spine), dev_bf16(inp.v_spine),
                                           dev_bf16(inp.k_blk), dev_bf16(inp.v_blk), out_dtype=torch.bfloat16)
     torch.cuda.synchronize()
-    rng = np.random.default_rng(1)
-    rows = [(n, j, int(rng.integers(sh.block)), int(rng.integers(sh.n_q_heads)))
-            for n in range(sh.batch) for j in range(sh.n_boundaries)]
+    rows = _cfg3_rows(sh, np.random.default_rng(1))
+    assert len(rows) == 4096 and len({(n, j) for (n, j, _, _) in rows}) == sh.batch * sh.n_boundaries
+    assert {h for (_, _, _, h) in rows} == set(range(sh.n_q_heads))
     ref = OA.draft_rows(inp.q, inp.k_ctx, inp.v_ctx, inp.ctx_offsets, inp.k_spine, inp.v_spine, inp.k_blk, inp.v_blk, rows)
     o = out.float().cpu().numpy()
     got = np.stack([o[n, j, i, h] for (n, j, i, h) in rows]).astype(np.float64)
-    assert np.abs(got - ref).max() <= TOL
+    worst = float(np.abs(got - ref).max())
+    print(f"cfg3 full size, {len(rows)} rows: max |delta| {worst:.3e}")
+    assert worst <= TOL
     assert int(status.item()) == 0
     # invariant at any size: rows are convex combinations, so |out| <= max |v| seen by that KV head
     assert np.isfinite(o).all()
+
+
+def test_general_shape_kernel():
+    """Shapes whose spine prefix and own blocks do not fit the tensor-core kernel's single tail tile
+    (roundup8(n_spine) + block rows of the boundaries a tile pair touches > 128) run on the general CUDA-core kernel."""
+    _compare(W.make_attn_inputs(W.AttnShape((70, 200), 4, 2, 64, 3, 64, 1, 64), 13))
+    _compare(W.make_attn_inputs(W.AttnShape((33,), 8, 2, 128, 4, 48, 1, 40), 14), with_blk=True)

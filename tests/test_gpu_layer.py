@@ -1,19 +1,24 @@
 """GPU parity of the full backbone block (dpara_draft_all_boundaries with a layer) against the oracle's
 block, boundary by boundary.
 
-Bound on the fp32 output y: |delta| <= 1e-2 * max(1, rms(y)), i.e. the stated 1e-2 at unit scale (the error
-is additive noise of the down projection, independent of the element's own size).  Derivation:
-the oracle mirrors the block's bf16 rounding points, but the tensor-core attention rounds probabilities to
-bf16 before the PV product, so its output differs from the oracle's by ~1e-3 relative; that flips the bf16
-rounding of `a` on a large share of elements, which perturbs h1 by ~3e-5, flips ~1 % of the bf16 `hn`
-elements, moves gate/up by ~6e-4 relative and so flips the rounding of most `act` elements by one ulp:
-sqrt(12288) * (2^-8 * 0.5) * 0.02 ~ 4e-3 rms on y (measured 3.2e-3 rms, y rms 2.5, |y| up to 11), whose
-5-sigma tail over 65 536 outputs per boundary is ~1.6e-2.  The rms is asserted as well."""
+Two kinds of check.
+(1) Stage-wise, teacher-forced, at the literal 1e-2: each stage of the oracle's block is fed the KERNEL's own
+    input to that stage (read back from the workspace, dpara_layer_workspace_layout) and its result must match
+    the kernel's output of that stage: q/k/v from x, attention `a` from the kernel's q/k/v, h1 from the kernel's
+    `a`, `act` from the kernel's h1, y from the kernel's act and h1.  A stage that disagrees by more than the
+    bound is a bug in that stage, whatever the stages before it did.
+(2) Free-running: y of the whole chain against the oracle's whole chain.  Here rounding decisions differ: the
+    tensor-core attention rounds probabilities to bf16 before the PV product, so `a` differs by ~1e-3 relative,
+    which flips the bf16 rounding of `a`, of ~1 % of `hn` and of most `act` elements by one ulp; the down
+    projection turns those flips into additive noise ~4e-3 rms on y, independent of the element's size.  The
+    small shapes are held to the literal 1e-2; the long-context workload (rms(y) = 2.5, 65 536 outputs per
+    boundary block: 5-sigma tail ~1.6e-2) to 1e-2 * max(1, rms(y)) and rms <= 5e-3, with the measured maxima printed."""
 import numpy as np
 import pytest
 import torch
 
 import workloads as W
+from oracle import attention as OA
 from oracle import layer as OL
 
 pytestmark = pytest.mark.gpu
@@ -24,7 +29,7 @@ def _dev(bits):
     return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda().view(torch.bfloat16)
 
 
-def _run_layer(ain, lin, qk_norm=True, use_rope=True):
+def _run_layer(ain, lin, qk_norm=True, use_rope=True, want_stages=False):
     import paper_2609_27396_b200 as dp
     sh = ain.shape
     M = sh.batch * sh.n_boundaries * sh.block
@@ -43,7 +48,65 @@ def _run_layer(ain, lin, qk_norm=True, use_rope=True):
     torch.cuda.synchronize()
     assert int(plan.status.item()) == 0
     assert plan.workspace_bytes > 0
+    if want_stages:
+        stages = {k: v.float().cpu().numpy() for k, v in dp.layer_intermediates(plan).items()}
+        return y.cpu().numpy(), y16.float().cpu().numpy(), stages
     return y.cpu().numpy(), y16.float().cpu().numpy()
+
+
+def _stagewise(ain, lin, y, st, blocks):
+    """Teacher-forced check of every stage on the listed (request, boundary) blocks; returns the largest
+    deviation seen per stage.  bf16 stages may differ from the oracle's rounding by one ulp (2^-8 relative)
+    where the fp32 value sits next to a rounding boundary; fp32 stages and `a` are held to 1e-2."""
+    sh, L = ain.shape, lin.shape
+    Hq, Hkv, D, Bq, J = sh.n_q_heads, sh.n_kv_heads, sh.head_dim, sh.block, sh.n_boundaries
+    G = Hq // Hkv
+    orc = OL.LayerOracle(lin, ain)
+    f64 = lambda a: a.astype(np.float64)
+    worst = dict(q=0.0, k=0.0, v=0.0, a=0.0, h1=0.0, hn=0.0, act=0.0, y=0.0)
+    ulp = lambda ref: 2.0 ** -8 * np.abs(ref) + 1e-6
+
+    def upd(name, got, ref, bound):
+        d = np.abs(got - ref)
+        worst[name] = max(worst[name], float(d.max()))
+        assert np.all(d <= bound), (name, float(d.max()))
+
+    for (n, j) in blocks:
+        r0 = (n * J + j) * Bq
+        rows = slice(r0, r0 + Bq)
+        # x -> q, k, v (the oracle's own chain; the kernel's GEMM accumulates in fp32, so single-ulp flips are allowed)
+        _, q, k, v = orc.qkv_rows(n, j)
+        kq, kk, kv = (f64(st[name][rows]) for name in ("q", "k", "v"))
+        upd("q", kq, q.reshape(Bq, Hq * D), 2 * ulp(q.reshape(Bq, Hq * D)) + 2e-3)
+        upd("k", kk, k.reshape(Bq, Hkv * D), 2 * ulp(k.reshape(Bq, Hkv * D)) + 2e-3)
+        upd("v", kv, v.reshape(Bq, Hkv * D), ulp(v.reshape(Bq, Hkv * D)) + 1e-4)
+        # kernel's q, k, v -> a
+        lo, hi = int(ain.ctx_offsets[n]), int(ain.ctx_offsets[n + 1])
+        na = max(0, min(j + orc.prefix_base, sh.spine))
+        a_ref = np.zeros((Bq, Hq, D))
+        for g in range(Hkv):
+            keys = np.concatenate([OA.bf16_bits_to_f64(ain.k_ctx[lo:hi, g]), OA.bf16_bits_to_f64(ain.k_spine[n, :na, g]),
+                                   kk.reshape(Bq, Hkv, D)[:, g]])
+            vals = np.concatenate([OA.bf16_bits_to_f64(ain.v_ctx[lo:hi, g]), OA.bf16_bits_to_f64(ain.v_spine[n, :na, g]),
+                                   kv.reshape(Bq, Hkv, D)[:, g]])
+            for h in range(g * G, (g + 1) * G):
+                a_ref[:, h], _ = OA.softmax_attention(kq.reshape(Bq, Hq, D)[:, h], keys, vals, orc.scale)
+        ka = f64(st["a"][rows])
+        upd("a", ka, a_ref.reshape(Bq, Hq * D), TOL)
+        # kernel's a -> h1
+        x = OA.bf16_bits_to_f64(lin.x[n, j])
+        upd("h1", f64(st["h1"][rows]), x + OL.linear(ka, orc.w_o), TOL)
+        # kernel's h1 -> hn -> act (hn from the kernel's fp32 h1; act from the kernel's hn)
+        kh1 = f64(st["h1"][rows])
+        hn_ref = OA.round_to_bf16(OL.rmsnorm(kh1, orc.g2, L.rms_eps)).astype(np.float64)
+        khn = f64(st["hn"][rows])
+        upd("hn", khn, hn_ref, ulp(hn_ref))
+        act_ref = OL.swiglu_linear(khn, orc.w_gu)
+        kact = f64(st["act"][rows])
+        upd("act", kact, act_ref, ulp(act_ref) + 1e-4)
+        # kernel's act, h1 -> y
+        upd("y", f64(y[n, j]), kh1 + OL.linear(kact, orc.w_down), TOL)
+    return worst
 
 
 @pytest.mark.parametrize("ashape,lshape,norm,rope", [
@@ -56,8 +119,9 @@ def test_layer_parity(ashape, lshape, norm, rope):
     lshape = dataclasses.replace(lshape, qk_norm=norm, use_rope=rope)
     ain = W.make_attn_inputs(ashape, 31, with_q=False, with_blk=False)
     lin = W.make_layer_inputs(lshape, ashape, 31)
-    y, y16 = _run_layer(ain, lin, norm, rope)
+    y, y16, st = _run_layer(ain, lin, norm, rope, want_stages=True)
     orc = OL.LayerOracle(lin, ain)
+    print("stage-wise max |delta|:", _stagewise(ain, lin, y, st, [(n, j) for n in range(ashape.batch) for j in range(ashape.n_boundaries)]))
     worst = 0.0
     for n in range(ashape.batch):
         for j in range(ashape.n_boundaries):
@@ -73,13 +137,21 @@ def test_cfg5_full_size_sampled_boundaries():
     w = W.workload(5)
     ain = W.make_attn_inputs(w.attn, w.seed, with_q=False, with_blk=False)
     lin = W.make_layer_inputs(w.layer, w.attn, w.seed)
-    y, y16 = _run_layer(ain, lin, True, True)
+    y, y16, st = _run_layer(ain, lin, True, True, want_stages=True)
     assert np.isfinite(y).all()
     orc = OL.LayerOracle(lin, ain)
     rng = np.random.default_rng(5)
-    picks = {(0, 0), (3, 15)} | {(int(rng.integers(4)), int(rng.integers(16))) for _ in range(4)}
-    for (n, j) in sorted(picks):
+    picks = sorted({(0, 0), (3, 15), (1, 7), (2, 8)} | {(int(rng.integers(4)), int(rng.integers(16))) for _ in range(8)})
+    # (1) every stage, fed the kernel's own input to it, at the literal bound
+    stage_worst = _stagewise(ain, lin, y, st, picks)
+    # (2) the free-running chain: noise of rounding flips, bound scaled by rms(y); measured maxima are printed
+    free_max, free_rms, y_rms = 0.0, 0.0, 0.0
+    for (n, j) in picks:
         ref = orc.boundary(n, j)["y"].astype(np.float64)
         d = np.abs(y[n, j] - ref)
-        assert np.all(d <= TOL * max(1.0, float(np.sqrt((ref * ref).mean())))), (n, j, float(d.max()))
+        rms_ref = float(np.sqrt((ref * ref).mean()))
+        free_max, free_rms, y_rms = max(free_max, float(d.max())), max(free_rms, float(np.sqrt((d * d).mean()))), max(y_rms, rms_ref)
+        assert np.all(d <= TOL * max(1.0, rms_ref)), (n, j, float(d.max()))
         assert np.sqrt((d * d).mean()) <= 5e-3
+    print(f"cfg5 layer, {len(picks)} of 64 blocks: stage-wise max |delta| {stage_worst}; free-running y max |delta| {free_max:.3e}, "
+          f"rms {free_rms:.3e}, rms(y) {y_rms:.2f}")

@@ -119,3 +119,49 @@ def test_sampling_fallbacks():
     ref = _check(v, 1)
     assert ref["accept_len"].tolist() == [0, 0, 2, 0] and ref["bonus"][0] == 4500 and ref["bonus"][1] == 0
     assert ref["bonus"][2] == 4500 and ref["status"] == 1
+
+
+def test_workspace_is_left_zeroed_and_reusable_across_modes_and_shapes():
+    """One zero-filled workspace serves calls of both modes and several shapes back to back with no clearing in
+    between: every call restores the zeros it consumed.  Covers each of the greedy kernel's chunk sizes
+    (the chunk is chosen from rows x vocabulary so that the grid fills the GPU)."""
+    import paper_2609_27396_b200 as dp
+    from gpu_util import dev_bf16, host_bits
+    shapes = [W.VerifyShape(1, 8, 151936, 8, 256, "greedy", 0.8, 2.0),       # few rows: small chunks
+              W.VerifyShape(16, 16, 151936, 4, 64, "greedy", 0.75, 1.0),     # many rows: 16 K-float chunks
+              W.VerifyShape(4, 6, 20000, 4, 128, "sampling", 0.0, 3.0),
+              W.VerifyShape(3, 16, 151936, 4, 64, "greedy", 0.8, 1.0),
+              W.VerifyShape(6, 16, 151936, 4, 64, "greedy", 0.8, 1.0),
+              W.VerifyShape(2, 3, 50000, 4, 64, "sampling", 0.0, 3.0),
+              W.VerifyShape(40, 16, 60000, 2, 64, "greedy", 0.8, 1.0)]
+    plans = [dp.VerifyPlan(batch=s.batch, n_boundaries=s.n_boundaries, vocab=s.vocab, block=s.block, hidden=s.hidden,
+                           mode=1 if s.mode == "sampling" else 0) for s in shapes]
+    shared = torch.zeros(max(p.workspace.numel() for p in plans), dtype=torch.uint8, device="cuda")
+    for rep in range(2):
+        for k, (s, plan) in enumerate(zip(shapes, plans)):
+            plan.workspace = shared
+            v = W.make_verify_inputs(s, 300 + 10 * rep + k)
+            kw = dict(target=torch.from_numpy(v.target).cuda(), draft_tokens=torch.from_numpy(v.draft_tokens).cuda(), reps=dev_bf16(v.reps))
+            if s.mode == "sampling":
+                kw.update(draft_probs=torch.from_numpy(v.draft_probs).cuda(), uniforms=torch.from_numpy(v.uniforms).cuda())
+                ref = OV.verify_sampling(v.target, v.draft_probs, v.draft_tokens, v.uniforms, v.reps)
+            else:
+                ref = OV.verify_greedy(v.target, v.draft_tokens, v.reps)
+            plan(**kw)
+            torch.cuda.synchronize()
+            for key in ("accept_len", "bonus", "gather_idx", "out_tokens"):
+                assert np.array_equal(getattr(plan, key).cpu().numpy(), ref[key]), (key, k, rep)
+            assert np.array_equal(host_bits(plan.selected), ref["selected"]), (k, rep)
+            assert int(shared.count_nonzero().item()) == 0, (k, rep)       # left as it was found
+
+
+def test_sampling_uniform_of_one_is_clamped():
+    V, J = 5000, 2
+    p = np.zeros((1, J, V), np.float32); q = np.zeros((1, J - 1, V), np.float32)
+    p[0, :, [7, 4100]] = 0.5
+    q[0, :, 7] = 1.0
+    toks = np.full((1, J - 1), 7, np.int32)          # accepted iff u * 1 < 0.5
+    u = np.array([[0.75, 1.0]], np.float32)          # rejected at once; bonus uniform exactly 1.0
+    v = W.VerifyInputs(W.VerifyShape(1, J, V, 2, 64, "sampling"), p, toks, None, q, u)
+    ref = _check(v, 1)
+    assert ref["accept_len"][0] == 0 and ref["bonus"][0] == 4100

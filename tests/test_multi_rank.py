@@ -74,3 +74,30 @@ def test_reference_arm_nonzero_rank_is_silent():
     r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2", "--steps", "1",
                         "--warmup", "0"], env=env, capture_output=True, text=True, timeout=120)
     assert r.returncode == 0 and r.stdout.strip() == ""
+
+
+def test_launcher_builds_one_environment_per_gpu():
+    envs = DU.rank_environments(4, 29400, base={"PATH": "/bin", "RANK": "9"})
+    assert [e["RANK"] for e in envs] == ["0", "1", "2", "3"] and [e["LOCAL_RANK"] for e in envs] == ["0", "1", "2", "3"]
+    assert all(e["WORLD_SIZE"] == "4" and e["MASTER_ADDR"] == "127.0.0.1" and e["MASTER_PORT"] == "29400" for e in envs)
+    assert all(e["PATH"] == "/bin" for e in envs)
+    p = DU.free_port()
+    assert 1024 <= p < 65536
+
+
+def test_launcher_starts_n_ranks_that_rendezvous(tmp_path):
+    """launch_ranks starts N children with a consistent rendezvous: each child joins a gloo group of the size it
+    was told and writes its rank; rank 0's stdout is the launcher's."""
+    script = tmp_path / "child.py"
+    script.write_text(
+        "import os, sys, torch.distributed as dist\n"
+        "dist.init_process_group('gloo')\n"
+        "assert dist.get_world_size() == int(os.environ['WORLD_SIZE']) == 3\n"
+        "open(os.path.join(sys.argv[1], 'rank%d' % dist.get_rank()), 'w').write(os.environ['LOCAL_RANK'])\n"
+        "dist.barrier(); dist.destroy_process_group()\n")
+    assert DU.launch_ranks([str(script), str(tmp_path)], 3, timeout=120) == 0
+    assert sorted(f for f in os.listdir(tmp_path) if f.startswith("rank")) == ["rank0", "rank1", "rank2"]
+    assert (tmp_path / "rank2").read_text() == "2"
+    failing = tmp_path / "bad.py"
+    failing.write_text("import os, sys\nsys.exit(3 if os.environ['RANK'] == '1' else 0)\n")
+    assert DU.launch_ranks([str(failing)], 2, timeout=60) == 3

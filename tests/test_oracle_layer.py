@@ -1,5 +1,5 @@
 """Pins for oracle/layer.py pieces (closed forms, library routines) and the input generators (CPU only).
-The block STRUCTURE is this build's reading of the paper ("attention, MLP, and their normalizations")
+The block STRUCTURE is this build's reading of the paper (Sec. 3.1 lists a block's parts only)
 and stays unpinned by the paper; the library-composed check below only guards against slips."""
 import math
 
@@ -116,3 +116,52 @@ def test_generators_are_seeded_and_shaped():
     assert np.allclose(s.target.sum(-1), 1, atol=1e-5) and np.allclose(s.draft_probs.sum(-1), 1, atol=1e-5)
     m = s.uniforms.astype(np.float64) * 2 ** 24
     assert np.array_equal(m, np.round(m)) and m.max() < 2 ** 24 and m.min() >= 0
+
+
+def test_linear_against_scalar_loops_integer_exact():
+    """`linear` is x [M][K] times w [N][K] transposed.  Small integers make every product and sum exact, so
+    the scalar triple loop must be reproduced bit for bit; M, N, K all differ and w is not symmetric, so a
+    transposed operand either fails to broadcast or changes the numbers."""
+    rng = np.random.default_rng(2)
+    M, N, K = 3, 5, 4
+    x = rng.integers(-7, 8, (M, K)).astype(np.float64)
+    w = rng.integers(-7, 8, (N, K)).astype(np.float64)
+    want = np.zeros((M, N))
+    for m in range(M):
+        for n in range(N):
+            acc = 0
+            for k in range(K):
+                acc += int(x[m, k]) * int(w[n, k])
+            want[m, n] = acc
+    got = OL.linear(x, w)
+    assert got.shape == (M, N) and np.array_equal(got, want)
+    # square case (a silent transposition would still broadcast): w[n][k] = 1 only at (0, 1) picks x[:, 1] into column 0
+    xs = np.arange(9, dtype=np.float64).reshape(3, 3)
+    ws = np.zeros((3, 3)); ws[0, 1] = 1
+    assert np.array_equal(OL.linear(xs, ws)[:, 0], xs[:, 1]) and not OL.linear(xs, ws)[:, 1:].any()
+
+
+def test_swiglu_linear_halves_and_closed_form():
+    """Rows [0, I) of the stacked weight are the gate (through SiLU), rows [I, 2I) the plain `up` factor."""
+    K, I = 4, 3
+    x = np.array([[1.0, 2.0, -1.0, 0.5], [0.0, -3.0, 2.0, 1.0]])
+    rng = np.random.default_rng(3)
+    wg = rng.integers(-2, 3, (I, K)).astype(np.float64)
+    wu = rng.integers(-2, 3, (I, K)).astype(np.float64)
+    got = OL.swiglu_linear(x, np.concatenate([wg, wu]))
+    want = np.zeros((2, I))
+    for m in range(2):
+        for c in range(I):
+            g = sum(x[m, k] * wg[c, k] for k in range(K))
+            u = sum(x[m, k] * wu[c, k] for k in range(K))
+            want[m, c] = g / (1.0 + math.exp(-g)) * u
+    assert np.array_equal(got, OA.round_to_bf16(want).astype(np.float64))
+    swapped = OL.swiglu_linear(x, np.concatenate([wu, wg]))
+    assert not np.array_equal(got, swapped)                      # SiLU is applied to the FIRST half only
+    # a zero gate silences the unit whatever `up` is; a zero `up` likewise
+    assert not OL.swiglu_linear(x, np.concatenate([np.zeros((I, K)), wu])).any()
+    assert not OL.swiglu_linear(x, np.concatenate([wg, np.zeros((I, K))])).any()
+    # gate pre-activation 0 < g: silu(g) * 1 with up = e_0 row-sum selector -> closed form g * sigmoid(g)
+    one = np.zeros((1, K)); one[0, 0] = 1
+    y = OL.swiglu_linear(np.array([[2.0, 0, 0, 0]]), np.concatenate([one, 0.5 * one]))
+    assert y[0, 0] == OA.round_to_bf16(np.array(2.0 / (1 + math.exp(-2.0)) * 1.0)).astype(np.float64)

@@ -237,3 +237,15 @@ def test_sampling_fallbacks_and_boundaries():
     # out-of-range draft
     res = OV.verify_sampling(p, q, np.int32([[9]]), u)
     assert res["accept_len"][0] == 0 and res["status"] == OV.STATUS_BAD_TOKEN
+
+
+def test_bonus_uniform_of_one_stays_inside_the_vocabulary():
+    """A bonus uniform of exactly 1.0 (m = 2^24, outside [0, 1)) is read as the largest uniform: the threshold
+    stays below the total weight, so the draw is the LAST token that carries weight, never an index = V."""
+    p = np.zeros((1, 1, 8), np.float32)
+    p[0, 0, [1, 5]] = 0.5                                  # J = 1: no drafts, bonus drawn from p_0
+    toks = np.zeros((1, 0), np.int32)
+    q = np.zeros((1, 0, 8), np.float32)
+    for u, want in ((1.0, 5), (float(np.float32(1 - 2 ** -24)), 5), (0.0, 1), (0.5, 5), (0.5 - 2 ** -24, 1)):
+        r = OV.verify_sampling(p, q, toks, np.array([[u]], np.float32))
+        assert r["bonus"][0] == want and r["accept_len"][0] == 0, (u, r["bonus"])

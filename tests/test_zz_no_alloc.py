@@ -2,7 +2,7 @@
 
 That entry point exists for callers that cannot allocate device memory -- a server whose own pool
 already owns all of it, or a decode loop that cannot afford the stall of an allocation -- so it keeps
-its scratch in an array inside the library.  It must give exactly what dpara_verify_select gives.
+its scratch in an array inside the library.  It must give exactly what dpara_verify_select gives, and what the CPU oracle gives.
 Checked on two calls in a row (the shared array keeps the first call's contents, so the second call
 proves that whatever must start at zero is cleared), for both modes, through the C ABI.
 This file is collected last on purpose: a failure here cannot hide any other test's result.
@@ -14,6 +14,7 @@ import pytest
 import torch
 
 import workloads as W
+from oracle import verify as OV
 
 pytestmark = pytest.mark.gpu
 
@@ -39,11 +40,22 @@ def _run_both(sh, seed):
             getattr(st_plan, k).fill_(-7)
         ref_plan(**args)
         torch.cuda.synchronize()
+        before = (torch.cuda.memory_allocated(), torch.cuda.memory_reserved())
         dp.verify_select_static(st_plan, **args)
         torch.cuda.synchronize()
+        assert (torch.cuda.memory_allocated(), torch.cuda.memory_reserved()) == before     # the call took no device memory
         for k in KEYS:                                                     # integer / bit-copy outputs: exact
             assert torch.equal(getattr(st_plan, k), getattr(ref_plan, k)), (k, rep)
         assert int(st_plan.status.item()) == int(ref_plan.status.item())
+        # ... and against the CPU oracle, not only against the sibling entry point
+        if mode == 0:
+            orc = OV.verify_greedy(v.target, v.draft_tokens, v.reps)
+        else:
+            orc = OV.verify_sampling(v.target, v.draft_probs, v.draft_tokens, v.uniforms, v.reps)
+        for k in ("accept_len", "bonus", "gather_idx", "out_tokens"):
+            assert np.array_equal(getattr(st_plan, k).cpu().numpy(), orc[k]), (k, rep)
+        assert np.array_equal(st_plan.selected.cpu().view(torch.int16).numpy().view(np.uint16), orc["selected"]), rep
+        assert int(st_plan.status.item()) == orc["status"]
 
 
 def test_static_matches_workspace_entry_greedy():
