@@ -4,7 +4,7 @@ block, boundary by boundary.
 Two kinds of check.
 (1) Stage-wise, teacher-forced, at the literal 1e-2: each stage of the oracle's block is fed the KERNEL's own
     input to that stage (read back from the workspace, dpara_layer_workspace_layout) and its result must match
-    the kernel's output of that stage: q/k/v from x, attention `a` from the kernel's q/k/v, h1 from the kernel's
+    the kernel's output of that stage: xn from x, qkv from the kernel's xn, q/k from the kernel's qkv, attention `a` from the kernel's q/k/v, h1 from the kernel's
     `a`, `act` from the kernel's h1, y from the kernel's act and h1.  A stage that disagrees by more than the
     bound is a bug in that stage, whatever the stages before it did.
 (2) Free-running: y of the whole chain against the oracle's whole chain.  Here rounding decisions differ: the
@@ -56,15 +56,16 @@ def _run_layer(ain, lin, qk_norm=True, use_rope=True, want_stages=False):
 
 def _stagewise(ain, lin, y, st, blocks):
     """Teacher-forced check of every stage on the listed (request, boundary) blocks; returns the largest
-    deviation seen per stage.  bf16 stages may differ from the oracle's rounding by one ulp (2^-8 relative)
+    deviation seen per stage.  bf16 stages may differ from the oracle's rounding by one step (at most 2^-7 relative)
     where the fp32 value sits next to a rounding boundary; fp32 stages and `a` are held to 1e-2."""
     sh, L = ain.shape, lin.shape
     Hq, Hkv, D, Bq, J = sh.n_q_heads, sh.n_kv_heads, sh.head_dim, sh.block, sh.n_boundaries
     G = Hq // Hkv
     orc = OL.LayerOracle(lin, ain)
     f64 = lambda a: a.astype(np.float64)
-    worst = dict(q=0.0, k=0.0, v=0.0, a=0.0, h1=0.0, hn=0.0, act=0.0, y=0.0)
-    ulp = lambda ref: 2.0 ** -8 * np.abs(ref) + 1e-6
+    worst = dict(xn=0.0, qkv=0.0, q=0.0, k=0.0, a=0.0, h1=0.0, hn=0.0, act=0.0, y=0.0)
+    r16 = lambda a: OA.round_to_bf16(a).astype(np.float64)
+    ulp = lambda ref: 2.0 ** -7 * np.abs(ref) + 1e-6      # one bf16 step is at most 2^-7 of the value
 
     def upd(name, got, ref, bound):
         d = np.abs(got - ref)
@@ -74,12 +75,28 @@ def _stagewise(ain, lin, y, st, blocks):
     for (n, j) in blocks:
         r0 = (n * J + j) * Bq
         rows = slice(r0, r0 + Bq)
-        # x -> q, k, v (the oracle's own chain; the kernel's GEMM accumulates in fp32, so single-ulp flips are allowed)
-        _, q, k, v = orc.qkv_rows(n, j)
+        # x -> xn -> qkv -> (per-head norm, rotary embedding) -> q, k; v is the plain copy
+        x = OA.bf16_bits_to_f64(lin.x[n, j])
+        xn_ref = r16(OL.rmsnorm(x, orc.g1, L.rms_eps))
+        kxn = f64(st["xn"][rows])
+        upd("xn", kxn, xn_ref, ulp(xn_ref))
+        qkv_ref = r16(OL.linear(kxn, orc.w_qkv))
+        kqkv = f64(st["qkv"][rows])
+        upd("qkv", kqkv, qkv_ref, ulp(qkv_ref) + 1e-5)
         kq, kk, kv = (f64(st[name][rows]) for name in ("q", "k", "v"))
-        upd("q", kq, q.reshape(Bq, Hq * D), 2 * ulp(q.reshape(Bq, Hq * D)) + 2e-3)
-        upd("k", kk, k.reshape(Bq, Hkv * D), 2 * ulp(k.reshape(Bq, Hkv * D)) + 2e-3)
-        upd("v", kv, v.reshape(Bq, Hkv * D), ulp(v.reshape(Bq, Hkv * D)) + 1e-4)
+        assert np.array_equal(kv, kqkv[:, (Hq + Hkv) * D:])
+        pos = sh.ctx_lens[n] + j + 2 + np.arange(Bq)
+        for name, got, lo_c, H, gain in (("q", kq, 0, Hq, orc.gq), ("k", kk, Hq * D, Hkv, orc.gk)):
+            t = kqkv[:, lo_c:lo_c + H * D].reshape(Bq, H, D)
+            bound = np.zeros_like(t)
+            if L.qk_norm:
+                t = r16(OL.rmsnorm(t, gain, L.rms_eps))
+                bound = bound + ulp(t)
+            if L.use_rope:
+                # a one-step difference in either member of a rotated pair (d, d + D/2) moves both outputs
+                bound = bound + np.roll(bound, D // 2, axis=-1)
+                t = r16(OL.rope(t.transpose(1, 0, 2), pos, L.rope_theta).transpose(1, 0, 2))
+            upd(name, got, t.reshape(Bq, H * D), (bound + ulp(t)).reshape(Bq, H * D))
         # kernel's q, k, v -> a
         lo, hi = int(ain.ctx_offsets[n]), int(ain.ctx_offsets[n + 1])
         na = max(0, min(j + orc.prefix_base, sh.spine))
@@ -94,7 +111,6 @@ def _stagewise(ain, lin, y, st, blocks):
         ka = f64(st["a"][rows])
         upd("a", ka, a_ref.reshape(Bq, Hq * D), TOL)
         # kernel's a -> h1
-        x = OA.bf16_bits_to_f64(lin.x[n, j])
         upd("h1", f64(st["h1"][rows]), x + OL.linear(ka, orc.w_o), TOL)
         # kernel's h1 -> hn -> act (hn from the kernel's fp32 h1; act from the kernel's hn)
         kh1 = f64(st["h1"][rows])
