@@ -46,14 +46,14 @@ __device__ __forceinline__ void gather_branch(const uint8_t *__restrict__ reps, 
     const uint4 *s = reinterpret_cast<const uint4 *>(src);
     uint4 *d = reinterpret_cast<uint4 *>(dst);
     const size_t nv = bytes >> 4;
-    // 16 independent 16-byte loads in flight per thread: the copy is one CTA's job, so latency matters
+    // 8 independent 16-byte loads in flight per thread: the copy is one CTA's job, so latency matters
     size_t i = tid;
-    for (; i + 15 * (size_t)nthreads < nv; i += 16 * (size_t)nthreads) {
-      uint4 v[16];
+    for (; i + 7 * (size_t)nthreads < nv; i += 8 * (size_t)nthreads) {
+      uint4 v[8];
 #pragma unroll
-      for (int k = 0; k < 16; ++k) v[k] = __ldcs(s + i + k * (size_t)nthreads);
+      for (int k = 0; k < 8; ++k) v[k] = __ldcs(s + i + k * (size_t)nthreads);
 #pragma unroll
-      for (int k = 0; k < 16; ++k) d[i + k * (size_t)nthreads] = v[k];
+      for (int k = 0; k < 8; ++k) d[i + k * (size_t)nthreads] = v[k];
     }
     for (; i < nv; i += nthreads) d[i] = __ldcs(s + i);
   } else {
@@ -93,7 +93,7 @@ __device__ __forceinline__ void write_result(const VerifyParams &P, int n, int r
 
 // ------------------------------------------------------------------------------------------ greedy
 template <int kGreedyLoads>
-__global__ void __launch_bounds__(kVsThreads) verify_greedy_kernel(const VerifyParams P) {
+__global__ void __launch_bounds__(kVsThreads, kGreedyLoads >= 16 ? 3 : (kGreedyLoads >= 8 ? 4 : 6)) verify_greedy_kernel(const VerifyParams P) {
   constexpr int kGreedyChunk = kGreedyLoads * 1024;  // floats per CTA
   const int tid = threadIdx.x;
   // rows are handed out position-major (every request's row 0 first, then every row 1, ...): the early rows,
@@ -443,13 +443,13 @@ __global__ void __launch_bounds__(kVsThreads) verify_sampling_kernel(const Verif
   if (P.reps) gather_branch(P.reps, P.selected, n, P.J, r, P.rep_bytes, tid, kVsThreads);
 }
 
-// Greedy: 16-byte loads in flight per thread.  As many as possible (fewer, larger CTAs amortise the
-// reduction), but few enough that rows x chunks fills the GPU about four times over: a single request's 8 rows
-// split into 16 K-float chunks would leave half of the SMs idle.
+// Greedy: 16-byte loads in flight per thread.  As many as possible (fewer, larger CTAs amortise the reduction
+// and the completion atomics: measured 37 / 38 / 43 / 64 us at 16 / 8 / 4 / 2 loads for 16 requests x 16 rows),
+// but few enough that rows x chunks gives every SM a CTA (a single request's 8 rows: 8 loads, 152 CTAs).
 static int greedy_loads_of(const dpara_verify_io *io) {
   const long long rows = (long long)io->batch * io->n_boundaries;
   for (int l = kMaxGreedyLoads; l > 1; l >>= 1)
-    if (rows * ((io->vocab + l * 1024 - 1) / (l * 1024)) >= 4 * kNumSM) return l;
+    if (rows * ((io->vocab + l * 1024 - 1) / (l * 1024)) >= kNumSM) return l;
   return 1;
 }
 
