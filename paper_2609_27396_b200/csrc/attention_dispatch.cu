@@ -1,4 +1,4 @@
-// Chooses the attention kernel for a shape and fills its parameters.
+// Fills the attention kernel's parameters from the C-ABI structs and launches it.
 #include <math.h>
 
 #include "attention_tc.cuh"
@@ -36,8 +36,8 @@ dpara_status launch_attention(const dpara_shape *shape, const dpara_attn_io *io,
   fill_attn_params(P, shape, io, status_word);
   if (P.hi <= P.lo) return DPARA_OK;
   TcPlan plan = plan_attention_tc(shape, io->host_ctx_offsets);
-  if (plan.eligible) return launch_attention_tc(P, plan, io->host_ctx_offsets, workspace, st);
-  return launch_attention_simt(P, st);
+  if (!plan.eligible) return DPARA_ERR_UNSUPPORTED;  // group size > 16, block > 64, spine > 64, or more than 2^31 rows
+  return launch_attention_tc(P, plan, io->host_ctx_offsets, workspace, st);
 }
 
 }  // namespace dpara

@@ -1,4 +1,4 @@
-// Parameters shared by the attention kernels (plain structs, passed by value).
+// Parameters of the attention kernel (plain struct, passed by value).
 #pragma once
 #include "common.cuh"
 
@@ -17,7 +17,5 @@ struct AttnParams {
   float scale;                      // softmax scale (natural-exp domain)
   int32_t *status_word;
 };
-
-dpara_status launch_attention_simt(const AttnParams &P, cudaStream_t st);
 
 }  // namespace dpara

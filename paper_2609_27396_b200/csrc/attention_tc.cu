@@ -1,14 +1,18 @@
 // All-boundary attention on the 5th-generation tensor cores (Sec. 3.2, Fig. 4).
 //
-// Work item = (request n, KV head g, pair of 128-row query tiles, KV split).  The query rows of one
-// (n, g) are ordered (boundary j, slot i, head-in-group), so one 128-row tile holds whole (j, i) rows
-// of all G query heads that share the KV head, and every K/V byte streamed from HBM serves all
-// boundaries and all heads of the group at once.
+// Work item = (request n, KV head g, pair of 128-row query tiles, KV split).  Every K/V byte streamed from
+// HBM serves all boundaries and all query heads of the group that share the KV head.  The G heads of a
+// group are cut into "head blocks" of 8, 4, 2 or 1 heads (the binary digits of G: G = 5 -> 4 + 1); a
+// query tile holds hb heads x (128 / hb) consecutive (boundary j, slot i) rows of one head block, ordered
+// (j, i, head), which is one 3-D TMA box of the q tensor -- so every tile is full whatever G is (a tile of
+// 128 / G whole (j, i) rows of all G heads leaves rows idle and a part-filled last tile when G is not a
+// power of two).
 //
 //   warp 8      TMA producer: Q tiles once, then K and V tiles of 128 keys through one ring of tile slots
 //               (order K0 K1 V0 K2 V1 ...).  The context needs no mask at all (every row sees the whole
-//               cache); the spine prefix and the boundaries' own blocks are packed into ONE extra "tail"
-//               tile per CTA.
+//               cache); the spine prefix and the own blocks of the boundaries a tile pair touches are
+//               packed into extra "tail" tiles (the first holds the spine and as many blocks as fit next to
+//               it; usually it is the only one).
 //   warps 9, 10 one thread per query tile issues tcgen05.mma:  S = Q_t K^T  (A, B from shared memory) and
 //               O_t += P_t V  (A = P_t from tensor memory, B = V, MN-major).
 //   warps 0-3   softmax of tile 0, warps 4-7 softmax of tile 1: thread = row.  tcgen05.ld the S row into
@@ -40,13 +44,18 @@ constexpr int kThreads = 384;  // warps 0-7 softmax, 8 TMA producer, 9 and 10 MM
 constexpr float kRescaleLog2 = 8.0f;
 constexpr int kMaxOrdered = 128;
 constexpr int kMaxSched = 3072;  // items a host-built schedule can hold (kernel parameter space)
+constexpr int kMaxHeadBlocks = 4;  // G <= 16: at most four binary digits unless G == 16 (one block)
 }  // namespace
 
 
 struct TcParams {
-  CUtensorMap map_q, map_kc, map_vc, map_ks, map_vs, map_kb, map_vb;
+  CUtensorMap map_q[kMaxHeadBlocks], map_kc, map_vc, map_ks, map_vs, map_kb0, map_vb0, map_kb, map_vb;
   AttnParams a;
-  int JI_T, n_ji, n_tiles, n_pairs, nsplit, S8, R_blk, has_blk, has_tail, n_items;
+  // head blocks: block k covers heads [h0[k], h0[k] + (1 << hb_log2[k])) of every group; its tiles hold
+  // 128 >> hb_log2[k] (j, i) rows; its tile pairs are pair_start[k] .. pair_start[k + 1] - 1
+  int n_hblk, hb_log2[kMaxHeadBlocks], h0[kMaxHeadBlocks], pair_start[kMaxHeadBlocks + 1];
+  // tail tiles: the first holds the spine (S8 = S rounded up to 8 rows) and cap0 blocks, the others cap blocks
+  int n_ji, n_pairs, nsplit, S8, cap0, cap, has_blk, has_tail, n_items;
   float *part_o;   // split-KV partials [item slot][2][D / 4][128 rows] float4 (unnormalised rows; a warp's lanes are
                    // consecutive rows, so its stores and the merge's loads are contiguous 512-byte runs)
   float2 *part_ml; // [item slot][2][128] (row max in raw-score units, row sum)
@@ -83,10 +92,20 @@ struct TcCfg {
 
 // One unit of work of a persistent CTA.
 struct Item {
-  int n, g, pair, split, ntq, L, t0, t1, nctx, n_ctx_it, n_iter, jb0, slot;
+  int n, g, pair, split, ntq, L, t0, t1, nctx, n_ctx_it, n_tail, n_iter, jb0, slot;
+  int blk, hs, h0, ji_t, ji0;  // head block, log2(heads per row group), first head, (j, i) rows per tile, first (j, i) row
   long long c0;
-  bool do_tail;
 };
+
+// The low k bits set (k <= 0: none, k >= 32: all).
+__device__ __forceinline__ uint32_t bits_below(int k) { return k <= 0 ? 0u : (k >= 32 ? 0xffffffffu : ((1u << k) - 1u)); }
+
+// Tail tiles a tile pair needs: its boundaries' own blocks, cap0 of them next to the spine in the first tile.
+__host__ __device__ __forceinline__ int tail_tiles(int has_tail, int has_blk, int nbk, int cap0, int cap) {
+  if (!has_tail) return 0;
+  if (!has_blk || nbk <= cap0) return 1;
+  return 1 + (nbk - cap0 + cap - 1) / cap;
+}
 
 __device__ __forceinline__ Item decode_item(const TcParams &P, int id) {
   const AttnParams &A = P.a;
@@ -97,7 +116,15 @@ __device__ __forceinline__ Item decode_item(const TcParams &P, int id) {
   I.g = y;
   I.pair = x / P.nsplit;
   I.split = x % P.nsplit;
-  I.ntq = min(2, P.n_tiles - I.pair * 2);
+  int blk = 0;
+  while (blk + 1 < P.n_hblk && I.pair >= P.pair_start[blk + 1]) ++blk;
+  I.blk = blk;
+  I.hs = P.hb_log2[blk];
+  I.h0 = P.h0[blk];
+  I.ji_t = 128 >> I.hs;
+  const int pl = I.pair - P.pair_start[blk];
+  I.ntq = min(2, (P.n_ji + I.ji_t - 1) / I.ji_t - pl * 2);
+  I.ji0 = pl * 2 * I.ji_t;
   if (P.use_ctx_p) {
     I.c0 = P.ctx_off_p[I.n];
     I.L = P.ctx_len_p[I.n];
@@ -109,9 +136,10 @@ __device__ __forceinline__ Item decode_item(const TcParams &P, int id) {
   I.t0 = (int)((long long)I.split * I.nctx / P.nsplit);
   I.t1 = (int)((long long)(I.split + 1) * I.nctx / P.nsplit);
   I.n_ctx_it = I.t1 - I.t0;
-  I.do_tail = P.has_tail && I.split == P.nsplit - 1;
-  I.n_iter = I.n_ctx_it + (I.do_tail ? 1 : 0);
-  I.jb0 = A.lo + (I.pair * 2 * P.JI_T) / A.Bq;  // first boundary whose block keys sit in the tail tile
+  I.jb0 = A.lo + I.ji0 / A.Bq;  // first boundary whose block keys sit in the tail tiles
+  const int ji_last = min(I.ji0 + I.ntq * I.ji_t, P.n_ji) - 1;
+  I.n_tail = I.split == P.nsplit - 1 ? tail_tiles(P.has_tail, P.has_blk, ji_last / A.Bq - I.ji0 / A.Bq + 1, P.cap0, P.cap) : 0;
+  I.n_iter = I.n_ctx_it + I.n_tail;
   I.slot = ((I.n * A.Hkv + I.g) * P.n_pairs + I.pair) * P.nsplit + I.split;
   return I;
 }
@@ -168,7 +196,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
   if (warp == 8) {
     // ------------------------------------------------------------------ producer
     if (lane == 0) {
-      prefetch_tensormap(&P.map_q);
+      prefetch_tensormap(&P.map_q[0]);
     }
     int ld = 0, k = 0;  // running K/V load counter, processed-item counter
     bool ok = true;
@@ -180,11 +208,12 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
       ok = __all_sync(0xffffffffu, mbar_wait(q_empty, (k & 1) ^ 1u, abort_flag));
       if (!ok) break;
       if (lane == 0) {
-        const int qrow0 = (I.n * A.J + A.lo) * A.Bq + I.pair * 2 * P.JI_T;
-        mbar_arrive_expect_tx(q_full, (uint32_t)(I.ntq * P.JI_T * A.G * 128 * Cfg::kSlabs));
+        const int qrow0 = (I.n * A.J + A.lo) * A.Bq + I.ji0;
+        mbar_arrive_expect_tx(q_full, (uint32_t)(I.ntq * Cfg::kTileBytes));
         for (int t = 0; t < I.ntq; ++t)
           for (int sb = 0; sb < Cfg::kSlabs; ++sb)
-            tma_load_3d(sQ + t * Cfg::kTileBytes + sb * Cfg::kSlabBytes, &P.map_q, q_full, sb * 64, I.g * A.G, qrow0 + t * P.JI_T);
+            tma_load_3d(sQ + t * Cfg::kTileBytes + sb * Cfg::kSlabBytes, &P.map_q[I.blk], q_full, sb * 64, I.g * A.G + I.h0,
+                        qrow0 + t * I.ji_t);
       }
       // load order K0 K1 V0 K2 V1 ... K(n-1) V(n-2) V(n-1): the order the MMA issuer consumes them in
       // (the scores of iteration it + 1 are issued before the PV product of iteration it); slot = (ld + q) % kSlots
@@ -211,15 +240,23 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
             __syncwarp();
           }
           if (lane == 0) {
-            uint32_t bytes = 0;
-            if (A.S > 0) bytes += (uint32_t)A.S * 128 * Cfg::kSlabs;
-            if (P.has_blk) bytes += (uint32_t)P.R_blk * 128 * Cfg::kSlabs;
-            mbar_arrive_expect_tx(kv_full + sl, bytes);
-            for (int sb = 0; sb < Cfg::kSlabs; ++sb) {
-              if (A.S > 0) tma_load_3d(dst + sb * Cfg::kSlabBytes, is_v ? &P.map_vs : &P.map_ks, kv_full + sl, sb * 64, I.g, I.n * A.S);
-              if (P.has_blk)
-                tma_load_3d(dst + sb * Cfg::kSlabBytes + P.S8 * 128, is_v ? &P.map_vb : &P.map_kb, kv_full + sl, sb * 64, I.g,
-                            (I.n * A.J + I.jb0) * A.Bq);
+            const int tk = it - I.n_ctx_it;  // tail tile 0: spine rows, then cap0 blocks; tail tile k >= 1: cap blocks
+            if (tk == 0) {
+              uint32_t bytes = 0;
+              if (A.S > 0) bytes += (uint32_t)A.S * 128 * Cfg::kSlabs;
+              if (P.has_blk) bytes += (uint32_t)(P.cap0 * A.Bq) * 128 * Cfg::kSlabs;
+              mbar_arrive_expect_tx(kv_full + sl, bytes);
+              for (int sb = 0; sb < Cfg::kSlabs; ++sb) {
+                if (A.S > 0) tma_load_3d(dst + sb * Cfg::kSlabBytes, is_v ? &P.map_vs : &P.map_ks, kv_full + sl, sb * 64, I.g, I.n * A.S);
+                if (P.has_blk)
+                  tma_load_3d(dst + sb * Cfg::kSlabBytes + P.S8 * 128, is_v ? &P.map_vb0 : &P.map_kb0, kv_full + sl, sb * 64, I.g,
+                              (I.n * A.J + I.jb0) * A.Bq);
+              }
+            } else {
+              mbar_arrive_expect_tx(kv_full + sl, (uint32_t)(P.cap * A.Bq) * 128 * Cfg::kSlabs);
+              for (int sb = 0; sb < Cfg::kSlabs; ++sb)
+                tma_load_3d(dst + sb * Cfg::kSlabBytes, is_v ? &P.map_vb : &P.map_kb, kv_full + sl, sb * 64, I.g,
+                            (I.n * A.J + I.jb0 + P.cap0 + (tk - 1) * P.cap) * A.Bq);
             }
           }
         }
@@ -335,9 +372,9 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
     for (int qi = q_begin; qi < q_end && ok; qi += q_step) {
       const int id = P.use_sched ? (int)P.sched[qi] : qi;
       const Item I = decode_item(P, id);
-      const int ji = (I.pair * 2 + t) * P.JI_T + r / A.G;
-      const bool valid = (t < I.ntq) && (r < P.JI_T * A.G) && (ji < P.n_ji);
-      const int j = A.lo + ji / A.Bq, i = ji % A.Bq, h = I.g * A.G + r % A.G;
+      const int ji = I.ji0 + t * I.ji_t + (r >> I.hs);
+      const bool valid = (t < I.ntq) && (ji < P.n_ji);
+      const int j = A.lo + ji / A.Bq, i = ji % A.Bq, h = I.g * A.G + I.h0 + (r & ((1 << I.hs) - 1));
       const size_t orow = (((size_t)I.n * A.J + j) * A.Bq + i) * A.Hq + h;
       // split-KV: this CTA's partial rows go to an L2-resident scratch slot and are merged after a cluster barrier
       const size_t pslot = ((size_t)I.slot * 2 + t) * 128 + r;
@@ -355,11 +392,23 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
         continue;
       }
       const int n_iter = I.n_iter;
-      const int na = max(0, min(j + A.pb, A.S));
-      const int b0 = P.has_blk ? P.S8 + (j - I.jb0) * A.Bq : 0, b1 = P.has_blk ? b0 + A.Bq : 0;
+      const int jrel = j - I.jb0;  // this row's boundary, counted from the first one whose block sits in the tail tiles
       float m_used = -INFINITY, l = 0.f;
 
       for (int it = 0; it < n_iter; ++it) {
+        // tail tile tk: the anchor prefix sits in tile 0; this row's own block in tile kt at key rows [boff, boff + Bq)
+        // (worked out before the score row occupies the registers)
+        // The visible keys of the tile as a 128-bit mask (four words), so that masking a score is one bit test.
+        uint32_t vis[4] = {0u, 0u, 0u, 0u};
+        if (it >= I.n_ctx_it) {
+          const int tk = it - I.n_ctx_it;
+          const int kt = !P.has_blk ? -1 : (jrel < P.cap0 ? 0 : 1 + (jrel - P.cap0) / P.cap);
+          const int boff = jrel < P.cap0 ? P.S8 + jrel * A.Bq : ((jrel - P.cap0) % P.cap) * A.Bq;
+          const int na_t = tk == 0 ? max(0, min(I.jb0 + jrel + A.pb, A.S)) : 0;
+          const int b0 = tk == kt ? boff : 0, b1 = tk == kt ? boff + A.Bq : 0;
+#pragma unroll
+          for (int w = 0; w < 4; ++w) vis[w] = bits_below(na_t - 32 * w) | (bits_below(b1 - 32 * w) & ~bits_below(b0 - 32 * w));
+        }
         ok = __all_sync(0xffffffffu, mbar_wait(s_full + t, (cnt + it) & 1, abort_flag, 6));
         if (!ok) break;
         tc_fence_after();
@@ -377,7 +426,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
         for (int kx = 0; kx < 128; ++kx) s[kx] = __uint_as_float(su[kx]);
         if (it >= I.n_ctx_it) {
 #pragma unroll
-          for (int kx = 0; kx < 128; ++kx) s[kx] = ((kx < na) || (kx >= b0 && kx < b1)) ? s[kx] : -INFINITY;
+          for (int kx = 0; kx < 128; ++kx) s[kx] = ((vis[kx >> 5] >> (kx & 31)) & 1u) ? s[kx] : -INFINITY;
         } else if (it == I.n_ctx_it - 1 && I.t1 == I.nctx && (I.L & 127)) {
           const int nv = I.L & 127;
 #pragma unroll
@@ -516,9 +565,9 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
       for (int u = threadIdx.x; u < rows_per * kParts; u += 256) {
         const int R = (int)rank * rows_per + u % rows_per, part = u / rows_per;
         const int t = R >> 7, r = R & 127;
-        const int ji = (I.pair * 2 + t) * P.JI_T + r / A.G;
-        if (t >= I.ntq || r >= P.JI_T * A.G || ji >= P.n_ji) continue;
-        const int j = A.lo + ji / A.Bq, i = ji % A.Bq, h = I.g * A.G + r % A.G;
+        const int ji = I.ji0 + t * I.ji_t + (r >> I.hs);
+        if (t >= I.ntq || ji >= P.n_ji) continue;
+        const int j = A.lo + ji / A.Bq, i = ji % A.Bq, h = I.g * A.G + I.h0 + (r & ((1 << I.hs) - 1));
         const size_t orow = (((size_t)I.n * A.J + j) * A.Bq + i) * A.Hq + h;
         float2 ml[8];
 #pragma unroll
@@ -601,15 +650,25 @@ TcPlan plan_attention_tc(const dpara_shape *s, const int64_t *host_off) {
   const int G = s->n_q_heads / s->n_kv_heads;
   const int nb = s->boundary_hi - s->boundary_lo;
   if (nb <= 0) return p;
-  p.JI_T = 128 / G;
+  if (G > 16 || s->n_spine > 64 || s->block > 64) return p;
   p.n_ji = nb * s->block;
-  p.n_tiles = (p.n_ji + p.JI_T - 1) / p.JI_T;
-  p.n_pairs = (p.n_tiles + 1) / 2;
+  // head blocks = binary digits of G, widest first; block k's tiles hold 128 / hb (j, i) rows
+  p.n_hblk = 0;
+  p.n_pairs = 0;
+  for (int bit = 4, h0 = 0; bit >= 0; --bit) {
+    if (!(G & (1 << bit))) continue;
+    const int ji_t = 128 >> bit, tiles = (p.n_ji + ji_t - 1) / ji_t;
+    p.hb_log2[p.n_hblk] = bit;
+    p.h0[p.n_hblk] = h0;
+    p.pair_start[p.n_hblk] = p.n_pairs;
+    p.n_pairs += (tiles + 1) / 2;
+    h0 += 1 << bit;
+    ++p.n_hblk;
+  }
+  p.pair_start[p.n_hblk] = p.n_pairs;
   p.S8 = (s->n_spine + 7) & ~7;
-  int nbmax = (2 * p.JI_T - 1) / s->block + 2;
-  if (nbmax > nb) nbmax = nb;
-  p.R_blk = nbmax * s->block;
-  if (G > 16 || p.JI_T < 1 || p.JI_T > 256 || s->n_spine > 64 || p.R_blk > 256 || p.S8 + p.R_blk > 128) return p;
+  p.cap = 128 / s->block;
+  p.cap0 = (128 - p.S8) / s->block;  // >= 1: S8 <= 64 and block <= 64
   long long max_l = 0, tot = host_off[s->batch] - host_off[0];
   for (int n = 0; n < s->batch; ++n) max_l = (host_off[n + 1] - host_off[n]) > max_l ? (host_off[n + 1] - host_off[n]) : max_l;
   if (tot + 128 >= (1ll << 31) || (long long)s->batch * s->n_boundaries * s->block >= (1ll << 31)) return p;
@@ -664,8 +723,11 @@ dpara_status launch_attention_tc(const AttnParams &A, const TcPlan &plan, const 
   TcParams P;
   memset(&P, 0, sizeof(P));
   P.a = A;
-  P.JI_T = plan.JI_T; P.n_ji = plan.n_ji; P.n_tiles = plan.n_tiles; P.n_pairs = plan.n_pairs; P.nsplit = plan.nsplit;
-  P.S8 = plan.S8; P.R_blk = plan.R_blk; P.has_blk = A.k_blk != nullptr;
+  P.n_ji = plan.n_ji; P.n_pairs = plan.n_pairs; P.nsplit = plan.nsplit;
+  P.n_hblk = plan.n_hblk;
+  for (int k = 0; k < plan.n_hblk; ++k) { P.hb_log2[k] = plan.hb_log2[k]; P.h0[k] = plan.h0[k]; }
+  for (int k = 0; k <= plan.n_hblk; ++k) P.pair_start[k] = plan.pair_start[k];
+  P.S8 = plan.S8; P.cap0 = plan.cap0; P.cap = plan.cap; P.has_blk = A.k_blk != nullptr;
   P.has_tail = (A.S > 0) || P.has_blk;
   P.n_items = (int)(plan.items * plan.nsplit);
   P.c_log2 = A.scale * 1.4426950408889634f;
@@ -673,7 +735,9 @@ dpara_status launch_attention_tc(const AttnParams &A, const TcPlan &plan, const 
   const uint64_t rs = (uint64_t)D * 2;
   const long long tot = host_off[A.b] - host_off[0];
   const uint64_t nq = (uint64_t)A.b * A.J * A.Bq;
-  bool ok = make_tmap_bf16_3d(&P.map_q, A.q, D, A.Hq, nq, rs, rs * A.Hq, 64, A.G, plan.JI_T);
+  bool ok = true;
+  for (int k = 0; k < plan.n_hblk; ++k)
+    ok = ok && make_tmap_bf16_3d(&P.map_q[k], A.q, D, A.Hq, nq, rs, rs * A.Hq, 64, 1u << plan.hb_log2[k], 128u >> plan.hb_log2[k]);
   if (tot > 0) {
     ok = ok && make_tmap_bf16_3d(&P.map_kc, A.k_ctx, D, A.Hkv, host_off[A.b], rs, rs * A.Hkv, 64, 1, 128);
     ok = ok && make_tmap_bf16_3d(&P.map_vc, A.v_ctx, D, A.Hkv, host_off[A.b], rs, rs * A.Hkv, 64, 1, 128);
@@ -683,8 +747,10 @@ dpara_status launch_attention_tc(const AttnParams &A, const TcPlan &plan, const 
     ok = ok && make_tmap_bf16_3d(&P.map_vs, A.v_spine, D, A.Hkv, (uint64_t)A.b * A.S, rs, rs * A.Hkv, 64, 1, A.S);
   }
   if (P.has_blk) {
-    ok = ok && make_tmap_bf16_3d(&P.map_kb, A.k_blk, D, A.Hkv, nq, rs, rs * A.Hkv, 64, 1, plan.R_blk);
-    ok = ok && make_tmap_bf16_3d(&P.map_vb, A.v_blk, D, A.Hkv, nq, rs, rs * A.Hkv, 64, 1, plan.R_blk);
+    ok = ok && make_tmap_bf16_3d(&P.map_kb0, A.k_blk, D, A.Hkv, nq, rs, rs * A.Hkv, 64, 1, plan.cap0 * A.Bq);
+    ok = ok && make_tmap_bf16_3d(&P.map_vb0, A.v_blk, D, A.Hkv, nq, rs, rs * A.Hkv, 64, 1, plan.cap0 * A.Bq);
+    ok = ok && make_tmap_bf16_3d(&P.map_kb, A.k_blk, D, A.Hkv, nq, rs, rs * A.Hkv, 64, 1, plan.cap * A.Bq);
+    ok = ok && make_tmap_bf16_3d(&P.map_vb, A.v_blk, D, A.Hkv, nq, rs, rs * A.Hkv, 64, 1, plan.cap * A.Bq);
   }
   if (!ok) return DPARA_ERR_CUDA;
   P.use_ctx_p = A.b <= kMaxOrdered;
@@ -714,8 +780,12 @@ dpara_status launch_attention_tc(const AttnParams &A, const TcPlan &plan, const 
       const int z = id / per_req, x = id % X;
       const int n = P.use_order ? (int)P.req_order[z] : z;
       const long long L = host_off[n + 1] - host_off[n];
-      const int n_iter = (int)((L + 127) >> 7) + (P.has_tail ? 1 : 0);
-      const int ntq = std::min(2, plan.n_tiles - x * 2);
+      int blk = 0;
+      while (blk + 1 < plan.n_hblk && x >= plan.pair_start[blk + 1]) ++blk;
+      const int ji_t = 128 >> plan.hb_log2[blk], pl = x - plan.pair_start[blk];
+      const int ntq = std::min(2, (plan.n_ji + ji_t - 1) / ji_t - pl * 2);
+      const int ji0 = pl * 2 * ji_t, ji_last = std::min(ji0 + ntq * ji_t, plan.n_ji) - 1;
+      const int n_iter = (int)((L + 127) >> 7) + tail_tiles(P.has_tail, P.has_blk, ji_last / A.Bq - ji0 / A.Bq + 1, plan.cap0, plan.cap);
       cost[id] = {n_iter * (ntq == 2 ? 3300 : 2700) + 11000, id};
     }
     std::stable_sort(cost.begin(), cost.end(), [](const std::pair<int, int> &a, const std::pair<int, int> &b) { return a.first > b.first; });

@@ -6,10 +6,10 @@ namespace dpara {
 
 struct TcPlan {
   bool eligible;        // false: shape outside what the tensor-core kernel handles (use the general kernel)
-  int JI_T;             // (boundary, slot) rows per 128-row query tile = 128 / G
-  int n_ji, n_tiles, n_pairs;
+  int n_ji, n_pairs;    // (boundary, slot) rows per request; tile pairs per (request, KV head), all head blocks
+  int n_hblk, hb_log2[4], h0[4], pair_start[5];  // head blocks (binary digits of the group size) and their tile pairs
   int nsplit;           // KV splits per (request, KV head, tile pair)
-  int S8, R_blk;        // tail tile: block keys start at row S8 and span R_blk rows
+  int S8, cap0, cap;    // tail tiles: spine rows rounded up to 8; own blocks held by the first / by every later tail tile
   long long items;      // batch * Hkv * n_pairs
   size_t workspace_bytes;
 };

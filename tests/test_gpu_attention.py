@@ -66,6 +66,10 @@ def test_cfg1_tiny():
     W.AttnShape((0, 5), 4, 2, 64, 3, 2),                  # an empty context
     W.AttnShape((140,), 16, 1, 128, 3, 3),                # one KV head, group 16, odd block
     W.AttnShape((520,), 8, 2, 128, 16, 16, 1, 16),        # 16 boundaries x 16 slots
+    W.AttnShape((300, 130), 6, 2, 128, 6, 8),             # group size 3: head blocks 2 + 1
+    W.AttnShape((131, 64), 12, 2, 64, 16, 16),            # group size 6: 4 + 2, the 2-head block spans 3 tail tiles
+    W.AttnShape((257,), 7, 1, 128, 5, 7),                 # group size 7: 4 + 2 + 1, odd block
+    W.AttnShape((90, 140), 15, 1, 64, 9, 5),              # group size 15: four head blocks
 ])
 def test_shapes(shape):
     _compare(W.make_attn_inputs(shape, 77))
@@ -151,8 +155,8 @@ def test_cfg3_full_size_sampled_rows():
     assert np.isfinite(o).all()
 
 
-def test_general_shape_kernel():
-    """Shapes whose spine prefix and own blocks do not fit the tensor-core kernel's single tail tile
-    (roundup8(n_spine) + block rows of the boundaries a tile pair touches > 128) run on the general CUDA-core kernel."""
+def test_several_tail_tiles():
+    """Shapes whose spine prefix and own blocks do not fit one 128-key tail tile (roundup8(n_spine) + block rows of
+    the boundaries a tile pair touches > 128): the blocks spill into further tail tiles."""
     _compare(W.make_attn_inputs(W.AttnShape((70, 200), 4, 2, 64, 3, 64, 1, 64), 13))
     _compare(W.make_attn_inputs(W.AttnShape((33,), 8, 2, 128, 4, 48, 1, 40), 14), with_blk=True)
