@@ -45,6 +45,7 @@ constexpr float kRescaleLog2 = 8.0f;
 constexpr int kMaxOrdered = 128;
 constexpr int kMaxSched = 3072;  // items a host-built schedule can hold (kernel parameter space)
 constexpr int kMaxHeadBlocks = 4;  // G <= 16: at most four binary digits unless G == 16 (one block)
+constexpr int kMaxPairs = 256;     // 64 boundaries x 64 slots in tiles of 8 (j, i) rows = 512 tiles
 }  // namespace
 
 
@@ -54,6 +55,14 @@ struct TcParams {
   // head blocks: block k covers heads [h0[k], h0[k] + (1 << hb_log2[k])) of every group; its tiles hold
   // 128 >> hb_log2[k] (j, i) rows; its tile pairs are pair_start[k] .. pair_start[k + 1] - 1
   int n_hblk, hb_log2[kMaxHeadBlocks], h0[kMaxHeadBlocks], pair_start[kMaxHeadBlocks + 1];
+  // per tile pair, worked out on the host so that taking up an item costs a few loads, not a dozen divisions
+  struct PairInfo {
+    int16_t ji0;      // first (j, i) row
+    int16_t jb0_rel;  // first boundary whose block keys sit in the tail tiles, relative to boundary_lo
+    uint8_t blk, hs, h0, ntq, n_tail, pad[3];
+  } pair[kMaxPairs];
+  int nsplit_log2;
+
   // tail tiles: the first holds the spine (S8 = S rounded up to 8 rows) and cap0 blocks, the others cap blocks
   int n_ji, n_pairs, nsplit, S8, cap0, cap, has_blk, has_tail, n_items;
   float *part_o;   // split-KV partials [item slot][2][D / 4][128 rows] float4 (unnormalised rows; a warp's lanes are
@@ -100,6 +109,23 @@ struct Item {
 // The low k bits set (k <= 0: none, k >= 32: all).
 __device__ __forceinline__ uint32_t bits_below(int k) { return k <= 0 ? 0u : (k >= 32 ? 0xffffffffu : ((1u << k) - 1u)); }
 
+// 4 x 4 transpose of 16-byte pieces among the four lanes of a quad: on return x[v] of lane c is what lane v of the
+// quad held in x[c].
+__device__ __forceinline__ void quad_transpose(uint4 (&x)[4], int lane) {
+  auto swap_step = [&](int mask, uint4 &lo0, uint4 &lo1, uint4 &hi0, uint4 &hi1) {
+    // lanes with the mask bit clear send (hi0, hi1) and receive into them; the others send (lo0, lo1) and receive into them
+    const bool up = lane & mask;
+    uint4 a = up ? lo0 : hi0, b = up ? lo1 : hi1;
+    a.x = __shfl_xor_sync(0xffffffffu, a.x, mask); a.y = __shfl_xor_sync(0xffffffffu, a.y, mask);
+    a.z = __shfl_xor_sync(0xffffffffu, a.z, mask); a.w = __shfl_xor_sync(0xffffffffu, a.w, mask);
+    b.x = __shfl_xor_sync(0xffffffffu, b.x, mask); b.y = __shfl_xor_sync(0xffffffffu, b.y, mask);
+    b.z = __shfl_xor_sync(0xffffffffu, b.z, mask); b.w = __shfl_xor_sync(0xffffffffu, b.w, mask);
+    if (up) { lo0 = a; lo1 = b; } else { hi0 = a; hi1 = b; }
+  };
+  swap_step(2, x[0], x[1], x[2], x[3]);  // exchange the off-diagonal 2 x 2 blocks
+  swap_step(1, x[0], x[2], x[1], x[3]);  // transpose inside the 2 x 2 blocks
+}
+
 // Tail tiles a tile pair needs: its boundaries' own blocks, cap0 of them next to the spine in the first tile.
 __host__ __device__ __forceinline__ int tail_tiles(int has_tail, int has_blk, int nbk, int cap0, int cap) {
   if (!has_tail) return 0;
@@ -110,21 +136,20 @@ __host__ __device__ __forceinline__ int tail_tiles(int has_tail, int has_blk, in
 __device__ __forceinline__ Item decode_item(const TcParams &P, int id) {
   const AttnParams &A = P.a;
   Item I;
-  const int X = P.n_pairs * P.nsplit;
-  const int x = id % X, y = (id / X) % A.Hkv, z = id / (X * A.Hkv);
-  I.n = P.use_order ? (int)P.req_order[z] : z;
-  I.g = y;
-  I.pair = x / P.nsplit;
-  I.split = x % P.nsplit;
-  int blk = 0;
-  while (blk + 1 < P.n_hblk && I.pair >= P.pair_start[blk + 1]) ++blk;
-  I.blk = blk;
-  I.hs = P.hb_log2[blk];
-  I.h0 = P.h0[blk];
+  const unsigned X = (unsigned)(P.n_pairs << P.nsplit_log2);
+  const unsigned yz = (unsigned)id / X, x = (unsigned)id - yz * X;
+  const unsigned z = yz / (unsigned)A.Hkv;
+  I.g = (int)(yz - z * (unsigned)A.Hkv);
+  I.n = P.use_order ? (int)P.req_order[z] : (int)z;
+  I.pair = (int)(x >> P.nsplit_log2);
+  I.split = (int)(x & ((1u << P.nsplit_log2) - 1u));
+  const TcParams::PairInfo pi = P.pair[I.pair];
+  I.blk = pi.blk;
+  I.hs = pi.hs;
+  I.h0 = pi.h0;
   I.ji_t = 128 >> I.hs;
-  const int pl = I.pair - P.pair_start[blk];
-  I.ntq = min(2, (P.n_ji + I.ji_t - 1) / I.ji_t - pl * 2);
-  I.ji0 = pl * 2 * I.ji_t;
+  I.ntq = pi.ntq;
+  I.ji0 = pi.ji0;
   if (P.use_ctx_p) {
     I.c0 = P.ctx_off_p[I.n];
     I.L = P.ctx_len_p[I.n];
@@ -133,14 +158,13 @@ __device__ __forceinline__ Item decode_item(const TcParams &P, int id) {
     I.L = (int)(A.ctx_offsets[I.n + 1] - I.c0);
   }
   I.nctx = (I.L + 127) >> 7;
-  I.t0 = (int)((long long)I.split * I.nctx / P.nsplit);
-  I.t1 = (int)((long long)(I.split + 1) * I.nctx / P.nsplit);
+  I.t0 = (int)(((unsigned)I.split * (unsigned)I.nctx) >> P.nsplit_log2);  // nctx < 2^24, split < 8
+  I.t1 = (int)(((unsigned)(I.split + 1) * (unsigned)I.nctx) >> P.nsplit_log2);
   I.n_ctx_it = I.t1 - I.t0;
-  I.jb0 = A.lo + I.ji0 / A.Bq;  // first boundary whose block keys sit in the tail tiles
-  const int ji_last = min(I.ji0 + I.ntq * I.ji_t, P.n_ji) - 1;
-  I.n_tail = I.split == P.nsplit - 1 ? tail_tiles(P.has_tail, P.has_blk, ji_last / A.Bq - I.ji0 / A.Bq + 1, P.cap0, P.cap) : 0;
+  I.jb0 = A.lo + pi.jb0_rel;  // first boundary whose block keys sit in the tail tiles
+  I.n_tail = I.split == (1 << P.nsplit_log2) - 1 ? pi.n_tail : 0;
   I.n_iter = I.n_ctx_it + I.n_tail;
-  I.slot = ((I.n * A.Hkv + I.g) * P.n_pairs + I.pair) * P.nsplit + I.split;
+  I.slot = (((I.n * A.Hkv + I.g) * P.n_pairs + I.pair) << P.nsplit_log2) + I.split;
   return I;
 }
 
@@ -504,6 +528,11 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
       if (!ok) break;
       tc_fence_after();
       const float inv = l > 0.f ? 1.0f / l : 0.f;
+      // output rows of the four lanes of this thread's quad (all ones: no such row)
+      size_t qrow[4];
+#pragma unroll
+      for (int v = 0; v < 4; ++v)
+        qrow[v] = (size_t)__shfl_sync(0xffffffffu, valid ? (unsigned long long)orow : ~0ull, (lane & ~3) + v);
 #pragma unroll 1
       for (int cc = 0; cc < D / 32; ++cc) {
         uint32_t o[32];
@@ -522,17 +551,24 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
             for (int v = 0; v < 8; ++v)
               dst[v] = make_float4(__uint_as_float(o[4 * v]) * inv, __uint_as_float(o[4 * v + 1]) * inv,
                                    __uint_as_float(o[4 * v + 2]) * inv, __uint_as_float(o[4 * v + 3]) * inv);
-          } else {
-            uint4 *dst = reinterpret_cast<uint4 *>(static_cast<uint16_t *>(A.out) + orow * D + cc * 32);
-#pragma unroll
-            for (int v = 0; v < 4; ++v) {
-              uint32_t w[4];
-#pragma unroll
-              for (int e = 0; e < 4; ++e)
-                w[e] = pack_bf16(__uint_as_float(o[8 * v + 2 * e]) * inv, __uint_as_float(o[8 * v + 2 * e + 1]) * inv);
-              dst[v] = make_uint4(w[0], w[1], w[2], w[3]);
-            }
           }
+        }
+        if (P.nsplit == 1 && !A.out_f32) {
+          // bf16 output: the thread's 32 columns are four 16-byte pieces of its row.  Written as they are, one store
+          // instruction of a warp touches 32 rows (32 partial sectors).  The four lanes of a quad swap pieces (a 4 x 4
+          // transpose by two butterfly steps) so that store v of a quad is 64 contiguous bytes of row 4q + v.
+          uint4 x[4];
+#pragma unroll
+          for (int v = 0; v < 4; ++v)
+            x[v] = make_uint4(pack_bf16(__uint_as_float(o[8 * v]) * inv, __uint_as_float(o[8 * v + 1]) * inv),
+                              pack_bf16(__uint_as_float(o[8 * v + 2]) * inv, __uint_as_float(o[8 * v + 3]) * inv),
+                              pack_bf16(__uint_as_float(o[8 * v + 4]) * inv, __uint_as_float(o[8 * v + 5]) * inv),
+                              pack_bf16(__uint_as_float(o[8 * v + 6]) * inv, __uint_as_float(o[8 * v + 7]) * inv));
+          quad_transpose(x, lane);
+#pragma unroll
+          for (int v = 0; v < 4; ++v)
+            if (qrow[v] != ~size_t(0))
+              *reinterpret_cast<uint4 *>(static_cast<uint16_t *>(A.out) + qrow[v] * D + cc * 32 + (lane & 3) * 8) = x[v];
         }
       }
       tc_fence_before();  // the O_t reads above are ordered before this warp's next p_full arrive
@@ -728,8 +764,22 @@ dpara_status launch_attention_tc(const AttnParams &A, const TcPlan &plan, const 
   for (int k = 0; k < plan.n_hblk; ++k) { P.hb_log2[k] = plan.hb_log2[k]; P.h0[k] = plan.h0[k]; }
   for (int k = 0; k <= plan.n_hblk; ++k) P.pair_start[k] = plan.pair_start[k];
   P.S8 = plan.S8; P.cap0 = plan.cap0; P.cap = plan.cap; P.has_blk = A.k_blk != nullptr;
+  P.nsplit_log2 = plan.nsplit == 8 ? 3 : (plan.nsplit == 4 ? 2 : (plan.nsplit == 2 ? 1 : 0));
   P.has_tail = (A.S > 0) || P.has_blk;
   P.n_items = (int)(plan.items * plan.nsplit);
+  for (int x = 0; x < plan.n_pairs; ++x) {
+    int blk = 0;
+    while (blk + 1 < plan.n_hblk && x >= plan.pair_start[blk + 1]) ++blk;
+    const int ji_t = 128 >> plan.hb_log2[blk], pl = x - plan.pair_start[blk];
+    const int ntq = std::min(2, (plan.n_ji + ji_t - 1) / ji_t - pl * 2);
+    const int ji0 = pl * 2 * ji_t, ji_last = std::min(ji0 + ntq * ji_t, plan.n_ji) - 1;
+    TcParams::PairInfo &pi = P.pair[x];
+    pi.ji0 = (int16_t)ji0;
+    pi.jb0_rel = (int16_t)(ji0 / A.Bq);
+    pi.blk = (uint8_t)blk; pi.hs = (uint8_t)plan.hb_log2[blk]; pi.h0 = (uint8_t)plan.h0[blk]; pi.ntq = (uint8_t)ntq;
+    pi.n_tail = (uint8_t)tail_tiles(P.has_tail, P.has_blk, ji_last / A.Bq - ji0 / A.Bq + 1, plan.cap0, plan.cap);
+  }
+
   P.c_log2 = A.scale * 1.4426950408889634f;
   const int D = A.D;
   const uint64_t rs = (uint64_t)D * 2;
@@ -780,12 +830,8 @@ dpara_status launch_attention_tc(const AttnParams &A, const TcPlan &plan, const 
       const int z = id / per_req, x = id % X;
       const int n = P.use_order ? (int)P.req_order[z] : z;
       const long long L = host_off[n + 1] - host_off[n];
-      int blk = 0;
-      while (blk + 1 < plan.n_hblk && x >= plan.pair_start[blk + 1]) ++blk;
-      const int ji_t = 128 >> plan.hb_log2[blk], pl = x - plan.pair_start[blk];
-      const int ntq = std::min(2, (plan.n_ji + ji_t - 1) / ji_t - pl * 2);
-      const int ji0 = pl * 2 * ji_t, ji_last = std::min(ji0 + ntq * ji_t, plan.n_ji) - 1;
-      const int n_iter = (int)((L + 127) >> 7) + tail_tiles(P.has_tail, P.has_blk, ji_last / A.Bq - ji0 / A.Bq + 1, plan.cap0, plan.cap);
+      const int ntq = P.pair[x].ntq;
+      const int n_iter = (int)((L + 127) >> 7) + P.pair[x].n_tail;
       cost[id] = {n_iter * (ntq == 2 ? 3300 : 2700) + 11000, id};
     }
     std::stable_sort(cost.begin(), cost.end(), [](const std::pair<int, int> &a, const std::pair<int, int> &b) { return a.first > b.first; });
