@@ -14,5 +14,7 @@ verify    : accepted length, bonus token and branch selection (paper Sec. 2.1, A
 layer     : one drafter backbone block around the attention (paper Sec. 3.1 only lists a block's
             parts -- attention, MLP, norms; the block structure is this build's reading
             -- PARITY UNPINNED by the paper for the structure itself, pinned only piecewise).
+cache     : the feature-cache update of Alg. 1 (verified rows appended, rejected suffix dropped) as keys/values of
+            every drafter layer, row by row.
 """
-from . import attention, verify, layer  # noqa: F401
+from . import attention, verify, layer, cache  # noqa: F401

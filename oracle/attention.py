@@ -49,11 +49,19 @@ def softmax_attention(q: np.ndarray, k: np.ndarray, v: np.ndarray, scale: float)
     return o, (m + np.log(l))[:, 0]
 
 
+def context_rows(n: int, ctx_offsets, ctx_lens=None) -> Tuple[int, int]:
+    """Cache rows [lo, hi) that hold request n's context.  Packed layout (ctx_lens None): request n owns rows
+    ctx_offsets[n] .. ctx_offsets[n + 1].  Layout with slack for in-place appends: rows ctx_offsets[n] ..
+    ctx_offsets[n] + ctx_lens[n] are filled, whatever lies behind them is not part of the context."""
+    lo = int(ctx_offsets[n])
+    return lo, (int(ctx_offsets[n + 1]) if ctx_lens is None else lo + int(ctx_lens[n]))
+
+
 def visible_keys(n: int, j: int, g: int, k_ctx, v_ctx, ctx_offsets, k_spine, v_spine, k_blk, v_blk,
-                 prefix_base: int) -> Tuple[np.ndarray, np.ndarray]:
+                 prefix_base: int, ctx_lens=None) -> Tuple[np.ndarray, np.ndarray]:
     """Keys/values (float64) that boundary j of request n reads for KV head g, in the order
     context, anchor prefix, own block."""
-    lo, hi = int(ctx_offsets[n]), int(ctx_offsets[n + 1])
+    lo, hi = context_rows(n, ctx_offsets, ctx_lens)
     S = k_spine.shape[1]
     n_anchor = max(0, min(j + prefix_base, S))
     ks = [bf16_bits_to_f64(k_ctx[lo:hi, g]), bf16_bits_to_f64(k_spine[n, :n_anchor, g])]
@@ -66,7 +74,7 @@ def visible_keys(n: int, j: int, g: int, k_ctx, v_ctx, ctx_offsets, k_spine, v_s
 
 def draft_all_boundaries(q, k_ctx, v_ctx, ctx_offsets, k_spine, v_spine, k_blk, v_blk,
                          prefix_base: int = 1, scale: Optional[float] = None,
-                         boundary_lo: int = 0, boundary_hi: Optional[int] = None):
+                         boundary_lo: int = 0, boundary_hi: Optional[int] = None, ctx_lens=None):
     """Representations of every boundary in [boundary_lo, boundary_hi).
 
     q [b][J][Bq][Hq][D], k/v tensors as bf16 bit patterns (see workloads.AttnInputs); query head h
@@ -86,7 +94,7 @@ def draft_all_boundaries(q, k_ctx, v_ctx, ctx_offsets, k_spine, v_spine, k_blk, 
         for j in range(boundary_lo, boundary_hi):
             for g in range(Hkv):
                 keys, vals = visible_keys(n, j, g, k_ctx, v_ctx, ctx_offsets, k_spine, v_spine, k_blk, v_blk,
-                                          prefix_base)
+                                          prefix_base, ctx_lens)
                 for h in range(g * G, (g + 1) * G):
                     o, l = softmax_attention(bf16_bits_to_f64(q[n, j, :, h]), keys, vals, scale)
                     out[n, j, :, h] = o
@@ -110,7 +118,7 @@ def draft_rows(q, k_ctx, v_ctx, ctx_offsets, k_spine, v_spine, k_blk, v_blk,
     return np.stack(res) if res else np.zeros((0, D))
 
 
-def spine_rows(q_spine, k_ctx, v_ctx, ctx_offsets, k_spine, v_spine, scale: Optional[float] = None):
+def spine_rows(q_spine, k_ctx, v_ctx, ctx_offsets, k_spine, v_spine, scale: Optional[float] = None, ctx_lens=None):
     """The spine tokens as query rows (Sec. 3.2, Fig. 4: the anchors run causally among themselves and see the
     whole cached context): anchor a of request n attends the context and spine rows 0..a, itself included.
     q_spine [b][S][Hq][D], k_spine / v_spine [b][S][Hkv][D] (bf16 bit patterns).  Returns float64 [b][S][Hq][D].
@@ -122,7 +130,7 @@ def spine_rows(q_spine, k_ctx, v_ctx, ctx_offsets, k_spine, v_spine, scale: Opti
         scale = 1.0 / math.sqrt(D)
     out = np.zeros((b, S, Hq, D))
     for n in range(b):
-        lo, hi = int(ctx_offsets[n]), int(ctx_offsets[n + 1])
+        lo, hi = context_rows(n, ctx_offsets, ctx_lens)
         for a in range(S):
             for h in range(Hq):
                 g = h // G

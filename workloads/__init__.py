@@ -307,6 +307,48 @@ def make_head_inputs(shape: HeadShape, seed: int) -> HeadInputs:
     return HeadInputs(shape, reps, w_lm, ar_w, ar_e, bonus)
 
 
+@dataclass
+class CacheInputs:
+    """One round of the feature-cache update for `n_layers` drafter layers (caches laid out with slack)."""
+    row_start: np.ndarray    # [b] int64: first cache row of request n
+    capacity: np.ndarray     # [b] int64: rows request n owns
+    ctx_len: np.ndarray      # [b] int64: rows filled before the update
+    features: np.ndarray     # [b][J][F] bf16 bits: target features of t_0..t_d
+    accept_len: np.ndarray   # [b] int32
+    w_kv: list               # per layer [2 * Hkv * D][F] bf16 bits (rows = [keys | values])
+    norm_w: list             # per layer [F] bf16 bits
+    knorm_w: list            # per layer [D] bf16 bits
+    k_cache: list            # per layer [rows][Hkv][D] bf16 bits (filled part random, the rest a sentinel pattern)
+    v_cache: list
+
+
+def make_cache_inputs(ctx_lens: Sequence[int], n_rows: int, feat_dim: int, n_kv_heads: int, head_dim: int,
+                      n_layers: int, seed: int, accept_len: Optional[Sequence[int]] = None, slack: int = 0,
+                      weight_sigma: float = 0.02) -> CacheInputs:
+    """Caches with `n_rows + slack` spare rows per request behind the filled part; accepted lengths uniform in
+    [0, n_rows) unless given; unfilled rows hold the bit pattern 0x7FC1 (a NaN) so that a stray write or read shows."""
+    rng = np.random.Generator(np.random.Philox(seed ^ 0xCAC4E))
+    b = len(ctx_lens)
+    cap = np.asarray([int(L) + n_rows + slack for L in ctx_lens], dtype=np.int64)
+    start = np.zeros(b, dtype=np.int64)
+    start[1:] = np.cumsum(cap)[:-1]
+    rows = int(cap.sum())
+    feats = _normal_bf16(rng, (b, n_rows, feat_dim))
+    acc = (rng.integers(0, n_rows, size=b) if accept_len is None else np.asarray(accept_len)).astype(np.int32)
+    w_kv, g1, gk, kc, vc = [], [], [], [], []
+    for _ in range(n_layers):
+        w_kv.append(_normal_bf16(rng, (2 * n_kv_heads * head_dim, feat_dim), weight_sigma))
+        g1.append(f32_to_bf16_bits(1.0 + 0.1 * rng.standard_normal(feat_dim, dtype=np.float32)))
+        gk.append(f32_to_bf16_bits(1.0 + 0.1 * rng.standard_normal(head_dim, dtype=np.float32)))
+        k = np.full((rows, n_kv_heads, head_dim), 0x7FC1, np.uint16)
+        v = np.full((rows, n_kv_heads, head_dim), 0x7FC1, np.uint16)
+        for n, L in enumerate(ctx_lens):
+            k[start[n]:start[n] + L] = _normal_bf16(rng, (int(L), n_kv_heads, head_dim))
+            v[start[n]:start[n] + L] = _normal_bf16(rng, (int(L), n_kv_heads, head_dim))
+        kc.append(k); vc.append(v)
+    return CacheInputs(start, cap, np.asarray(ctx_lens, dtype=np.int64), feats, acc, w_kv, g1, gk, kc, vc)
+
+
 def scaled(w: Workload, **kw) -> Workload:
     """A smaller variant of a named workload (same structure) for tests; kw override AttnShape/VerifyShape fields."""
     a = w.attn
