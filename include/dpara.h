@@ -54,6 +54,7 @@ typedef enum {
 /* bits OR-ed into *status_word by kernels */
 #define DPARA_STATUS_BAD_TOKEN 1u /* a draft token outside [0, vocab): rejected at that position */
 #define DPARA_STATUS_TIMEOUT 2u   /* a bounded device-side wait gave up; outputs of that tile are undefined */
+#define DPARA_STATUS_CACHE_FULL 4u /* dpara_cache_append: a request's new rows did not fit its cache; it was left as it was */
 
 typedef enum { DPARA_BF16 = 0, DPARA_F32 = 1 } dpara_dtype;
 
@@ -87,6 +88,12 @@ typedef struct {
   void *out;                       /* [b][J][Bq][Hq][D], dtype out_dtype; rows of boundaries outside [lo,hi) untouched */
   int32_t out_dtype;               /* dpara_dtype */
   float *out_lse;                  /* optional [b][J][Bq][Hq]: natural-log sum-exp of the scaled scores (NULL ok) */
+  /* Caches kept with slack for in-place appends (dpara_cache_append): both NULL = packed (request n's context is all
+   * of rows ctx_offsets[n]..ctx_offsets[n+1)); both given = only the first ctx_lens[n] of those rows are context.
+   * The unused rows must hold finite numbers (clear the cache once when it is allocated): the last, part-filled key
+   * tile of a request carries them through the tensor core with weight exactly 0, and 0 x NaN is NaN. */
+  const int64_t *ctx_lens;         /* [b] device */
+  const int64_t *host_ctx_lens;    /* [b] HOST copy of the same values */
 } dpara_attn_io;
 
 /* Full-layer mode (one pre-norm backbone block; Sec. 3.1 lists the block's trainable parts without giving
@@ -109,7 +116,8 @@ typedef struct {
 
 /* Bytes of scratch dpara_draft_all_boundaries needs for these shapes (0 is possible).
  * host_ctx_offsets: [b+1] host array.  full_layer != 0: include the block's intermediates
- * (hidden/intermediate are taken from `layer`, which may be NULL when full_layer == 0). */
+ * (hidden/intermediate are taken from `layer`, which may be NULL when full_layer == 0).  The figure is an upper bound
+ * over all context lengths that fit the offsets, so one workspace serves a cache that grows in place. */
 size_t dpara_draft_workspace_bytes(const dpara_shape *shape, const int64_t *host_ctx_offsets,
                                    const dpara_layer_io *layer, int full_layer);
 
@@ -242,6 +250,42 @@ typedef struct {
 } dpara_head_io;
 size_t dpara_head_workspace_bytes(int32_t b, int32_t block, int32_t vocab);
 dpara_status dpara_draft_head(const dpara_head_io *io, void *workspace, size_t workspace_bytes, int32_t *status_word, void *stream);
+
+/* Feature-cache update (Alg. 1, the line after the head loop: the verified features of t_0..t_r are appended to the
+ * cache and the rejected drafts t_{r+1..d} dropped; Sec. 3.3 states it in words; App. D, single-GPU paragraph: history
+ * features are projected incrementally).  The drafter layers read the cache as keys and values; this call projects the
+ * new rows for every layer and appends them in place.  Reading of the projection (the paper gives no equations), per
+ * layer l and feature row c at position p:  cn = bf16(rmsnorm(c) g_l);  [k | v] = bf16(cn Wkv_l^T);
+ * k = bf16(rmsnorm_over_D(k) gk_l) when knorm is given;  k = bf16(rope(k, p)) (rotate-half) when use_rope.
+ * Cache layout: request n owns rows [row_start[n], row_start[n] + capacity[n]) of every layer's k/v tensor
+ * ([rows][Hkv][D] bf16); the first ctx_len[n] are filled.  The call writes the r_n + 1 rows of t_0..t_{r_n}
+ * (r_n = accept_len[n], read on the device: queue this call behind dpara_verify_select) at rows
+ * row_start[n] + ctx_len[n] + i, positions ctx_len[n] + i, then adds r_n + 1 to ctx_len[n].  A request whose rows do not
+ * fit (or whose accept_len is outside [0, n_rows)) is left untouched and DPARA_STATUS_CACHE_FULL is OR-ed into
+ * *status_word.  The draft call reads such a cache through dpara_attn_io.ctx_lens.
+ *   features      device [b][n_rows][feat_dim] bf16: target features of t_0..t_d from the verification forward
+ *   host_*        HOST arrays of n_layers DEVICE pointers: w_kv [2 Hkv D][feat_dim] bf16 (rows = keys, then values),
+ *                 norm_w [feat_dim] and knorm_w [D] bf16 gains (array or entries may be NULL), k_ctx / v_ctx caches
+ *   row_start, capacity   device [b] int64;   ctx_len   device [b] int64, in/out
+ * Workspace: dpara_cache_append_workspace_bytes(), 16-byte aligned, private to the call while it runs.
+ * Errors: INVALID_ARG, UNSUPPORTED (head_dim not 64/128, feat_dim % 64 != 0), WORKSPACE, CUDA. */
+typedef struct {
+  int32_t batch, n_rows, feat_dim, n_kv_heads, head_dim, n_layers;
+  const void *features;
+  const int32_t *accept_len;
+  const void *const *host_w_kv;
+  const void *const *host_norm_w;
+  const void *const *host_knorm_w;
+  void *const *host_k_ctx;
+  void *const *host_v_ctx;
+  const int64_t *row_start;
+  const int64_t *capacity;
+  int64_t *ctx_len;
+  float rms_eps, rope_theta;
+  int32_t use_rope;
+} dpara_cache_io;
+size_t dpara_cache_append_workspace_bytes(const dpara_cache_io *io);
+dpara_status dpara_cache_append(const dpara_cache_io *io, void *workspace, size_t workspace_bytes, int32_t *status_word, void *stream);
 
 const char *dpara_status_string(dpara_status s);
 

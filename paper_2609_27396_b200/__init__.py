@@ -24,7 +24,7 @@ lib = C.CDLL(LIB_PATH)
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_STATIC_LIMIT = 0, -1, -2, -3, -4, -5, -6
 VERIFY_STATIC_SCRATCH_BYTES = 256 * 1024
-STATUS_BAD_TOKEN, STATUS_TIMEOUT = 1, 2
+STATUS_BAD_TOKEN, STATUS_TIMEOUT, STATUS_CACHE_FULL = 1, 2, 4
 BF16, F32 = 0, 1
 
 
@@ -38,7 +38,7 @@ class AttnIO(C.Structure):
     _fields_ = [("q", C.c_void_p), ("k_ctx", C.c_void_p), ("v_ctx", C.c_void_p), ("ctx_offsets", C.c_void_p),
                 ("host_ctx_offsets", C.c_void_p), ("k_spine", C.c_void_p), ("v_spine", C.c_void_p),
                 ("k_blk", C.c_void_p), ("v_blk", C.c_void_p), ("out", C.c_void_p), ("out_dtype", C.c_int32),
-                ("out_lse", C.c_void_p)]
+                ("out_lse", C.c_void_p), ("ctx_lens", C.c_void_p), ("host_ctx_lens", C.c_void_p)]
 
 
 class LayerIO(C.Structure):
@@ -151,7 +151,9 @@ class DraftPlan:
     def __init__(self, *, ctx_offsets: Sequence[int], n_boundaries: int, block: int, n_q_heads: int, n_kv_heads: int,
                  head_dim: int, prefix_base: int = 1, n_spine: Optional[int] = None, boundary_lo: int = 0,
                  boundary_hi: Optional[int] = None, softmax_scale: float = 0.0, layer: Optional[LayerIO] = None,
-                 device="cuda"):
+                 ctx_lens: Optional[Sequence[int]] = None, device="cuda"):
+        """ctx_lens: for caches kept with slack (dpara_cache_append) -- request n's context is the first ctx_lens[n] of
+        its rows ctx_offsets[n]..ctx_offsets[n+1]; update it between calls with set_ctx_lens()."""
         b = len(ctx_offsets) - 1
         self.shape = Shape(b, n_boundaries, block, n_q_heads, n_kv_heads, head_dim, prefix_base,
                            n_boundaries if n_spine is None else n_spine, boundary_lo,
@@ -164,12 +166,27 @@ class DraftPlan:
         self.workspace_bytes = int(need)
         self.workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=device)
         self.status = torch.zeros(1, dtype=torch.int32, device=device)
+        self.host_lens = self.dev_lens = None
+        if ctx_lens is not None:
+            self.host_lens = (C.c_int64 * b)(*[int(x) for x in ctx_lens])
+            self.dev_lens = torch.tensor([int(x) for x in ctx_lens], dtype=torch.int64, device=device)
+
+    def set_ctx_lens(self, ctx_lens: Sequence[int], dev_lens: Optional[torch.Tensor] = None) -> None:
+        """New context lengths (host values; `dev_lens`: a device tensor that already holds them, e.g. the one
+        dpara_cache_append updated, else they are copied to the device here)."""
+        for n, x in enumerate(ctx_lens):
+            self.host_lens[n] = int(x)
+        if dev_lens is not None:
+            self.dev_lens = dev_lens
+        else:
+            self.dev_lens.copy_(torch.tensor([int(x) for x in ctx_lens], dtype=torch.int64))
 
     def __call__(self, *, q=None, k_ctx=None, v_ctx=None, k_spine=None, v_spine=None, k_blk=None, v_blk=None,
                  out=None, out_lse=None, stream=None) -> None:
         io = AttnIO(_ptr(q), _ptr(k_ctx), _ptr(v_ctx), self.dev_off.data_ptr(), C.cast(self.host_off, C.c_void_p).value,
                     _ptr(k_spine), _ptr(v_spine), _ptr(k_blk), _ptr(v_blk), _ptr(out),
-                    F32 if (out is not None and out.dtype == torch.float32) else BF16, _ptr(out_lse))
+                    F32 if (out is not None and out.dtype == torch.float32) else BF16, _ptr(out_lse),
+                    _ptr(self.dev_lens), C.cast(self.host_lens, C.c_void_p).value if self.host_lens is not None else None)
         rc = lib.dpara_draft_all_boundaries(C.byref(self.shape), C.byref(io),
                                             C.byref(self.layer) if self.layer is not None else None,
                                             self.workspace.data_ptr(), self.workspace.numel(), self.status.data_ptr(),
@@ -328,3 +345,48 @@ def draft_head(sel_reps, w_lm, ar_w, ar_e, bonus, stream=None):
     plan = HeadPlan(b, block, hidden, w_lm.shape[0], ar_w.shape[1], sel_reps.device)
     plan.run(sel_reps, w_lm, ar_w, ar_e, bonus, stream)
     return plan.next_tokens, plan
+
+
+# ----------------------------------------------------------------------------- feature-cache append
+class CacheIO(C.Structure):
+    _fields_ = [("batch", C.c_int32), ("n_rows", C.c_int32), ("feat_dim", C.c_int32), ("n_kv_heads", C.c_int32),
+                ("head_dim", C.c_int32), ("n_layers", C.c_int32), ("features", C.c_void_p), ("accept_len", C.c_void_p),
+                ("host_w_kv", C.c_void_p), ("host_norm_w", C.c_void_p), ("host_knorm_w", C.c_void_p),
+                ("host_k_ctx", C.c_void_p), ("host_v_ctx", C.c_void_p), ("row_start", C.c_void_p), ("capacity", C.c_void_p),
+                ("ctx_len", C.c_void_p), ("rms_eps", C.c_float), ("rope_theta", C.c_float), ("use_rope", C.c_int32)]
+
+
+lib.dpara_cache_append_workspace_bytes.restype = C.c_size_t
+lib.dpara_cache_append_workspace_bytes.argtypes = [C.POINTER(CacheIO)]
+lib.dpara_cache_append.restype = C.c_int
+lib.dpara_cache_append.argtypes = [C.POINTER(CacheIO), C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
+EXPORTED += ["dpara_cache_append_workspace_bytes", "dpara_cache_append"]
+
+
+class CachePlan:
+    """dpara_cache_append for fixed shapes and fixed per-layer tensors (weights, caches): pointer tables, workspace and
+    status word are set up once; run() allocates nothing."""
+
+    def __init__(self, *, batch: int, n_rows: int, w_kv: Sequence[torch.Tensor], k_ctx: Sequence[torch.Tensor],
+                 v_ctx: Sequence[torch.Tensor], row_start: torch.Tensor, capacity: torch.Tensor, ctx_len: torch.Tensor,
+                 norm_w: Optional[Sequence[torch.Tensor]] = None, knorm_w: Optional[Sequence[torch.Tensor]] = None,
+                 rms_eps: float = 1e-6, rope_theta: float = 1e6, use_rope: bool = True):
+        n_layers = len(w_kv)
+        Hkv, D = k_ctx[0].shape[1], k_ctx[0].shape[2]
+        self._keep = (list(w_kv), list(k_ctx), list(v_ctx), row_start, capacity, ctx_len, norm_w, knorm_w)
+        table = lambda ts: (C.c_void_p * n_layers)(*[_ptr(t) for t in ts]) if ts is not None else None
+        self._tabs = [table(w_kv), table(norm_w), table(knorm_w), table(k_ctx), table(v_ctx)]
+        cast = lambda t: C.cast(t, C.c_void_p).value if t is not None else None
+        self.io = CacheIO(batch, n_rows, w_kv[0].shape[1], Hkv, D, n_layers, None, None, *[cast(t) for t in self._tabs],
+                          _ptr(row_start), _ptr(capacity), _ptr(ctx_len), rms_eps, rope_theta, 1 if use_rope else 0)
+        self.workspace_bytes = int(lib.dpara_cache_append_workspace_bytes(C.byref(self.io)))
+        self.workspace = torch.empty(max(self.workspace_bytes, 16), dtype=torch.uint8, device=ctx_len.device)
+        self.status = torch.zeros(1, dtype=torch.int32, device=ctx_len.device)
+        self.ctx_len = ctx_len
+
+    def run(self, features: torch.Tensor, accept_len: torch.Tensor, stream=None) -> None:
+        self.io.features, self.io.accept_len = _ptr(features), _ptr(accept_len)
+        rc = lib.dpara_cache_append(C.byref(self.io), self.workspace.data_ptr(), self.workspace.numel(), self.status.data_ptr(),
+                                    _stream_ptr(stream))
+        if rc != OK:
+            raise DparaError(rc)

@@ -65,6 +65,10 @@ extern "C" dpara_status dpara_draft_all_boundaries(const dpara_shape *shape, con
   s = validate_offsets(shape, io->host_ctx_offsets);
   if (s != DPARA_OK) return s;
   if (!io->ctx_offsets) return DPARA_ERR_INVALID_ARG;
+  if ((io->ctx_lens == nullptr) != (io->host_ctx_lens == nullptr)) return DPARA_ERR_INVALID_ARG;
+  if (io->host_ctx_lens)
+    for (int n = 0; n < shape->batch; ++n)
+      if (io->host_ctx_lens[n] < 0 || io->host_ctx_lens[n] > io->host_ctx_offsets[n + 1] - io->host_ctx_offsets[n]) return DPARA_ERR_INVALID_ARG;
   const bool has_ctx = io->host_ctx_offsets[shape->batch] > 0;
   if (has_ctx && (!io->k_ctx || !io->v_ctx)) return DPARA_ERR_INVALID_ARG;
   if (shape->n_spine > 0 && (!io->k_spine || !io->v_spine)) return DPARA_ERR_INVALID_ARG;

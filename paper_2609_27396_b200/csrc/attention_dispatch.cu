@@ -11,6 +11,7 @@ void fill_attn_params(AttnParams &P, const dpara_shape *s, const dpara_attn_io *
   P.k_ctx = static_cast<const uint16_t *>(io->k_ctx);
   P.v_ctx = static_cast<const uint16_t *>(io->v_ctx);
   P.ctx_offsets = io->ctx_offsets;
+  P.ctx_lens = io->ctx_lens;
   P.k_spine = static_cast<const uint16_t *>(io->k_spine);
   P.v_spine = static_cast<const uint16_t *>(io->v_spine);
   P.k_blk = static_cast<const uint16_t *>(io->k_blk);
@@ -26,8 +27,8 @@ void fill_attn_params(AttnParams &P, const dpara_shape *s, const dpara_attn_io *
 }
 
 size_t attention_workspace_bytes(const dpara_shape *shape, const int64_t *host_off) {
-  TcPlan plan = plan_attention_tc(shape, host_off);
-  return plan.eligible ? align_up(plan.workspace_bytes, 256) : 0;
+  TcPlan plan = plan_attention_tc(shape, host_off, nullptr);
+  return plan.eligible ? align_up(plan.workspace_max_bytes, 256) : 0;
 }
 
 dpara_status launch_attention(const dpara_shape *shape, const dpara_attn_io *io, void *workspace, int32_t *status_word,
@@ -35,9 +36,9 @@ dpara_status launch_attention(const dpara_shape *shape, const dpara_attn_io *io,
   AttnParams P;
   fill_attn_params(P, shape, io, status_word);
   if (P.hi <= P.lo) return DPARA_OK;
-  TcPlan plan = plan_attention_tc(shape, io->host_ctx_offsets);
+  TcPlan plan = plan_attention_tc(shape, io->host_ctx_offsets, io->host_ctx_lens);
   if (!plan.eligible) return DPARA_ERR_UNSUPPORTED;  // group size > 16, block > 64, spine > 64, or more than 2^31 rows
-  return launch_attention_tc(P, plan, io->host_ctx_offsets, workspace, st);
+  return launch_attention_tc(P, plan, io->host_ctx_offsets, io->host_ctx_lens, workspace, st);
 }
 
 }  // namespace dpara

@@ -155,7 +155,7 @@ __device__ __forceinline__ Item decode_item(const TcParams &P, int id) {
     I.L = P.ctx_len_p[I.n];
   } else {
     I.c0 = A.ctx_offsets[I.n];
-    I.L = (int)(A.ctx_offsets[I.n + 1] - I.c0);
+    I.L = (int)(A.ctx_lens ? A.ctx_lens[I.n] : A.ctx_offsets[I.n + 1] - I.c0);
   }
   I.nctx = (I.L + 127) >> 7;
   I.t0 = (int)(((unsigned)I.split * (unsigned)I.nctx) >> P.nsplit_log2);  // nctx < 2^24, split < 8
@@ -681,7 +681,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
 }
 
 // ------------------------------------------------------------------------------------------------ host
-TcPlan plan_attention_tc(const dpara_shape *s, const int64_t *host_off) {
+TcPlan plan_attention_tc(const dpara_shape *s, const int64_t *host_off, const int64_t *host_lens) {
+  auto len_of = [&](int n) { return host_lens ? host_lens[n] : host_off[n + 1] - host_off[n]; };
   TcPlan p{};
   const int G = s->n_q_heads / s->n_kv_heads;
   const int nb = s->boundary_hi - s->boundary_lo;
@@ -706,7 +707,7 @@ TcPlan plan_attention_tc(const dpara_shape *s, const int64_t *host_off) {
   p.cap = 128 / s->block;
   p.cap0 = (128 - p.S8) / s->block;  // >= 1: S8 <= 64 and block <= 64
   long long max_l = 0, tot = host_off[s->batch] - host_off[0];
-  for (int n = 0; n < s->batch; ++n) max_l = (host_off[n + 1] - host_off[n]) > max_l ? (host_off[n + 1] - host_off[n]) : max_l;
+  for (int n = 0; n < s->batch; ++n) max_l = len_of(n) > max_l ? len_of(n) : max_l;
   if (tot + 128 >= (1ll << 31) || (long long)s->batch * s->n_boundaries * s->block >= (1ll << 31)) return p;
   const long long items = (long long)s->batch * s->n_kv_heads * p.n_pairs;
   const int max_tiles = (int)((max_l + 127) / 128);
@@ -720,6 +721,7 @@ TcPlan plan_attention_tc(const dpara_shape *s, const int64_t *host_off) {
   p.nsplit = nsplit;
   p.items = items;
   p.workspace_bytes = nsplit > 1 ? (size_t)items * nsplit * 256 * ((size_t)s->head_dim + 2) * 4 : 0;
+  p.workspace_max_bytes = items < 96 ? (size_t)items * 8 * 256 * ((size_t)s->head_dim + 2) * 4 : 0;
   p.eligible = true;
   return p;
 }
@@ -755,7 +757,9 @@ static dpara_status launch_tc_d(const TcParams &P, const TcPlan &plan, cudaStrea
   return DPARA_OK;
 }
 
-dpara_status launch_attention_tc(const AttnParams &A, const TcPlan &plan, const int64_t *host_off, void *workspace, cudaStream_t st) {
+dpara_status launch_attention_tc(const AttnParams &A, const TcPlan &plan, const int64_t *host_off, const int64_t *host_lens,
+                                 void *workspace, cudaStream_t st) {
+  auto len_of = [&](int n) { return host_lens ? host_lens[n] : host_off[n + 1] - host_off[n]; };
   TcParams P;
   memset(&P, 0, sizeof(P));
   P.a = A;
@@ -805,16 +809,16 @@ dpara_status launch_attention_tc(const AttnParams &A, const TcPlan &plan, const 
   if (!ok) return DPARA_ERR_CUDA;
   P.use_ctx_p = A.b <= kMaxOrdered;
   if (P.use_ctx_p)
-    for (int n = 0; n < A.b; ++n) { P.ctx_off_p[n] = host_off[n]; P.ctx_len_p[n] = (int)(host_off[n + 1] - host_off[n]); }
+    for (int n = 0; n < A.b; ++n) { P.ctx_off_p[n] = host_off[n]; P.ctx_len_p[n] = (int)len_of(n); }
   P.use_order = A.b <= kMaxOrdered && A.b > 1;
   if (P.use_order) {
     int idx[kMaxOrdered];
     for (int n = 0; n < A.b; ++n) idx[n] = n;
     for (int a = 1; a < A.b; ++a) {  // insertion sort by decreasing length (stable)
       const int v = idx[a];
-      const long long lv = host_off[v + 1] - host_off[v];
+      const long long lv = len_of(v);
       int c = a - 1;
-      while (c >= 0 && host_off[idx[c] + 1] - host_off[idx[c]] < lv) { idx[c + 1] = idx[c]; --c; }
+      while (c >= 0 && len_of(idx[c]) < lv) { idx[c + 1] = idx[c]; --c; }
       idx[c + 1] = v;
     }
     for (int n = 0; n < A.b; ++n) P.req_order[n] = (uint8_t)idx[n];
@@ -829,7 +833,7 @@ dpara_status launch_attention_tc(const AttnParams &A, const TcPlan &plan, const 
     for (int id = 0; id < P.n_items; ++id) {
       const int z = id / per_req, x = id % X;
       const int n = P.use_order ? (int)P.req_order[z] : z;
-      const long long L = host_off[n + 1] - host_off[n];
+      const long long L = len_of(n);
       const int ntq = P.pair[x].ntq;
       const int n_iter = (int)((L + 127) >> 7) + P.pair[x].n_tail;
       cost[id] = {n_iter * (ntq == 2 ? 3300 : 2700) + 11000, id};

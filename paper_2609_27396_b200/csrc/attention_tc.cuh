@@ -11,11 +11,13 @@ struct TcPlan {
   int nsplit;           // KV splits per (request, KV head, tile pair)
   int S8, cap0, cap;    // tail tiles: spine rows rounded up to 8; own blocks held by the first / by every later tail tile
   long long items;      // batch * Hkv * n_pairs
-  size_t workspace_bytes;
+  size_t workspace_bytes;      // split-KV scratch this launch uses
+  size_t workspace_max_bytes;  // ... and the most any context lengths within the same offsets can need
 };
 
-TcPlan plan_attention_tc(const dpara_shape *s, const int64_t *host_ctx_offsets);
-dpara_status launch_attention_tc(const AttnParams &A, const TcPlan &plan, const int64_t *host_ctx_offsets, void *workspace,
-                                 cudaStream_t st);
+// host_ctx_lens may be null (request n fills rows host_ctx_offsets[n] .. host_ctx_offsets[n + 1])
+TcPlan plan_attention_tc(const dpara_shape *s, const int64_t *host_ctx_offsets, const int64_t *host_ctx_lens);
+dpara_status launch_attention_tc(const AttnParams &A, const TcPlan &plan, const int64_t *host_ctx_offsets,
+                                 const int64_t *host_ctx_lens, void *workspace, cudaStream_t st);
 
 }  // namespace dpara

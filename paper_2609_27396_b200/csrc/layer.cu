@@ -79,7 +79,7 @@ struct QkParams {
   const uint16_t *qkv;
   const uint16_t *qnorm_w, *knorm_w;
   uint16_t *q, *k, *v;
-  const int64_t *ctx_offsets;
+  const int64_t *ctx_offsets, *ctx_lens;
   int J, Bq, Hq, Hkv, D;
   int use_rope, use_norm;
   float eps, theta;
@@ -91,7 +91,7 @@ __global__ void __launch_bounds__(128) qk_norm_rope_kernel(const QkParams P) {
   const int half = P.D / 2;
   const int i = row % P.Bq, j = (row / P.Bq) % P.J, n = row / (P.Bq * P.J);
   if (P.use_rope) {
-    const double pos = (double)(P.ctx_offsets[n + 1] - P.ctx_offsets[n]) + j + 2 + i;
+    const double pos = (double)(P.ctx_lens ? P.ctx_lens[n] : P.ctx_offsets[n + 1] - P.ctx_offsets[n]) + j + 2 + i;
     for (int d = tid; d < half; d += 128) {
       const double inv = pow((double)P.theta, -2.0 * d / P.D);
       double sn, cs;
@@ -179,6 +179,14 @@ void layer_workspace_offsets(const dpara_shape *shape, const dpara_layer_io *lay
   for (int i = 0; i < 9; ++i) out[i] = attn_bytes + o[i];
 }
 
+dpara_status launch_rmsnorm_bf16(const void *x, const void *gain, void *out, int M, int H, float eps, cudaStream_t st) {
+  if (H % 8) return DPARA_ERR_UNSUPPORTED;
+  rmsnorm_kernel<false><<<M, 128, 0, st>>>(x, static_cast<const uint16_t *>(gain), static_cast<uint16_t *>(out), H, eps);
+  DPARA_CHECK_LAUNCH();
+  count_launches(1);
+  return DPARA_OK;
+}
+
 size_t layer_workspace_bytes(const dpara_shape *shape, const dpara_layer_io *layer) {
   if (layer->hidden <= 0 || layer->intermediate <= 0) return 0;
   return layer_ws_layout(shape, layer, 0).total;  // the attention's own scratch is added by the caller
@@ -214,7 +222,7 @@ dpara_status launch_layer(const dpara_shape *shape, const dpara_attn_io *io, con
 
   QkParams qp;
   qp.qkv = qkv; qp.qnorm_w = static_cast<const uint16_t *>(L->qnorm_w); qp.knorm_w = static_cast<const uint16_t *>(L->knorm_w);
-  qp.q = q; qp.k = k; qp.v = v; qp.ctx_offsets = io->ctx_offsets;
+  qp.q = q; qp.k = k; qp.v = v; qp.ctx_offsets = io->ctx_offsets; qp.ctx_lens = io->ctx_lens;
   qp.J = shape->n_boundaries; qp.Bq = shape->block; qp.Hq = shape->n_q_heads; qp.Hkv = shape->n_kv_heads; qp.D = D;
   qp.use_rope = L->use_rope; qp.use_norm = L->qnorm_w != nullptr; qp.eps = L->rms_eps; qp.theta = L->rope_theta;
   qk_norm_rope_kernel<<<M, 128, D * sizeof(float), st>>>(qp);

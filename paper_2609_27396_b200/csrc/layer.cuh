@@ -9,6 +9,9 @@ size_t attention_workspace_bytes(const dpara_shape *shape, const int64_t *host_c
 dpara_status launch_attention(const dpara_shape *shape, const dpara_attn_io *io, void *workspace, int32_t *status_word,
                               cudaStream_t st);
 
+// out[row] = bf16(x[row] / sqrt(mean(x^2) + eps) * gain) for M rows of H bf16 elements (gain may be null)
+dpara_status launch_rmsnorm_bf16(const void *x, const void *gain, void *out, int M, int H, float eps, cudaStream_t st);
+
 // full backbone block around the attention
 size_t layer_workspace_bytes(const dpara_shape *shape, const dpara_layer_io *layer);
 // byte offsets of xn, qkv, q, k, v, a, h1, hn, act inside the workspace of a full-layer call
