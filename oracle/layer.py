@@ -73,7 +73,13 @@ def rope(x: np.ndarray, pos: np.ndarray, theta: float) -> np.ndarray:
 
 
 class LayerOracle:
-    """Holds the decoded weights so that several boundaries can be evaluated without re-decoding."""
+    """Holds the decoded weights so that several boundaries can be evaluated without re-decoding.
+
+    `boundary(n, j)` is the block for the mask slots of one boundary with the spine's keys/values SUPPLIED (the call
+    that takes them as inputs).  `request(n, x_rows)` is the block for ALL rows of a request -- the d+1 spine tokens as
+    causal query rows (Sec. 3.2, Fig. 4: every anchor reads the cache, itself and the earlier anchors) followed by
+    nothing else changed for the mask slots -- with the spine's keys/values PRODUCED by the block itself, which is what
+    lets blocks be stacked (`backbone`)."""
 
     def __init__(self, lin, attn_in, prefix_base: int = 1, scale: Optional[float] = None):
         sh = attn_in.shape
@@ -130,3 +136,66 @@ class LayerOracle:
         act = swiglu_linear(hn, self.w_gu)
         y = (h1 + linear(act, self.w_down)).astype(np.float32)
         return dict(y=y, q=q, k=k, v=v, a=a, h1=h1.astype(np.float32))
+
+    # ------------------------------------------------------------------ all rows of a request, spine included
+    def request(self, n: int, x_rows: np.ndarray, k_ctx=None, v_ctx=None, ctx_lens=None):
+        """x_rows [J*Bq + S][hidden] float64 (bf16 values): the request's mask-slot rows in (boundary, slot) order, then
+        its S spine rows.  Context keys/values default to the ones this oracle was built with.  Returns y [J*Bq + S][hidden]
+        (fp32 values, float64 array) and the intermediates.  Positions: spine row s at L + s, slot i of boundary j at
+        L + j + 2 + i."""
+        sh, L, A = self.sh, self.lsh, self.ain
+        Hq, Hkv, D, Bq, J, S = sh.n_q_heads, sh.n_kv_heads, sh.head_dim, sh.block, sh.n_boundaries, sh.spine
+        G = Hq // Hkv
+        k_ctx = A.k_ctx if k_ctx is None else k_ctx
+        v_ctx = A.v_ctx if v_ctx is None else v_ctx
+        lo = int(A.ctx_offsets[n])
+        Ln = int(A.ctx_offsets[n + 1]) - lo if ctx_lens is None else int(ctx_lens[n])
+        R = J * Bq + S
+        assert x_rows.shape[0] == R
+        x = np.asarray(x_rows, dtype=np.float64)
+        xn = _r16(rmsnorm(x, self.g1, L.rms_eps))
+        qkv = _r16(linear(xn, self.w_qkv))
+        q = qkv[:, : Hq * D].reshape(R, Hq, D)
+        k = qkv[:, Hq * D:(Hq + Hkv) * D].reshape(R, Hkv, D)
+        v = qkv[:, (Hq + Hkv) * D:].reshape(R, Hkv, D)
+        if L.qk_norm:
+            q = _r16(rmsnorm(q, self.gq, L.rms_eps))
+            k = _r16(rmsnorm(k, self.gk, L.rms_eps))
+        if L.use_rope:
+            pos = np.concatenate([Ln + j + 2 + np.arange(Bq) for j in range(J)] + [Ln + np.arange(S)])
+            q = _r16(rope(q.transpose(1, 0, 2), pos, L.rope_theta)).transpose(1, 0, 2)
+            k = _r16(rope(k.transpose(1, 0, 2), pos, L.rope_theta)).transpose(1, 0, 2)
+        ks, vs = k[J * Bq:], v[J * Bq:]                       # the spine's own keys/values, produced here
+        a = np.zeros((R, Hq, D))
+        for g in range(Hkv):
+            kc, vc = bf16_bits_to_f64(k_ctx[lo:lo + Ln, g]), bf16_bits_to_f64(v_ctx[lo:lo + Ln, g])
+            for h in range(g * G, (g + 1) * G):
+                for j in range(J):                            # a branch: cache, its anchor prefix, its own block
+                    na = max(0, min(j + self.prefix_base, S))
+                    r0 = j * Bq
+                    keys = np.concatenate([kc, ks[:na, g], k[r0:r0 + Bq, g]])
+                    vals = np.concatenate([vc, vs[:na, g], v[r0:r0 + Bq, g]])
+                    a[r0:r0 + Bq, h], _ = softmax_attention(q[r0:r0 + Bq, h], keys, vals, self.scale)
+                for s_ in range(S):                           # an anchor: cache, the earlier anchors, itself
+                    keys = np.concatenate([kc, ks[: s_ + 1, g]])
+                    vals = np.concatenate([vc, vs[: s_ + 1, g]])
+                    a[J * Bq + s_, h], _ = softmax_attention(q[J * Bq + s_: J * Bq + s_ + 1, h], keys, vals, self.scale)
+        a = _r16(a).reshape(R, Hq * D)
+        h1 = (x + linear(a, self.w_o)).astype(np.float32).astype(np.float64)
+        hn = _r16(rmsnorm(h1, self.g2, L.rms_eps))
+        act = swiglu_linear(hn, self.w_gu)
+        y = (h1 + linear(act, self.w_down)).astype(np.float32).astype(np.float64)
+        return dict(y=y, q=q, k=k, v=v, a=a, h1=h1)
+
+
+def backbone(layers, n: int, x_rows: np.ndarray, caches=None, ctx_lens=None) -> np.ndarray:
+    """A stack of blocks on one request's rows: block l reads block l-1's output rounded to bf16 (the residual
+    stream between blocks is bf16) and its own context cache.  layers: LayerOracle objects; caches: optional list of
+    (k_ctx, v_ctx) per layer.  Returns the last block's y [J*Bq + S][hidden] (fp32 values)."""
+    x = np.asarray(x_rows, dtype=np.float64)
+    y = None
+    for l, lay in enumerate(layers):
+        kc, vc = caches[l] if caches is not None else (None, None)
+        y = lay.request(n, x, kc, vc, ctx_lens)["y"]
+        x = _r16(y)
+    return y

@@ -165,3 +165,82 @@ def test_swiglu_linear_halves_and_closed_form():
     one = np.zeros((1, K)); one[0, 0] = 1
     y = OL.swiglu_linear(np.array([[2.0, 0, 0, 0]]), np.concatenate([one, 0.5 * one]))
     assert y[0, 0] == OA.round_to_bf16(np.array(2.0 / (1 + math.exp(-2.0)) * 1.0)).astype(np.float64)
+
+
+# ----------------------------------------------------------------------------- all rows of a request: spine tokens as queries
+def _rows(ain, lin, n, seed=0):
+    """x of request n in the combined order: mask-slot rows (boundary, slot), then spine rows (drawn here)."""
+    sh = ain.shape
+    xm = OA.bf16_bits_to_f64(lin.x[n]).reshape(sh.n_boundaries * sh.block, -1)
+    xs = OA.round_to_bf16(np.random.default_rng(seed).standard_normal((sh.spine, xm.shape[1]))).astype(np.float64)
+    return np.concatenate([xm, xs])
+
+
+def test_request_rows_reduce_to_the_supplied_spine_block():
+    """With the spine's keys/values taken from `request` and handed to `boundary` as inputs, the mask-slot rows agree
+    bit for bit: producing the spine inside the block changes nothing for the branches."""
+    ain, lin = _small()
+    sh = ain.shape
+    orc = OL.LayerOracle(lin, ain)
+    n = 1
+    full = orc.request(n, _rows(ain, lin, n))
+    JB = sh.n_boundaries * sh.block
+    ain.k_spine[n] = W.f32_to_bf16_bits(full["k"][JB:].astype(np.float32))
+    ain.v_spine[n] = W.f32_to_bf16_bits(full["v"][JB:].astype(np.float32))
+    orc2 = OL.LayerOracle(lin, ain)
+    for j in range(sh.n_boundaries):
+        assert np.array_equal(orc2.boundary(n, j)["y"].astype(np.float64), full["y"][j * sh.block:(j + 1) * sh.block])
+
+
+def test_spine_rows_of_the_block_follow_the_figures_mask():
+    """Fig. 4 through a whole block: anchor s reads the cache, itself and earlier anchors only; branch j reads anchors
+    < j + 1 and its own slots only.  Perturbing a row must leave every row that cannot see it bit-identical."""
+    ain, lin = _small()
+    sh = ain.shape
+    J, Bq, S = sh.n_boundaries, sh.block, sh.spine
+    JB = J * Bq
+    orc = OL.LayerOracle(lin, ain)
+    x = _rows(ain, lin, 0)
+    base = orc.request(0, x)["y"]
+    # change spine token 2 (of 3): anchors 0, 1 and branches 0, 1 (prefix 1, 2 anchors) must not move; anchor 2 and branch 2 must
+    x2 = x.copy(); x2[JB + 2] += 1.0
+    y2 = orc.request(0, x2)["y"]
+    same = list(range(0, 2 * Bq)) + [JB, JB + 1]
+    assert np.array_equal(y2[same], base[same])
+    assert not np.array_equal(y2[JB + 2], base[JB + 2]) and not np.array_equal(y2[2 * Bq:3 * Bq], base[2 * Bq:3 * Bq])
+    # change a mask slot of branch 1: only branch 1's rows move (bidirectional inside the branch, invisible elsewhere)
+    x3 = x.copy(); x3[1 * Bq] += 1.0
+    y3 = orc.request(0, x3)["y"]
+    others = [r for r in range(JB + S) if not (Bq <= r < 2 * Bq)]
+    assert np.array_equal(y3[others], base[others])
+    assert not np.array_equal(y3[Bq + 1], base[Bq + 1])
+    # the anchors' attention output equals the stand-alone spine attention on the block's own q, k, v
+    r = orc.request(0, x)
+    q = W.f32_to_bf16_bits(r["q"][JB:].astype(np.float32))[None]
+    k = W.f32_to_bf16_bits(r["k"][JB:].astype(np.float32))[None]
+    v = W.f32_to_bf16_bits(r["v"][JB:].astype(np.float32))[None]
+    lo, hi = int(ain.ctx_offsets[0]), int(ain.ctx_offsets[1])
+    want = OA.spine_rows(q, ain.k_ctx[lo:hi], ain.v_ctx[lo:hi], np.array([0, hi - lo]), k, v)[0]
+    assert np.array_equal(OA.round_to_bf16(want.reshape(S, -1)).astype(np.float64), r["a"][JB:])
+
+
+def test_stacked_blocks_keep_causality_and_isolation():
+    """Two blocks: the second reads the first one's rows (bf16).  What Fig. 4 forbids at one block stays forbidden through
+    the stack; and a second block with zero output projections passes the first block's result through."""
+    ain, lin = _small()
+    sh = ain.shape
+    J, Bq, S = sh.n_boundaries, sh.block, sh.spine
+    JB = J * Bq
+    lin2 = W.make_layer_inputs(W.LayerShape(64, 96), sh, 77)
+    l1, l2 = OL.LayerOracle(lin, ain), OL.LayerOracle(lin2, ain)
+    x = _rows(ain, lin, 0)
+    base = OL.backbone([l1, l2], 0, x)
+    x2 = x.copy(); x2[JB + 1] -= 0.5                                   # spine token 1
+    y2 = OL.backbone([l1, l2], 0, x2)
+    same = list(range(0, Bq)) + [JB]                                   # branch 0 (reads anchor 0 only) and anchor 0
+    assert np.array_equal(y2[same], base[same])
+    assert not np.array_equal(y2[Bq:2 * Bq], base[Bq:2 * Bq])           # branch 1 reads anchors 0, 1
+    lin2.w_o[:] = 0; lin2.w_down[:] = 0
+    y1 = l1.request(0, x)["y"]
+    thru = OL.backbone([l1, OL.LayerOracle(lin2, ain)], 0, x)
+    assert np.array_equal(thru, OA.round_to_bf16(y1).astype(np.float64))
