@@ -71,6 +71,10 @@ typedef struct {
   int32_t boundary_lo;  /* boundaries computed: [boundary_lo, boundary_hi); all = [0, J);        */
   int32_t boundary_hi;  /* a conventional single-anchor-set draft step = [j, j + 1)               */
   float softmax_scale;  /* 0 selects 1/sqrt(D) */
+  int32_t spine_queries; /* 0: only the mask slots are query rows (the spine's keys/values are inputs).  1: the S spine
+                            tokens are query rows as well (Sec. 3.2, Fig. 4: an anchor reads the cache, itself and the
+                            earlier anchors) -- q, out and out_lse then hold J*Bq + S rows per request, the mask-slot rows
+                            in (boundary, slot) order followed by the spine rows; needs boundary_lo = 0, boundary_hi = J */
 } dpara_shape;
 
 /* Tensors of the attention (Fig. 4).  Context keys/values are the drafter-side projection of the

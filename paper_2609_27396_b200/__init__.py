@@ -31,7 +31,8 @@ BF16, F32 = 0, 1
 class Shape(C.Structure):
     _fields_ = [("batch", C.c_int32), ("n_boundaries", C.c_int32), ("block", C.c_int32), ("n_q_heads", C.c_int32),
                 ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32), ("prefix_base", C.c_int32), ("n_spine", C.c_int32),
-                ("boundary_lo", C.c_int32), ("boundary_hi", C.c_int32), ("softmax_scale", C.c_float)]
+                ("boundary_lo", C.c_int32), ("boundary_hi", C.c_int32), ("softmax_scale", C.c_float),
+                ("spine_queries", C.c_int32)]
 
 
 class AttnIO(C.Structure):
@@ -151,13 +152,13 @@ class DraftPlan:
     def __init__(self, *, ctx_offsets: Sequence[int], n_boundaries: int, block: int, n_q_heads: int, n_kv_heads: int,
                  head_dim: int, prefix_base: int = 1, n_spine: Optional[int] = None, boundary_lo: int = 0,
                  boundary_hi: Optional[int] = None, softmax_scale: float = 0.0, layer: Optional[LayerIO] = None,
-                 ctx_lens: Optional[Sequence[int]] = None, device="cuda"):
+                 ctx_lens: Optional[Sequence[int]] = None, spine_queries: bool = False, device="cuda"):
         """ctx_lens: for caches kept with slack (dpara_cache_append) -- request n's context is the first ctx_lens[n] of
         its rows ctx_offsets[n]..ctx_offsets[n+1]; update it between calls with set_ctx_lens()."""
         b = len(ctx_offsets) - 1
         self.shape = Shape(b, n_boundaries, block, n_q_heads, n_kv_heads, head_dim, prefix_base,
                            n_boundaries if n_spine is None else n_spine, boundary_lo,
-                           n_boundaries if boundary_hi is None else boundary_hi, softmax_scale)
+                           n_boundaries if boundary_hi is None else boundary_hi, softmax_scale, 1 if spine_queries else 0)
         self.host_off = _host_offsets(ctx_offsets)
         self.dev_off = torch.tensor([int(x) for x in ctx_offsets], dtype=torch.int64, device=device)
         self.layer = layer
@@ -239,6 +240,23 @@ def draft_all_boundaries(q, k_ctx, v_ctx, ctx_offsets: Sequence[int], k_spine, v
     out = torch.zeros(q.shape, dtype=out_dtype, device=q.device)
     lse = torch.full((b, J, Bq, Hq), float("-inf"), dtype=torch.float32, device=q.device) if want_lse else None
     plan(q=q, k_ctx=k_ctx, v_ctx=v_ctx, k_spine=k_spine, v_spine=v_spine, k_blk=k_blk, v_blk=v_blk, out=out, out_lse=lse,
+         stream=stream)
+    return (out, lse, plan.status) if want_lse else (out, plan.status)
+
+
+def draft_with_spine_queries(q_rows, n_boundaries: int, block: int, k_ctx, v_ctx, ctx_offsets: Sequence[int], k_spine, v_spine,
+                             k_blk=None, v_blk=None, *, prefix_base: int = 1, softmax_scale: float = 0.0,
+                             out_dtype=torch.bfloat16, want_lse: bool = False, stream=None):
+    """dpara_draft_all_boundaries with spine_queries = 1 (attention only): q_rows [b][J*Bq + S][Hq][D] holds each request's
+    mask-slot rows in (boundary, slot) order followed by its S spine rows; out (and lse) come back in the same row order."""
+    b, R, Hq, D = q_rows.shape
+    S, Hkv = k_spine.shape[1], k_spine.shape[2]
+    assert R == n_boundaries * block + S
+    plan = DraftPlan(ctx_offsets=ctx_offsets, n_boundaries=n_boundaries, block=block, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=D,
+                     prefix_base=prefix_base, n_spine=S, softmax_scale=softmax_scale, spine_queries=True, device=q_rows.device)
+    out = torch.zeros(q_rows.shape, dtype=out_dtype, device=q_rows.device)
+    lse = torch.full((b, R, Hq), float("-inf"), dtype=torch.float32, device=q_rows.device) if want_lse else None
+    plan(q=q_rows, k_ctx=k_ctx, v_ctx=v_ctx, k_spine=k_spine, v_spine=v_spine, k_blk=k_blk, v_blk=v_blk, out=out, out_lse=lse,
          stream=stream)
     return (out, lse, plan.status) if want_lse else (out, plan.status)
 

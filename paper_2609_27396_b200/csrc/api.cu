@@ -17,6 +17,8 @@ static dpara_status validate_shape(const dpara_shape *s) {
   if (s->n_spine < 0 || s->prefix_base < 0) return DPARA_ERR_INVALID_ARG;
   if (s->boundary_lo < 0 || s->boundary_hi > s->n_boundaries || s->boundary_lo > s->boundary_hi) return DPARA_ERR_INVALID_ARG;
   if (!(s->softmax_scale >= 0.f)) return DPARA_ERR_INVALID_ARG;
+  if (s->spine_queries != 0 && s->spine_queries != 1) return DPARA_ERR_INVALID_ARG;
+  if (s->spine_queries && (s->boundary_lo != 0 || s->boundary_hi != s->n_boundaries || s->n_spine == 0)) return DPARA_ERR_UNSUPPORTED;
   if (s->head_dim != 64 && s->head_dim != 128) return DPARA_ERR_UNSUPPORTED;
   if (s->n_q_heads % s->n_kv_heads != 0) return DPARA_ERR_UNSUPPORTED;
   if (s->n_q_heads / s->n_kv_heads > 16 || s->block > 64 || s->n_spine > 64) return DPARA_ERR_UNSUPPORTED;

@@ -22,6 +22,10 @@ void fill_attn_params(AttnParams &P, const dpara_shape *s, const dpara_attn_io *
   P.b = s->batch; P.J = s->n_boundaries; P.Bq = s->block; P.Hq = s->n_q_heads; P.Hkv = s->n_kv_heads;
   P.D = s->head_dim; P.G = s->n_q_heads / s->n_kv_heads; P.S = s->n_spine; P.pb = s->prefix_base;
   P.lo = s->boundary_lo; P.hi = s->boundary_hi;
+  P.Sq = s->spine_queries ? s->n_spine : 0;
+  P.q_req_rows = s->n_boundaries * s->block + P.Sq;
+  P.blk_req_rows = s->n_boundaries * s->block;
+  P.spine_req_rows = s->n_spine;
   P.scale = s->softmax_scale > 0.f ? s->softmax_scale : 1.0f / sqrtf((float)s->head_dim);
   P.status_word = status_word;
 }

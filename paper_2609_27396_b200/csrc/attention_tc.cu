@@ -65,6 +65,7 @@ struct TcParams {
 
   // tail tiles: the first holds the spine (S8 = S rounded up to 8 rows) and cap0 blocks, the others cap blocks
   int n_ji, n_pairs, nsplit, S8, cap0, cap, has_blk, has_tail, n_items;
+  int n_rows;  // query rows per request and head: n_ji mask-slot rows, then the spine rows when they are queries
   float *part_o;   // split-KV partials [item slot][2][D / 4][128 rows] float4 (unnormalised rows; a warp's lanes are
                    // consecutive rows, so its stores and the merge's loads are contiguous 512-byte runs)
   float2 *part_ml; // [item slot][2][128] (row max in raw-score units, row sum)
@@ -232,7 +233,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
       ok = __all_sync(0xffffffffu, mbar_wait(q_empty, (k & 1) ^ 1u, abort_flag));
       if (!ok) break;
       if (lane == 0) {
-        const int qrow0 = (I.n * A.J + A.lo) * A.Bq + I.ji0;
+        const int qrow0 = I.n * A.q_req_rows + A.lo * A.Bq + I.ji0;
         mbar_arrive_expect_tx(q_full, (uint32_t)(I.ntq * Cfg::kTileBytes));
         for (int t = 0; t < I.ntq; ++t)
           for (int sb = 0; sb < Cfg::kSlabs; ++sb)
@@ -271,16 +272,16 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
               if (P.has_blk) bytes += (uint32_t)(P.cap0 * A.Bq) * 128 * Cfg::kSlabs;
               mbar_arrive_expect_tx(kv_full + sl, bytes);
               for (int sb = 0; sb < Cfg::kSlabs; ++sb) {
-                if (A.S > 0) tma_load_3d(dst + sb * Cfg::kSlabBytes, is_v ? &P.map_vs : &P.map_ks, kv_full + sl, sb * 64, I.g, I.n * A.S);
+                if (A.S > 0) tma_load_3d(dst + sb * Cfg::kSlabBytes, is_v ? &P.map_vs : &P.map_ks, kv_full + sl, sb * 64, I.g, I.n * A.spine_req_rows);
                 if (P.has_blk)
                   tma_load_3d(dst + sb * Cfg::kSlabBytes + P.S8 * 128, is_v ? &P.map_vb0 : &P.map_kb0, kv_full + sl, sb * 64, I.g,
-                              (I.n * A.J + I.jb0) * A.Bq);
+                              I.n * A.blk_req_rows + I.jb0 * A.Bq);
               }
             } else {
               mbar_arrive_expect_tx(kv_full + sl, (uint32_t)(P.cap * A.Bq) * 128 * Cfg::kSlabs);
               for (int sb = 0; sb < Cfg::kSlabs; ++sb)
                 tma_load_3d(dst + sb * Cfg::kSlabBytes, is_v ? &P.map_vb : &P.map_kb, kv_full + sl, sb * 64, I.g,
-                            (I.n * A.J + I.jb0 + P.cap0 + (tk - 1) * P.cap) * A.Bq);
+                            I.n * A.blk_req_rows + (I.jb0 + P.cap0 + (tk - 1) * P.cap) * A.Bq);
             }
           }
         }
@@ -397,9 +398,9 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
       const int id = P.use_sched ? (int)P.sched[qi] : qi;
       const Item I = decode_item(P, id);
       const int ji = I.ji0 + t * I.ji_t + (r >> I.hs);
-      const bool valid = (t < I.ntq) && (ji < P.n_ji);
-      const int j = A.lo + ji / A.Bq, i = ji % A.Bq, h = I.g * A.G + I.h0 + (r & ((1 << I.hs) - 1));
-      const size_t orow = (((size_t)I.n * A.J + j) * A.Bq + i) * A.Hq + h;
+      const bool valid = (t < I.ntq) && (ji < P.n_rows);
+      const int h = I.g * A.G + I.h0 + (r & ((1 << I.hs) - 1));
+      const size_t orow = ((size_t)I.n * A.q_req_rows + A.lo * A.Bq + ji) * A.Hq + h;
       // split-KV: this CTA's partial rows go to an L2-resident scratch slot and are merged after a cluster barrier
       const size_t pslot = ((size_t)I.slot * 2 + t) * 128 + r;
       if (I.n_iter == 0 || t >= I.ntq) {
@@ -416,7 +417,11 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
         continue;
       }
       const int n_iter = I.n_iter;
-      const int jrel = j - I.jb0;  // this row's boundary, counted from the first one whose block sits in the tail tiles
+      // a mask-slot row: its boundary, counted from the first one whose block sits in the tail tiles, and its anchor
+      // prefix; a spine row (an anchor as a query): no own block (-1), and anchors 0 .. itself
+      const bool is_spine = ji >= P.n_ji;
+      const int jrel = is_spine ? -1 : A.lo + ji / A.Bq - I.jb0;
+      const int na_row = is_spine ? ji - P.n_ji + 1 : max(0, min(A.lo + ji / A.Bq + A.pb, A.S));
       float m_used = -INFINITY, l = 0.f;
 
       for (int it = 0; it < n_iter; ++it) {
@@ -426,9 +431,9 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
         uint32_t vis[4] = {0u, 0u, 0u, 0u};
         if (it >= I.n_ctx_it) {
           const int tk = it - I.n_ctx_it;
-          const int kt = !P.has_blk ? -1 : (jrel < P.cap0 ? 0 : 1 + (jrel - P.cap0) / P.cap);
+          const int kt = (!P.has_blk || jrel < 0) ? -1 : (jrel < P.cap0 ? 0 : 1 + (jrel - P.cap0) / P.cap);
           const int boff = jrel < P.cap0 ? P.S8 + jrel * A.Bq : ((jrel - P.cap0) % P.cap) * A.Bq;
-          const int na_t = tk == 0 ? max(0, min(I.jb0 + jrel + A.pb, A.S)) : 0;
+          const int na_t = tk == 0 ? na_row : 0;
           const int b0 = tk == kt ? boff : 0, b1 = tk == kt ? boff + A.Bq : 0;
 #pragma unroll
           for (int w = 0; w < 4; ++w) vis[w] = bits_below(na_t - 32 * w) | (bits_below(b1 - 32 * w) & ~bits_below(b0 - 32 * w));
@@ -602,9 +607,9 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
         const int R = (int)rank * rows_per + u % rows_per, part = u / rows_per;
         const int t = R >> 7, r = R & 127;
         const int ji = I.ji0 + t * I.ji_t + (r >> I.hs);
-        if (t >= I.ntq || ji >= P.n_ji) continue;
-        const int j = A.lo + ji / A.Bq, i = ji % A.Bq, h = I.g * A.G + I.h0 + (r & ((1 << I.hs) - 1));
-        const size_t orow = (((size_t)I.n * A.J + j) * A.Bq + i) * A.Hq + h;
+        if (t >= I.ntq || ji >= P.n_rows) continue;
+        const int h = I.g * A.G + I.h0 + (r & ((1 << I.hs) - 1));
+        const size_t orow = ((size_t)I.n * A.q_req_rows + A.lo * A.Bq + ji) * A.Hq + h;
         float2 ml[8];
 #pragma unroll
         for (int sp = 0; sp < 8; ++sp)
@@ -689,12 +694,13 @@ TcPlan plan_attention_tc(const dpara_shape *s, const int64_t *host_off, const in
   if (nb <= 0) return p;
   if (G > 16 || s->n_spine > 64 || s->block > 64) return p;
   p.n_ji = nb * s->block;
+  p.n_rows = p.n_ji + (s->spine_queries ? s->n_spine : 0);
   // head blocks = binary digits of G, widest first; block k's tiles hold 128 / hb (j, i) rows
   p.n_hblk = 0;
   p.n_pairs = 0;
   for (int bit = 4, h0 = 0; bit >= 0; --bit) {
     if (!(G & (1 << bit))) continue;
-    const int ji_t = 128 >> bit, tiles = (p.n_ji + ji_t - 1) / ji_t;
+    const int ji_t = 128 >> bit, tiles = (p.n_rows + ji_t - 1) / ji_t;
     p.hb_log2[p.n_hblk] = bit;
     p.h0[p.n_hblk] = h0;
     p.pair_start[p.n_hblk] = p.n_pairs;
@@ -763,7 +769,7 @@ dpara_status launch_attention_tc(const AttnParams &A, const TcPlan &plan, const 
   TcParams P;
   memset(&P, 0, sizeof(P));
   P.a = A;
-  P.n_ji = plan.n_ji; P.n_pairs = plan.n_pairs; P.nsplit = plan.nsplit;
+  P.n_ji = plan.n_ji; P.n_rows = plan.n_rows; P.n_pairs = plan.n_pairs; P.nsplit = plan.nsplit;
   P.n_hblk = plan.n_hblk;
   for (int k = 0; k < plan.n_hblk; ++k) { P.hb_log2[k] = plan.hb_log2[k]; P.h0[k] = plan.h0[k]; }
   for (int k = 0; k <= plan.n_hblk; ++k) P.pair_start[k] = plan.pair_start[k];
@@ -775,20 +781,23 @@ dpara_status launch_attention_tc(const AttnParams &A, const TcPlan &plan, const 
     int blk = 0;
     while (blk + 1 < plan.n_hblk && x >= plan.pair_start[blk + 1]) ++blk;
     const int ji_t = 128 >> plan.hb_log2[blk], pl = x - plan.pair_start[blk];
-    const int ntq = std::min(2, (plan.n_ji + ji_t - 1) / ji_t - pl * 2);
+    const int ntq = std::min(2, (plan.n_rows + ji_t - 1) / ji_t - pl * 2);
+    // boundaries whose own blocks the pair's mask-slot rows need (none if the pair holds spine rows only)
     const int ji0 = pl * 2 * ji_t, ji_last = std::min(ji0 + ntq * ji_t, plan.n_ji) - 1;
     TcParams::PairInfo &pi = P.pair[x];
     pi.ji0 = (int16_t)ji0;
     pi.jb0_rel = (int16_t)(ji0 / A.Bq);
     pi.blk = (uint8_t)blk; pi.hs = (uint8_t)plan.hb_log2[blk]; pi.h0 = (uint8_t)plan.h0[blk]; pi.ntq = (uint8_t)ntq;
-    pi.n_tail = (uint8_t)tail_tiles(P.has_tail, P.has_blk, ji_last / A.Bq - ji0 / A.Bq + 1, plan.cap0, plan.cap);
+    pi.n_tail = (uint8_t)tail_tiles(P.has_tail, P.has_blk, ji_last >= ji0 ? ji_last / A.Bq - ji0 / A.Bq + 1 : 0, plan.cap0, plan.cap);
   }
 
   P.c_log2 = A.scale * 1.4426950408889634f;
   const int D = A.D;
   const uint64_t rs = (uint64_t)D * 2;
   const long long tot = host_off[A.b] - host_off[0];
-  const uint64_t nq = (uint64_t)A.b * A.J * A.Bq;
+  const uint64_t nq = (uint64_t)A.b * A.q_req_rows;
+  const uint64_t n_blk_rows = (uint64_t)(A.b - 1) * A.blk_req_rows + (uint64_t)A.J * A.Bq;
+  const uint64_t n_spine_rows = (uint64_t)(A.b - 1) * A.spine_req_rows + (uint64_t)A.S;
   bool ok = true;
   for (int k = 0; k < plan.n_hblk; ++k)
     ok = ok && make_tmap_bf16_3d(&P.map_q[k], A.q, D, A.Hq, nq, rs, rs * A.Hq, 64, 1u << plan.hb_log2[k], 128u >> plan.hb_log2[k]);
@@ -797,14 +806,14 @@ dpara_status launch_attention_tc(const AttnParams &A, const TcPlan &plan, const 
     ok = ok && make_tmap_bf16_3d(&P.map_vc, A.v_ctx, D, A.Hkv, host_off[A.b], rs, rs * A.Hkv, 64, 1, 128);
   }
   if (A.S > 0) {
-    ok = ok && make_tmap_bf16_3d(&P.map_ks, A.k_spine, D, A.Hkv, (uint64_t)A.b * A.S, rs, rs * A.Hkv, 64, 1, A.S);
-    ok = ok && make_tmap_bf16_3d(&P.map_vs, A.v_spine, D, A.Hkv, (uint64_t)A.b * A.S, rs, rs * A.Hkv, 64, 1, A.S);
+    ok = ok && make_tmap_bf16_3d(&P.map_ks, A.k_spine, D, A.Hkv, n_spine_rows, rs, rs * A.Hkv, 64, 1, A.S);
+    ok = ok && make_tmap_bf16_3d(&P.map_vs, A.v_spine, D, A.Hkv, n_spine_rows, rs, rs * A.Hkv, 64, 1, A.S);
   }
   if (P.has_blk) {
-    ok = ok && make_tmap_bf16_3d(&P.map_kb0, A.k_blk, D, A.Hkv, nq, rs, rs * A.Hkv, 64, 1, plan.cap0 * A.Bq);
-    ok = ok && make_tmap_bf16_3d(&P.map_vb0, A.v_blk, D, A.Hkv, nq, rs, rs * A.Hkv, 64, 1, plan.cap0 * A.Bq);
-    ok = ok && make_tmap_bf16_3d(&P.map_kb, A.k_blk, D, A.Hkv, nq, rs, rs * A.Hkv, 64, 1, plan.cap * A.Bq);
-    ok = ok && make_tmap_bf16_3d(&P.map_vb, A.v_blk, D, A.Hkv, nq, rs, rs * A.Hkv, 64, 1, plan.cap * A.Bq);
+    ok = ok && make_tmap_bf16_3d(&P.map_kb0, A.k_blk, D, A.Hkv, n_blk_rows, rs, rs * A.Hkv, 64, 1, plan.cap0 * A.Bq);
+    ok = ok && make_tmap_bf16_3d(&P.map_vb0, A.v_blk, D, A.Hkv, n_blk_rows, rs, rs * A.Hkv, 64, 1, plan.cap0 * A.Bq);
+    ok = ok && make_tmap_bf16_3d(&P.map_kb, A.k_blk, D, A.Hkv, n_blk_rows, rs, rs * A.Hkv, 64, 1, plan.cap * A.Bq);
+    ok = ok && make_tmap_bf16_3d(&P.map_vb, A.v_blk, D, A.Hkv, n_blk_rows, rs, rs * A.Hkv, 64, 1, plan.cap * A.Bq);
   }
   if (!ok) return DPARA_ERR_CUDA;
   P.use_ctx_p = A.b <= kMaxOrdered;

@@ -31,7 +31,7 @@ def test_status_strings_and_version():
 
 def _shape(**kw):
     d = dict(batch=1, n_boundaries=3, block=2, n_q_heads=4, n_kv_heads=2, head_dim=64, prefix_base=1, n_spine=3,
-             boundary_lo=0, boundary_hi=3, softmax_scale=0.0)
+             boundary_lo=0, boundary_hi=3, softmax_scale=0.0, spine_queries=0)
     d.update(kw)
     return dp.Shape(*[d[f[0]] for f in dp.Shape._fields_])
 
@@ -44,6 +44,8 @@ def test_draft_argument_validation():
     assert call(_shape(n_q_heads=3), io) == dp.ERR_UNSUPPORTED
     assert call(_shape(batch=0), io) == dp.ERR_INVALID_ARG
     assert call(_shape(boundary_hi=4), io) == dp.ERR_INVALID_ARG
+    assert call(_shape(spine_queries=2), io) == dp.ERR_INVALID_ARG
+    assert call(_shape(spine_queries=1, boundary_lo=1), io) == dp.ERR_UNSUPPORTED    # spine rows need the full boundary range
     assert call(_shape(), None) == dp.ERR_INVALID_ARG
     assert call(_shape(), io) == dp.ERR_INVALID_ARG                     # no host offsets
     io.host_ctx_offsets = C.cast(off, C.c_void_p).value

@@ -160,3 +160,36 @@ def test_several_tail_tiles():
     the boundaries a tile pair touches > 128): the blocks spill into further tail tiles."""
     _compare(W.make_attn_inputs(W.AttnShape((70, 200), 4, 2, 64, 3, 64, 1, 64), 13))
     _compare(W.make_attn_inputs(W.AttnShape((33,), 8, 2, 128, 4, 48, 1, 40), 14), with_blk=True)
+
+
+@pytest.mark.parametrize("shape", [
+    W.AttnShape((300, 77), 8, 2, 128, 8, 8),             # 64 + 8 rows per request: the spine rows share a tile with mask rows
+    W.AttnShape((129, 1, 257), 10, 2, 128, 4, 16),       # group size 5 (two head blocks), ragged
+    W.AttnShape((0, 40), 4, 2, 64, 3, 2),                # an empty context: anchor 0 reads itself only
+    W.AttnShape((520,), 8, 2, 128, 16, 16),              # 256 mask rows fill the tiles: the spine rows get a pair of their own
+    W.AttnShape((200, 130, 77, 300, 64, 1, 257, 129), 32, 8, 128, 8, 8),   # 64 items: persistent kernel without a KV split
+])
+def test_spine_tokens_as_query_rows(shape):
+    """spine_queries = 1: the mask-slot rows are unchanged and each spine token is a causal query row over the cache,
+    itself and the earlier spine tokens (oracle.attention.spine_rows)."""
+    import paper_2609_27396_b200 as dp
+    from gpu_util import dev_bf16
+    inp = W.make_attn_inputs(shape, 41)
+    b, J, Bq, Hq, D, S = shape.batch, shape.n_boundaries, shape.block, shape.n_q_heads, shape.head_dim, shape.spine
+    q_spine = W.make_attn_inputs(W.AttnShape(shape.ctx_lens, Hq, shape.n_kv_heads, D, S, 1), 42).q.reshape(b, S, Hq, D)
+    q_rows = np.concatenate([inp.q.reshape(b, J * Bq, Hq, D), q_spine], axis=1)
+    out, lse, status = dp.draft_with_spine_queries(dev_bf16(q_rows), J, Bq, dev_bf16(inp.k_ctx), dev_bf16(inp.v_ctx),
+                                                   [int(x) for x in inp.ctx_offsets], dev_bf16(inp.k_spine), dev_bf16(inp.v_spine),
+                                                   dev_bf16(inp.k_blk), dev_bf16(inp.v_blk), out_dtype=torch.float32, want_lse=True)
+    torch.cuda.synchronize()
+    o = out.cpu().numpy().astype(np.float64)
+    ref_mask, _ = _oracle(inp)
+    ref_spine = OA.spine_rows(q_spine, inp.k_ctx, inp.v_ctx, inp.ctx_offsets, inp.k_spine, inp.v_spine)
+    tol = _tol(np.concatenate([ref_mask.reshape(b, J * Bq, Hq, D), ref_spine], axis=1), shape.ctx_lens)
+    assert np.all(np.abs(o[:, :J * Bq] - ref_mask.reshape(b, J * Bq, Hq, D)) <= tol[:, :J * Bq])
+    assert np.all(np.abs(o[:, J * Bq:] - ref_spine) <= tol[:, J * Bq:])
+    assert np.isfinite(lse.cpu().numpy()).all() and int(status.item()) == 0
+    out16, _ = dp.draft_with_spine_queries(dev_bf16(q_rows), J, Bq, dev_bf16(inp.k_ctx), dev_bf16(inp.v_ctx),
+                                           [int(x) for x in inp.ctx_offsets], dev_bf16(inp.k_spine), dev_bf16(inp.v_spine),
+                                           dev_bf16(inp.k_blk), dev_bf16(inp.v_blk))
+    assert np.all(np.abs(out16.float().cpu().numpy()[:, J * Bq:] - ref_spine) <= tol[:, J * Bq:])
