@@ -103,7 +103,9 @@ typedef struct {
 /* Full-layer mode (one pre-norm backbone block; Sec. 3.1 lists the block's trainable parts without giving
  * equations -- the equations are this library's reading, stated with the call). */
 typedef struct {
-  const void *x;                                   /* [b][J][Bq][hidden] bf16 hidden states of the mask slots */
+  const void *x;                                   /* [b][J][Bq][hidden] bf16 hidden states of the mask slots; with
+                                                      shape->spine_queries: [b][J*Bq + S][hidden], each request's spine rows
+                                                      behind its mask-slot rows (y_f32 / y_bf16 likewise) */
   const void *w_qkv;                               /* [(Hq + 2 Hkv) D][hidden] bf16, rows = [q | k | v] */
   const void *w_o;                                 /* [hidden][Hq D] bf16 */
   const void *w_gate_up;                           /* [2 inter][hidden] bf16, rows [0,inter) gate, [inter,2 inter) up */
@@ -142,11 +144,32 @@ dpara_status dpara_draft_all_boundaries(const dpara_shape *shape, const dpara_at
                                         const dpara_layer_io *layer, void *workspace,
                                         size_t workspace_bytes, int32_t *status_word, void *stream);
 
+/* A stack of backbone blocks in one call (Alg. 1 line 1 runs the whole M-DFlash backbone on the spine; Sec. 3.2 / Fig. 4
+ * give the mask every block uses).  Block l reads block l-1's bf16 output (the residual stream between blocks is bf16)
+ * and its own context cache.  Meant for shape->spine_queries = 1, where every block produces the spine's keys/values
+ * itself (with spine_queries = 0 all blocks would read the same supplied spine keys/values); x and the outputs then hold
+ * J*Bq + S rows per request, the mask-slot rows followed by the spine rows.
+ *   host_layers   HOST array [n_layers] of dpara_layer_io: weights and flags of each block (all with the same hidden and
+ *                 intermediate sizes); x is taken from entry 0 only, y_f32 (required) and y_bf16 from the last entry only
+ *   host_k_ctx, host_v_ctx   HOST arrays [n_layers] of DEVICE pointers: each block's context keys/values, all laid out
+ *                 by io->ctx_offsets (and io->ctx_lens); io->k_ctx / io->v_ctx are ignored
+ * Workspace: dpara_backbone_workspace_bytes().  Errors: as dpara_draft_all_boundaries. */
+typedef struct {
+  int32_t n_layers;
+  const dpara_layer_io *host_layers;
+  const void *const *host_k_ctx;
+  const void *const *host_v_ctx;
+} dpara_backbone_io;
+size_t dpara_backbone_workspace_bytes(const dpara_shape *shape, const int64_t *host_ctx_offsets, const dpara_backbone_io *bb);
+dpara_status dpara_draft_backbone(const dpara_shape *shape, const dpara_attn_io *io, const dpara_backbone_io *bb, void *workspace,
+                                  size_t workspace_bytes, int32_t *status_word, void *stream);
+
 /* Where a full-layer call leaves the block's intermediates (the quantities named in the equations above;
  * the paper, Sec. 3.1, lists the block's parts without equations).  offsets[0..8] receive the byte offsets,
  * inside the call's workspace, of  xn [M][hidden] bf16,  qkv [M][(Hq+2Hkv)D] bf16,  q [M][Hq D] bf16,
  * k [M][Hkv D] bf16,  v [M][Hkv D] bf16,  a [M][Hq D] bf16,  h1 [M][hidden] fp32,  hn [M][hidden] bf16,
- * act [M][inter] bf16, with M = b * J * Bq rows in (request, boundary, slot) order.  They hold the last call's
+ * act [M][inter] bf16, with M = b * J * Bq rows in (request, boundary, slot) order (b * (J * Bq + S) rows, each request's
+ * spine rows behind its mask-slot rows, when shape->spine_queries is set).  They hold the last call's
  * values until the workspace is reused.  Host-only; nothing is launched.  For stage-by-stage checks.
  * Errors: INVALID_ARG, UNSUPPORTED (as dpara_draft_all_boundaries). */
 dpara_status dpara_layer_workspace_layout(const dpara_shape *shape, const int64_t *host_ctx_offsets,
@@ -173,6 +196,8 @@ typedef struct {
   int32_t *gather_idx;         /* [b] index of the selected branch (= r) */
   int32_t *out_tokens;         /* optional [b][J]: t_1..t_r, bonus, then -1 */
   void *selected;              /* [b][Bq][hidden] bf16 = reps[n][r] (required when reps != NULL) */
+  int32_t rep_req_rows;        /* rows of `hidden` elements from one request's representations to the next request's;
+                                  0 = J * Bq (packed).  J * Bq + S for the output of a call with spine query rows */
 } dpara_verify_io;
 
 /* Bytes of scratch dpara_verify_select needs; only the sizes and mode of `io` are read. 0 on bad sizes. */

@@ -53,7 +53,8 @@ class VerifyIO(C.Structure):
     _fields_ = [("batch", C.c_int32), ("n_boundaries", C.c_int32), ("vocab", C.c_int32), ("block", C.c_int32),
                 ("hidden", C.c_int32), ("mode", C.c_int32), ("target", C.c_void_p), ("draft_probs", C.c_void_p),
                 ("draft_tokens", C.c_void_p), ("uniforms", C.c_void_p), ("reps", C.c_void_p), ("accept_len", C.c_void_p),
-                ("bonus", C.c_void_p), ("gather_idx", C.c_void_p), ("out_tokens", C.c_void_p), ("selected", C.c_void_p)]
+                ("bonus", C.c_void_p), ("gather_idx", C.c_void_p), ("out_tokens", C.c_void_p), ("selected", C.c_void_p),
+                ("rep_req_rows", C.c_int32)]
 
 
 lib.dpara_draft_workspace_bytes.restype = C.c_size_t
@@ -207,7 +208,7 @@ def layer_intermediates(plan: "DraftPlan") -> dict:
     if rc != OK:
         raise DparaError(rc)
     sh, L = plan.shape, plan.layer
-    M = sh.batch * sh.n_boundaries * sh.block
+    M = sh.batch * (sh.n_boundaries * sh.block + (sh.n_spine if sh.spine_queries else 0))
     QD, KD = sh.n_q_heads * sh.head_dim, sh.n_kv_heads * sh.head_dim
     width = dict(xn=L.hidden, qkv=QD + 2 * KD, q=QD, k=KD, v=KD, a=QD, h1=L.hidden, hn=L.hidden, act=L.intermediate)
     res = {}
@@ -264,8 +265,10 @@ def draft_with_spine_queries(q_rows, n_boundaries: int, block: int, k_ctx, v_ctx
 class VerifyPlan:
     """Fixed-address outputs and workspace for repeated verify/select calls on one shape."""
 
-    def __init__(self, *, batch: int, n_boundaries: int, vocab: int, block: int, hidden: int, mode: int, device="cuda"):
+    def __init__(self, *, batch: int, n_boundaries: int, vocab: int, block: int, hidden: int, mode: int, rep_req_rows: int = 0,
+                 device="cuda"):
         self.io = VerifyIO(batch, n_boundaries, vocab, block, hidden, mode)
+        self.io.rep_req_rows = rep_req_rows
         self.accept_len = torch.zeros(batch, dtype=torch.int32, device=device)
         self.bonus = torch.zeros(batch, dtype=torch.int32, device=device)
         self.gather_idx = torch.zeros(batch, dtype=torch.int32, device=device)
@@ -406,5 +409,55 @@ class CachePlan:
         self.io.features, self.io.accept_len = _ptr(features), _ptr(accept_len)
         rc = lib.dpara_cache_append(C.byref(self.io), self.workspace.data_ptr(), self.workspace.numel(), self.status.data_ptr(),
                                     _stream_ptr(stream))
+        if rc != OK:
+            raise DparaError(rc)
+
+
+# ----------------------------------------------------------------------------- stack of backbone blocks
+class BackboneIO(C.Structure):
+    _fields_ = [("n_layers", C.c_int32), ("host_layers", C.c_void_p), ("host_k_ctx", C.c_void_p), ("host_v_ctx", C.c_void_p)]
+
+
+lib.dpara_backbone_workspace_bytes.restype = C.c_size_t
+lib.dpara_backbone_workspace_bytes.argtypes = [C.POINTER(Shape), C.c_void_p, C.POINTER(BackboneIO)]
+lib.dpara_draft_backbone.restype = C.c_int
+lib.dpara_draft_backbone.argtypes = [C.POINTER(Shape), C.POINTER(AttnIO), C.POINTER(BackboneIO), C.c_void_p, C.c_size_t, C.c_void_p,
+                                     C.c_void_p]
+EXPORTED += ["dpara_backbone_workspace_bytes", "dpara_draft_backbone"]
+
+
+class BackbonePlan:
+    """dpara_draft_backbone for fixed shapes, weights and caches: a stack of blocks with the spine tokens as query rows.
+    layers: LayerIO per block (make_layer_io; x of the first and y_f32 / y_bf16 of the last are the call's input and
+    outputs, [b][J*Bq + S][hidden]); k_ctx / v_ctx: one cache tensor per block."""
+
+    def __init__(self, *, ctx_offsets: Sequence[int], n_boundaries: int, block: int, n_q_heads: int, n_kv_heads: int, head_dim: int,
+                 layers: Sequence[LayerIO], k_ctx: Sequence[torch.Tensor], v_ctx: Sequence[torch.Tensor], prefix_base: int = 1,
+                 n_spine: Optional[int] = None, ctx_lens: Optional[Sequence[int]] = None, spine_queries: bool = True, device="cuda"):
+        b = len(ctx_offsets) - 1
+        nl = len(layers)
+        self.shape = Shape(b, n_boundaries, block, n_q_heads, n_kv_heads, head_dim, prefix_base,
+                           n_boundaries if n_spine is None else n_spine, 0, n_boundaries, 0.0, 1 if spine_queries else 0)
+        self.host_off = _host_offsets(ctx_offsets)
+        self.dev_off = torch.tensor([int(x) for x in ctx_offsets], dtype=torch.int64, device=device)
+        self.host_lens = self.dev_lens = None
+        if ctx_lens is not None:
+            self.host_lens = (C.c_int64 * b)(*[int(x) for x in ctx_lens])
+            self.dev_lens = torch.tensor([int(x) for x in ctx_lens], dtype=torch.int64, device=device)
+        self._keep = (list(k_ctx), list(v_ctx))
+        self.layers = (LayerIO * nl)(*layers)
+        self.kc = (C.c_void_p * nl)(*[_ptr(t) for t in k_ctx])
+        self.vc = (C.c_void_p * nl)(*[_ptr(t) for t in v_ctx])
+        self.bb = BackboneIO(nl, C.cast(self.layers, C.c_void_p).value, C.cast(self.kc, C.c_void_p).value, C.cast(self.vc, C.c_void_p).value)
+        self.workspace_bytes = int(lib.dpara_backbone_workspace_bytes(C.byref(self.shape), C.cast(self.host_off, C.c_void_p), C.byref(self.bb)))
+        self.workspace = torch.empty(max(self.workspace_bytes, 16), dtype=torch.uint8, device=device)
+        self.status = torch.zeros(1, dtype=torch.int32, device=device)
+
+    def __call__(self, *, k_spine=None, v_spine=None, stream=None) -> None:
+        io = AttnIO(None, None, None, self.dev_off.data_ptr(), C.cast(self.host_off, C.c_void_p).value, _ptr(k_spine), _ptr(v_spine),
+                    None, None, None, BF16, None, _ptr(self.dev_lens),
+                    C.cast(self.host_lens, C.c_void_p).value if self.host_lens is not None else None)
+        rc = lib.dpara_draft_backbone(C.byref(self.shape), C.byref(io), C.byref(self.bb), self.workspace.data_ptr(),
+                                      self.workspace.numel(), self.status.data_ptr(), _stream_ptr(stream))
         if rc != OK:
             raise DparaError(rc)

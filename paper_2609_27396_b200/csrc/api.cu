@@ -73,7 +73,8 @@ extern "C" dpara_status dpara_draft_all_boundaries(const dpara_shape *shape, con
       if (io->host_ctx_lens[n] < 0 || io->host_ctx_lens[n] > io->host_ctx_offsets[n + 1] - io->host_ctx_offsets[n]) return DPARA_ERR_INVALID_ARG;
   const bool has_ctx = io->host_ctx_offsets[shape->batch] > 0;
   if (has_ctx && (!io->k_ctx || !io->v_ctx)) return DPARA_ERR_INVALID_ARG;
-  if (shape->n_spine > 0 && (!io->k_spine || !io->v_spine)) return DPARA_ERR_INVALID_ARG;
+  const bool spine_made_inside = layer && shape->spine_queries;  // a block with spine query rows produces the spine's keys/values
+  if (shape->n_spine > 0 && !spine_made_inside && (!io->k_spine || !io->v_spine)) return DPARA_ERR_INVALID_ARG;
   if ((io->k_blk == nullptr) != (io->v_blk == nullptr)) return DPARA_ERR_INVALID_ARG;
   if (io->out_dtype != DPARA_BF16 && io->out_dtype != DPARA_F32) return DPARA_ERR_INVALID_ARG;
   if (!aligned16(io->k_ctx) || !aligned16(io->v_ctx) || !aligned16(io->k_spine) || !aligned16(io->v_spine) ||
@@ -87,6 +88,37 @@ extern "C" dpara_status dpara_draft_all_boundaries(const dpara_shape *shape, con
 
   if (!io->q || !io->out) return DPARA_ERR_INVALID_ARG;
   return launch_attention(shape, io, workspace, status_word, st);
+}
+
+extern "C" size_t dpara_backbone_workspace_bytes(const dpara_shape *shape, const int64_t *host_ctx_offsets, const dpara_backbone_io *bb) {
+  if (validate_shape(shape) != DPARA_OK || validate_offsets(shape, host_ctx_offsets) != DPARA_OK) return 0;
+  if (!bb || bb->n_layers <= 0 || !bb->host_layers || bb->host_layers[0].hidden <= 0 || bb->host_layers[0].intermediate <= 0) return 0;
+  return backbone_workspace_bytes(shape, host_ctx_offsets, bb);
+}
+
+extern "C" dpara_status dpara_draft_backbone(const dpara_shape *shape, const dpara_attn_io *io, const dpara_backbone_io *bb,
+                                             void *workspace, size_t workspace_bytes, int32_t *status_word, void *stream) {
+  dpara_status s = validate_shape(shape);
+  if (s != DPARA_OK) return s;
+  if (!io || !bb || bb->n_layers <= 0 || !bb->host_layers || !bb->host_k_ctx || !bb->host_v_ctx) return DPARA_ERR_INVALID_ARG;
+  s = validate_offsets(shape, io->host_ctx_offsets);
+  if (s != DPARA_OK) return s;
+  if (!io->ctx_offsets || (io->ctx_lens == nullptr) != (io->host_ctx_lens == nullptr)) return DPARA_ERR_INVALID_ARG;
+  if (io->host_ctx_lens)
+    for (int n = 0; n < shape->batch; ++n)
+      if (io->host_ctx_lens[n] < 0 || io->host_ctx_lens[n] > io->host_ctx_offsets[n + 1] - io->host_ctx_offsets[n]) return DPARA_ERR_INVALID_ARG;
+  if (shape->n_spine > 0 && !shape->spine_queries && (!io->k_spine || !io->v_spine)) return DPARA_ERR_INVALID_ARG;
+  const bool has_ctx = io->host_ctx_offsets[shape->batch] > 0;
+  for (int l = 0; l < bb->n_layers; ++l) {
+    if (bb->host_layers[l].hidden != bb->host_layers[0].hidden || bb->host_layers[l].intermediate != bb->host_layers[0].intermediate)
+      return DPARA_ERR_INVALID_ARG;
+    if (has_ctx && (!bb->host_k_ctx[l] || !bb->host_v_ctx[l] || !aligned16(bb->host_k_ctx[l]) || !aligned16(bb->host_v_ctx[l])))
+      return DPARA_ERR_INVALID_ARG;
+  }
+  if (!bb->host_layers[0].x || !bb->host_layers[bb->n_layers - 1].y_f32) return DPARA_ERR_INVALID_ARG;
+  const size_t need = dpara_backbone_workspace_bytes(shape, io->host_ctx_offsets, bb);
+  if (need == 0 || !workspace || workspace_bytes < need || !aligned16(workspace)) return DPARA_ERR_WORKSPACE;
+  return launch_backbone(shape, io, bb, workspace, status_word, static_cast<cudaStream_t>(stream));
 }
 
 extern "C" const char *dpara_status_string(dpara_status s) {

@@ -36,9 +36,11 @@ size_t attention_workspace_bytes(const dpara_shape *shape, const int64_t *host_o
 }
 
 dpara_status launch_attention(const dpara_shape *shape, const dpara_attn_io *io, void *workspace, int32_t *status_word,
-                              cudaStream_t st) {
+                              cudaStream_t st, int blk_req_rows, int spine_req_rows) {
   AttnParams P;
   fill_attn_params(P, shape, io, status_word);
+  if (blk_req_rows) P.blk_req_rows = blk_req_rows;
+  if (spine_req_rows) P.spine_req_rows = spine_req_rows;
   if (P.hi <= P.lo) return DPARA_OK;
   TcPlan plan = plan_attention_tc(shape, io->host_ctx_offsets, io->host_ctx_lens);
   if (!plan.eligible) return DPARA_ERR_UNSUPPORTED;  // group size > 16, block > 64, spine > 64, or more than 2^31 rows

@@ -75,12 +75,13 @@ __global__ void __launch_bounds__(128) rmsnorm_kernel(const void *__restrict__ x
 // (rounded to bf16), then rotate-half rotary embedding at the row's position (rounded to bf16).
 // Positions: slot i of boundary j of request n sits at L_n + j + 2 + i (spine row s at L_n + s, the
 // unknown bonus of boundary j at L_n + j + 1).  Angles are formed in double precision.
+// With spine query rows a request has J * Bq + S rows: the mask-slot rows, then the spine rows.
 struct QkParams {
   const uint16_t *qkv;
   const uint16_t *qnorm_w, *knorm_w;
   uint16_t *q, *k, *v;
   const int64_t *ctx_offsets, *ctx_lens;
-  int J, Bq, Hq, Hkv, D;
+  int J, Bq, Hq, Hkv, D, Sq;
   int use_rope, use_norm;
   float eps, theta;
 };
@@ -89,9 +90,11 @@ __global__ void __launch_bounds__(128) qk_norm_rope_kernel(const QkParams P) {
   extern __shared__ float s_cs[];  // cos[D/2], sin[D/2]
   const int row = blockIdx.x, tid = threadIdx.x;
   const int half = P.D / 2;
-  const int i = row % P.Bq, j = (row / P.Bq) % P.J, n = row / (P.Bq * P.J);
+  const int R = P.Bq * P.J + P.Sq;
+  const int n = row / R, rr = row % R;
   if (P.use_rope) {
-    const double pos = (double)(P.ctx_lens ? P.ctx_lens[n] : P.ctx_offsets[n + 1] - P.ctx_offsets[n]) + j + 2 + i;
+    const int rel = rr < P.Bq * P.J ? rr / P.Bq + 2 + rr % P.Bq : rr - P.Bq * P.J;  // mask slot (j, i): j + 2 + i; spine row s: s
+    const double pos = (double)(P.ctx_lens ? P.ctx_lens[n] : P.ctx_offsets[n + 1] - P.ctx_offsets[n]) + rel;
     for (int d = tid; d < half; d += 128) {
       const double inv = pow((double)P.theta, -2.0 * d / P.D);
       double sn, cs;
@@ -153,7 +156,7 @@ struct LayerWs {
 };
 
 LayerWs layer_ws_layout(const dpara_shape *s, const dpara_layer_io *l, size_t attn_bytes) {
-  const size_t M = (size_t)s->batch * s->n_boundaries * s->block;
+  const size_t M = (size_t)s->batch * (s->n_boundaries * s->block + (s->spine_queries ? s->n_spine : 0));
   const size_t H = l->hidden, I = l->intermediate, QD = (size_t)s->n_q_heads * s->head_dim, KD = (size_t)s->n_kv_heads * s->head_dim;
   LayerWs w;
   size_t o = 0;
@@ -198,7 +201,9 @@ dpara_status launch_layer(const dpara_shape *shape, const dpara_attn_io *io, con
   if (L->hidden <= 0 || L->intermediate <= 0) return DPARA_ERR_INVALID_ARG;
   if ((L->qnorm_w == nullptr) != (L->knorm_w == nullptr)) return DPARA_ERR_INVALID_ARG;
   if (shape->boundary_lo != 0 || shape->boundary_hi != shape->n_boundaries) return DPARA_ERR_UNSUPPORTED;
-  const int M = shape->batch * shape->n_boundaries * shape->block;
+  const int Sq = shape->spine_queries ? shape->n_spine : 0;
+  const int R = shape->n_boundaries * shape->block + Sq;  // rows per request: mask slots, then (if they are queries) the spine
+  const int M = shape->batch * R;
   const int H = L->hidden, I = L->intermediate, D = shape->head_dim;
   const int QD = shape->n_q_heads * D, KD = shape->n_kv_heads * D;
   if (H % 64 || I % 64 || QD % 64 || H % 8) return DPARA_ERR_UNSUPPORTED;
@@ -223,7 +228,7 @@ dpara_status launch_layer(const dpara_shape *shape, const dpara_attn_io *io, con
   QkParams qp;
   qp.qkv = qkv; qp.qnorm_w = static_cast<const uint16_t *>(L->qnorm_w); qp.knorm_w = static_cast<const uint16_t *>(L->knorm_w);
   qp.q = q; qp.k = k; qp.v = v; qp.ctx_offsets = io->ctx_offsets; qp.ctx_lens = io->ctx_lens;
-  qp.J = shape->n_boundaries; qp.Bq = shape->block; qp.Hq = shape->n_q_heads; qp.Hkv = shape->n_kv_heads; qp.D = D;
+  qp.J = shape->n_boundaries; qp.Bq = shape->block; qp.Hq = shape->n_q_heads; qp.Hkv = shape->n_kv_heads; qp.D = D; qp.Sq = Sq;
   qp.use_rope = L->use_rope; qp.use_norm = L->qnorm_w != nullptr; qp.eps = L->rms_eps; qp.theta = L->rope_theta;
   qk_norm_rope_kernel<<<M, 128, D * sizeof(float), st>>>(qp);
   DPARA_CHECK_LAUNCH();
@@ -231,7 +236,12 @@ dpara_status launch_layer(const dpara_shape *shape, const dpara_attn_io *io, con
 
   dpara_attn_io aio = *io;
   aio.q = q; aio.k_blk = k; aio.v_blk = v; aio.out = a; aio.out_dtype = DPARA_BF16; aio.out_lse = nullptr;
-  s = launch_attention(shape, &aio, base, status_word, st);
+  if (Sq) {
+    // the spine's keys/values are the block's own: rows J * Bq .. of each request in the k / v buffers
+    aio.k_spine = k + (size_t)shape->n_boundaries * shape->block * KD;
+    aio.v_spine = v + (size_t)shape->n_boundaries * shape->block * KD;
+  }
+  s = launch_attention(shape, &aio, base, status_word, st, Sq ? R : 0, Sq ? R : 0);
   if (s != DPARA_OK) return s;
 
   g = GemmArgs{};
@@ -248,6 +258,48 @@ dpara_status launch_layer(const dpara_shape *shape, const dpara_attn_io *io, con
   g = GemmArgs{};
   g.a = act; g.w = L->w_down; g.M = M; g.N = H; g.K = I; g.epi = 1; g.resid = h1; g.resid_bf16 = 0; g.out = L->y_f32; g.out_bf16 = L->y_bf16;
   return launch_gemm_tc(g, status_word, st);
+}
+
+// ------------------------------------------------------------------------------------------------ stack of blocks
+namespace {
+struct BackboneWs { size_t x0, x1, yf, layer, total; };
+BackboneWs backbone_ws_layout(const dpara_shape *s, const dpara_backbone_io *bb, size_t attn_bytes) {
+  const size_t M = (size_t)s->batch * (s->n_boundaries * s->block + (s->spine_queries ? s->n_spine : 0));
+  const size_t H = bb->host_layers[0].hidden;
+  BackboneWs w;
+  size_t o = 0;
+  auto take = [&](size_t bytes) { size_t r = o; o += align_up(bytes, 256); return r; };
+  w.layer = take(attn_bytes + layer_workspace_bytes(s, &bb->host_layers[0]));  // the attention scratch leads the block's scratch
+  w.x0 = take(M * H * 2);
+  w.x1 = take(M * H * 2);
+  w.yf = take(M * H * 4);
+  w.total = o;
+  return w;
+}
+}  // namespace
+
+size_t backbone_workspace_bytes(const dpara_shape *shape, const int64_t *host_ctx_offsets, const dpara_backbone_io *bb) {
+  return backbone_ws_layout(shape, bb, attention_workspace_bytes(shape, host_ctx_offsets)).total;
+}
+
+dpara_status launch_backbone(const dpara_shape *shape, const dpara_attn_io *io, const dpara_backbone_io *bb, void *workspace,
+                             int32_t *status_word, cudaStream_t st) {
+  const BackboneWs w = backbone_ws_layout(shape, bb, attention_workspace_bytes(shape, io->host_ctx_offsets));
+  uint8_t *base = static_cast<uint8_t *>(workspace);
+  void *xbuf[2] = {base + w.x0, base + w.x1};
+  const int last = bb->n_layers - 1;
+  for (int l = 0; l <= last; ++l) {
+    dpara_layer_io L = bb->host_layers[l];
+    L.x = l == 0 ? bb->host_layers[0].x : xbuf[(l - 1) & 1];
+    L.y_f32 = l == last ? bb->host_layers[last].y_f32 : reinterpret_cast<float *>(base + w.yf);
+    L.y_bf16 = l == last ? bb->host_layers[last].y_bf16 : xbuf[l & 1];
+    dpara_attn_io a = *io;
+    a.k_ctx = bb->host_k_ctx[l];
+    a.v_ctx = bb->host_v_ctx[l];
+    dpara_status s = launch_layer(shape, &a, &L, base + w.layer, status_word, st);
+    if (s != DPARA_OK) return s;
+  }
+  return DPARA_OK;
 }
 
 }  // namespace dpara

@@ -38,9 +38,9 @@ __device__ __forceinline__ unsigned long long warp_sum_u64(unsigned long long v)
 }
 
 // Copy of the selected branch: reps[n][r] -> selected[n], `bytes` per request.
-__device__ __forceinline__ void gather_branch(const uint8_t *__restrict__ reps, uint8_t *__restrict__ selected, int n, int J,
-                                              int r, size_t bytes, int tid, int nthreads) {
-  const uint8_t *src = reps + ((size_t)n * J + r) * bytes;
+__device__ __forceinline__ void gather_branch(const uint8_t *__restrict__ reps, uint8_t *__restrict__ selected, int n,
+                                              size_t req_bytes, int r, size_t bytes, int tid, int nthreads) {
+  const uint8_t *src = reps + (size_t)n * req_bytes + (size_t)r * bytes;
   uint8_t *dst = selected + (size_t)n * bytes;
   if ((bytes & 15) == 0 && ((reinterpret_cast<uintptr_t>(src) | reinterpret_cast<uintptr_t>(dst)) & 15) == 0) {
     const uint4 *s = reinterpret_cast<const uint4 *>(src);
@@ -77,6 +77,7 @@ struct VerifyParams {
   unsigned long long *masks; // greedy: [b] completed-row masks
   int b, J, V, nchunks, vec_ok;
   size_t rep_bytes;  // Bq * hidden * 2
+  size_t req_bytes;  // from one request's representations to the next request's (J * rep_bytes when packed)
 };
 
 // Outputs of request n, written by the first J threads of the finishing CTA.
@@ -227,7 +228,7 @@ __global__ void __launch_bounds__(kVsThreads, kGreedyLoads >= 16 ? 3 : (kGreedyL
       if (s_bad && P.status_word) atomicOr(reinterpret_cast<unsigned int *>(P.status_word), DPARA_STATUS_BAD_TOKEN);
     }
     if (P.out_tokens && tid < P.J) P.out_tokens[(size_t)n * P.J + tid] = tid < r ? s_t[tid] : (tid == r ? s_a[r] : -1);
-    if (P.reps) gather_branch(P.reps, P.selected, n, P.J, r, P.rep_bytes, tid, kVsThreads);
+    if (P.reps) gather_branch(P.reps, P.selected, n, P.req_bytes, r, P.rep_bytes, tid, kVsThreads);
   }
   // ---- leave the workspace as it was found.  Every row-completing CTA checks in here as its LAST access to
   // the workspace; a CTA that did not complete a row touched it last before its row counter moved, i.e. before
@@ -440,7 +441,7 @@ __global__ void __launch_bounds__(kVsThreads) verify_sampling_kernel(const Verif
   __syncthreads();
   for (int i = tid; i < 2 * P.nchunks; i += kVsThreads) P.ws64[(size_t)n * P.nchunks * 2 + i] = 0ull;
   if (tid == 0) P.counters[n] = 0u;
-  if (P.reps) gather_branch(P.reps, P.selected, n, P.J, r, P.rep_bytes, tid, kVsThreads);
+  if (P.reps) gather_branch(P.reps, P.selected, n, P.req_bytes, r, P.rep_bytes, tid, kVsThreads);
 }
 
 // Greedy: 16-byte loads in flight per thread.  As many as possible (fewer, larger CTAs amortise the reduction
@@ -481,6 +482,7 @@ static dpara_status validate_verify(const dpara_verify_io *io) {
   if (io->mode == 1 && (!io->uniforms || (io->n_boundaries > 1 && !io->draft_probs))) return DPARA_ERR_INVALID_ARG;
   if (io->reps) {
     if (!io->selected || io->block <= 0 || io->hidden <= 0) return DPARA_ERR_INVALID_ARG;
+    if (io->rep_req_rows < 0 || (io->rep_req_rows > 0 && io->rep_req_rows < io->n_boundaries * io->block)) return DPARA_ERR_INVALID_ARG;
   }
   return DPARA_OK;
 }
@@ -515,6 +517,7 @@ dpara_status launch_verify(const dpara_verify_io *io, void *ws, int32_t *status_
   P.V = io->vocab;
   P.nchunks = chunks_of(io);
   P.rep_bytes = (size_t)io->block * io->hidden * 2;
+  P.req_bytes = io->rep_req_rows > 0 ? (size_t)io->rep_req_rows * io->hidden * 2 : (size_t)io->n_boundaries * P.rep_bytes;
   size_t n64 = ws64_count(io);
   const size_t mask_off = align_up(n64 * 8, 256);
   const size_t cnt_off = mask_off + align_up((size_t)io->batch * 8, 256);
