@@ -31,9 +31,15 @@ import workloads as W  # noqa: E402
 
 METRIC = "all_boundary_draft_step_us"
 L2_FLUSH_BYTES = 256 << 20
-# dram__bytes_read.sum + dram__bytes_write.sum of one attention launch, from an ncu capture of this command's
-# workload (bytes per launch; None where no capture exists)
-NCU_DRAM_TRAFFIC = {"cfg3": 369188608, "cfg2": None}
+
+
+def ncu_dram_traffic(workload: str):
+    """dram__bytes_read.sum + dram__bytes_write.sum of one attention launch of this workload, as recorded from an ncu
+    capture in profiles/traffic.json (bytes per launch; None where no capture exists)."""
+    try:
+        return json.load(open(os.path.join(ROOT, "profiles", "traffic.json")))["attention"][workload]["dram_bytes_per_launch"]
+    except Exception:
+        return None
 
 
 # ----------------------------------------------------------------------------- algorithmic work (flops and bytes every launch must do)
@@ -209,6 +215,7 @@ class LayerRunner:
         lin = W.make_layer_inputs(l, a, seed)
         ver = W.make_verify_inputs(v, seed, reps=np.zeros((1,), np.uint16))
         bf = lambda bits: torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda().view(torch.bfloat16)
+        self.attn, self.layer, self.ctx_offsets = a, l, [int(x) for x in ain.ctx_offsets]
         self.t = {k: bf(getattr(lin, k)) for k in ("x", "w_qkv", "w_o", "w_gate_up", "w_down", "rms1_w", "rms2_w", "qnorm_w", "knorm_w")}
         self.kv = {k: bf(getattr(ain, k)) for k in ("k_ctx", "v_ctx", "k_spine", "v_spine")}
         self.y = torch.zeros((a.batch, a.n_boundaries, a.block, l.hidden), dtype=torch.float32, device="cuda")
@@ -238,6 +245,182 @@ class LayerRunner:
             ev[s][2].record()
         torch.cuda.synchronize()
         return [(e[0].elapsed_time(e[2]), e[0].elapsed_time(e[1]), e[1].elapsed_time(e[2])) for e in ev]
+
+
+def _median_us(fn, k, flush):
+    import torch
+    ts = []
+    for _ in range(3):
+        fn()
+    for _ in range(k):
+        flush.zero_()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(); fn(); e1.record()
+        torch.cuda.synchronize()
+        ts.append(e0.elapsed_time(e1) * 1e3)
+    return statistics.median(ts)
+
+
+def _layer_attention_only_us(self, k: int) -> float:
+    """The all-boundary attention of the full-layer workload on its own (random q / block keys of the right shape)."""
+    import torch
+    import paper_2609_27396_b200 as dp
+    a = self.attn
+    g = torch.Generator(device="cuda").manual_seed(1)
+    mk = lambda *sh: torch.randn(*sh, device="cuda", generator=g).to(torch.bfloat16)
+    q, kb, vb = mk(a.batch, a.n_boundaries, a.block, a.n_q_heads, a.head_dim), mk(a.batch, a.n_boundaries, a.block, a.n_kv_heads, a.head_dim), mk(a.batch, a.n_boundaries, a.block, a.n_kv_heads, a.head_dim)
+    out = torch.zeros_like(q)
+    plan = dp.DraftPlan(ctx_offsets=self.ctx_offsets, n_boundaries=a.n_boundaries, block=a.block, n_q_heads=a.n_q_heads,
+                        n_kv_heads=a.n_kv_heads, head_dim=a.head_dim, prefix_base=a.prefix_base, n_spine=a.spine)
+    return _median_us(lambda: plan(q=q, **self.kv, k_blk=kb, v_blk=vb, out=out), k, self.flush)
+
+
+def _layer_gemm_legs(self, peaks, k: int):
+    """Each projection of the block on its own (dpara_gemm_bf16 at the block's shapes)."""
+    import torch
+    import paper_2609_27396_b200 as dp
+    a, l = self.attn, self.layer
+    M = a.batch * a.n_boundaries * a.block
+    qd, kd = a.n_q_heads * a.head_dim, a.n_kv_heads * a.head_dim
+    g = torch.Generator(device="cuda").manual_seed(2)
+    act = lambda K: torch.randn(M, K, device="cuda", generator=g).to(torch.bfloat16)
+    res = {}
+    for name, w, K, N, epi in (("qkv", self.t["w_qkv"], l.hidden, qd + 2 * kd, 0), ("o", self.t["w_o"], qd, l.hidden, 1),
+                               ("gate_up", self.t["w_gate_up"], l.hidden, l.intermediate, 2), ("down", self.t["w_down"], l.intermediate, l.hidden, 1)):
+        x = act(K)
+        resid = torch.zeros(M, N, dtype=torch.float32, device="cuda") if epi == 1 else None
+        us = _median_us(lambda: dp.gemm_bf16(x, w, epilogue=epi, resid=resid), k, self.flush)
+        fl = 2.0 * M * K * N * (2 if epi == 2 else 1)
+        res[name] = {"M": M, "N": N, "K": K, "us": us, "tflops": fl / (us * 1e-6) / 1e12, "frac_of_measured_burst": fl / (us * 1e-6) / 1e12 / peaks["bf16_tflops"]}
+    return res
+
+
+LayerRunner.attention_only_us = _layer_attention_only_us
+LayerRunner.gemm_legs = _layer_gemm_legs
+
+
+def backbone_leg(w5: W.Workload, peaks, k: int):
+    """Two stacked blocks with the spine tokens as query rows (dpara_draft_backbone) at the full-layer workload's shapes:
+    M = b * (J * Bq + S) rows per block, each block with its own 32 K-token context cache."""
+    import torch
+    import paper_2609_27396_b200 as dp
+    a, l = w5.attn, w5.layer
+    n_layers = 2
+    R = a.n_boundaries * a.block + a.spine
+    g = torch.Generator(device="cuda").manual_seed(3)
+    mk = lambda sig, *sh: (torch.randn(*sh, device="cuda", generator=g) * sig).to(torch.bfloat16)
+    off = [0]
+    for L in a.ctx_lens:
+        off.append(off[-1] + L)
+    x = mk(1.0, a.batch, R, l.hidden)
+    y = torch.zeros(a.batch, R, l.hidden, dtype=torch.float32, device="cuda")
+    y16 = torch.zeros(a.batch, R, l.hidden, dtype=torch.bfloat16, device="cuda")
+    qd, kd = a.n_q_heads * a.head_dim, a.n_kv_heads * a.head_dim
+    layers, keep, kc, vc = [], [], [], []
+    for _ in range(n_layers):
+        t = dict(w_qkv=mk(l.weight_sigma, qd + 2 * kd, l.hidden), w_o=mk(l.weight_sigma, l.hidden, qd),
+                 w_gate_up=mk(l.weight_sigma, 2 * l.intermediate, l.hidden), w_down=mk(l.weight_sigma, l.hidden, l.intermediate),
+                 rms1_w=torch.ones(l.hidden, dtype=torch.bfloat16, device="cuda"), rms2_w=torch.ones(l.hidden, dtype=torch.bfloat16, device="cuda"),
+                 qnorm_w=torch.ones(a.head_dim, dtype=torch.bfloat16, device="cuda"), knorm_w=torch.ones(a.head_dim, dtype=torch.bfloat16, device="cuda"))
+        keep.append(t)
+        layers.append(dp.make_layer_io(x=x, **t, rms_eps=l.rms_eps, rope_theta=l.rope_theta, use_rope=True, y_f32=y, y_bf16=y16))
+        kc.append(mk(1.0, off[-1], a.n_kv_heads, a.head_dim)); vc.append(mk(1.0, off[-1], a.n_kv_heads, a.head_dim))
+    plan = dp.BackbonePlan(ctx_offsets=off, n_boundaries=a.n_boundaries, block=a.block, n_q_heads=a.n_q_heads, n_kv_heads=a.n_kv_heads,
+                           head_dim=a.head_dim, layers=layers, k_ctx=kc, v_ctx=vc, prefix_base=a.prefix_base, n_spine=a.spine)
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device="cuda")
+    us = _median_us(lambda: plan(), k, flush)
+    M = a.batch * R
+    rows_fl = 0.0
+    for L in a.ctx_lens:
+        for j in range(a.n_boundaries):
+            rows_fl += 4.0 * a.head_dim * a.block * a.n_q_heads * (L + min(j + a.prefix_base, a.spine) + a.block)
+        for s_ in range(a.spine):
+            rows_fl += 4.0 * a.head_dim * a.n_q_heads * (L + s_ + 1)
+    fl = n_layers * (rows_fl + 2.0 * M * (l.hidden * (qd + 2 * kd) + qd * l.hidden + 3 * l.hidden * l.intermediate))
+    return {"workload": f"{n_layers} blocks, spine tokens as query rows, {w5.name} shapes: M = {M} rows per block", "us": us, "us_per_block": us / n_layers,
+            "flops": fl, "tflops": fl / (us * 1e-6) / 1e12, "tensor_frac_of_measured_burst": fl / (us * 1e-6) / 1e12 / peaks["bf16_tflops"]}
+
+
+def small_step_leg(index: int, k: int):
+    w = W.workload(index)
+    r = StepRunner(w, w.seed)
+    for _ in range(5):
+        r.step()
+    p = r.timed_steps(k)
+    return {"workload": w.name, "step_us": statistics.median(x[0] for x in p) * 1e3, "attention_us": statistics.median(x[1] for x in p) * 1e3,
+            "verify_select_us": statistics.median(x[2] for x in p) * 1e3}
+
+
+def sampling_select_leg(peaks, k: int):
+    """Rejection-sampling verify/select (cfg4).  Algorithmic bytes: the 2 * gamma scalars of the accept tests plus rows p_r
+    and q_r of each request and the gathered branch (read + write) -- not the whole probability tensors."""
+    import torch
+    import paper_2609_27396_b200 as dp
+    w = W.workload(4)
+    v = w.verify
+    ver = W.make_verify_inputs(v, w.seed)
+    bf = lambda bits: torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda().view(torch.bfloat16)
+    t = dict(target=torch.from_numpy(ver.target).cuda(), draft_tokens=torch.from_numpy(ver.draft_tokens).cuda(), reps=bf(ver.reps),
+             draft_probs=torch.from_numpy(ver.draft_probs).cuda(), uniforms=torch.from_numpy(ver.uniforms).cuda())
+    plan = dp.VerifyPlan(batch=v.batch, n_boundaries=v.n_boundaries, vocab=v.vocab, block=v.block, hidden=v.hidden, mode=1)
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device="cuda")
+    us = _median_us(lambda: plan(**t), k, flush)
+    by = v.batch * (2 * v.vocab * 4 + 2 * v.block * v.hidden * 2)
+    return {"workload": w.name, "us": us, "algorithmic_bytes": by, "gbs": by / (us * 1e-6) / 1e9, "frac_of_measured_hbm": by / (us * 1e-6) / 1e9 / peaks["hbm_gbs"],
+            "bound": "latency (9.7 MB)"}
+
+
+def cache_append_leg(wl: W.Workload, peaks, k: int, n_layers: int = 5):
+    """Feature-cache append (dpara_cache_append) at the main workload's shapes: b requests x J candidate rows of `hidden`
+    features into the caches of n_layers drafter layers.  Algorithmic bytes: each layer's [keys | values] projection once."""
+    import torch
+    import paper_2609_27396_b200 as dp
+    a, v = wl.attn, wl.verify
+    J, F, Hkv, D = a.n_boundaries, v.hidden, a.n_kv_heads, a.head_dim
+    g = torch.Generator(device="cuda").manual_seed(4)
+    mk = lambda sig, *sh: (torch.randn(*sh, device="cuda", generator=g) * sig).to(torch.bfloat16)
+    cap = [L + 4 * J for L in a.ctx_lens]
+    start = [0]
+    for c in cap[:-1]:
+        start.append(start[-1] + c)
+    rows = sum(cap)
+    kc = [torch.zeros(rows, Hkv, D, dtype=torch.bfloat16, device="cuda") for _ in range(n_layers)]
+    vc = [torch.zeros(rows, Hkv, D, dtype=torch.bfloat16, device="cuda") for _ in range(n_layers)]
+    lens0 = torch.tensor(list(a.ctx_lens), dtype=torch.int64, device="cuda")
+    lens = lens0.clone()
+    plan = dp.CachePlan(batch=a.batch, n_rows=J, w_kv=[mk(0.02, 2 * Hkv * D, F) for _ in range(n_layers)], k_ctx=kc, v_ctx=vc,
+                        row_start=torch.tensor(start, dtype=torch.int64, device="cuda"), capacity=torch.tensor(cap, dtype=torch.int64, device="cuda"),
+                        ctx_len=lens, norm_w=[torch.ones(F, dtype=torch.bfloat16, device="cuda")] * n_layers,
+                        knorm_w=[torch.ones(D, dtype=torch.bfloat16, device="cuda") for _ in range(n_layers)])
+    feats = mk(1.0, a.batch, J, F)
+    acc = torch.randint(0, J, (a.batch,), device="cuda", generator=g).to(torch.int32)
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device="cuda")
+
+    def call():
+        lens.copy_(lens0)             # (a device-to-device copy of b lengths: keeps every timed call at the same fill level)
+        plan.run(feats, acc)
+    us = _median_us(call, k, flush)
+    by = n_layers * 2 * Hkv * D * F * 2 + a.batch * J * F * 2
+    return {"workload": f"{wl.name} shapes: b={a.batch}, {J} candidate rows x {F} features, {n_layers} layers, Hkv={Hkv}, D={D}", "us": us,
+            "us_per_layer": us / n_layers, "algorithmic_bytes": by, "gbs": by / (us * 1e-6) / 1e9,
+            "frac_of_measured_hbm": by / (us * 1e-6) / 1e9 / peaks["hbm_gbs"]}
+
+
+def parity_spot_check(run: "StepRunner", n_rows: int = 64):
+    """max |delta| of the timed attention output against the oracle on a few seeded rows of the bench workload (the
+    GPU tests check 4096 rows; this ties the timed configuration to the oracle inside the bench run itself)."""
+    from oracle import attention as OA
+    a = run.wl.attn
+    rng = np.random.default_rng(7)
+    rows = [(int(rng.integers(a.batch)), int(rng.integers(a.n_boundaries)), int(rng.integers(a.block)), int(rng.integers(a.n_q_heads)))
+            for _ in range(n_rows)]
+    i = run.inp
+    ref = OA.draft_rows(i.q, i.k_ctx, i.v_ctx, i.ctx_offsets, i.k_spine, i.v_spine, i.k_blk, i.v_blk, rows, prefix_base=a.prefix_base)
+    run.attention()
+    run.torch.cuda.synchronize()
+    o = run.out.float().cpu().numpy()
+    got = np.stack([o[n, j, s_, h] for (n, j, s_, h) in rows]).astype(np.float64)
+    return {"rows": n_rows, "attention_max_abs_delta": float(np.abs(got - ref).max()), "bound": 1e-2}
 
 
 class HeadRunner:
@@ -441,7 +624,7 @@ def main():
     by = attention_bytes(wl.attn)
     ach_tf = fl / (att_ms * 1e-3) / 1e12
     ach_gb = by / (att_ms * 1e-3) / 1e9
-    traffic = NCU_DRAM_TRAFFIC.get(args.workload)
+    traffic = ncu_dram_traffic(args.workload)
     roofline = {"kernel": "all-boundary attention", "bound": "tensor", "achieved": ach_tf, "peak": peaks["bf16_tflops"],
                 "unit": "TFLOP/s", "frac": ach_tf / peaks["bf16_tflops"], "traffic": traffic, "peak_source": peaks["source"] + " (burst)",
                 "hbm": {"achieved": ach_gb, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach_gb / peaks["hbm_gbs"],
@@ -483,8 +666,14 @@ def main():
             out["layer_cfg5"] = {"workload": w5.name, "step_us": statistics.median(p[0] for p in p5) * 1e3, "draft_layer_us": d5,
                                  "verify_select_us": statistics.median(p[2] for p in p5) * 1e3,
                                  "flops": fl5, "tflops": fl5 / (d5 * 1e-6) / 1e12,
-                                 "tensor_frac_of_measured_sustained": fl5 / (d5 * 1e-6) / 1e12 / (peaks["bf16_tflops_sustained"] or peaks["bf16_tflops"])}
+                                 "tensor_frac_of_measured_burst": fl5 / (d5 * 1e-6) / 1e12 / peaks["bf16_tflops"],
+                                 "tensor_frac_of_measured_sustained": fl5 / (d5 * 1e-6) / 1e12 / (peaks["bf16_tflops_sustained"] or peaks["bf16_tflops"]),
+                                 "attention_us": r5.attention_only_us(max(5, min(args.steps, 10))),
+                                 "attention_flops": attention_flops(w5.attn),
+                                 "gemms": r5.gemm_legs(peaks, max(5, min(args.steps, 10)))}
+            out["layer_cfg5"]["attention_tflops"] = attention_flops(w5.attn) / (out["layer_cfg5"]["attention_us"] * 1e-6) / 1e12
             del r5
+            out["backbone_cfg5"] = backbone_leg(w5, peaks, max(3, min(args.steps, 5)))
         if not args.no_head:
             rh = HeadRunner(wl, wl.seed)
             for _ in range(3):
@@ -501,6 +690,10 @@ def main():
                            "ar_loop": {"w_bytes_per_step": sh.vocab * sh.rank * 2, "hbm_bytes": arb,
                                        "w_read_gbs": sh.vocab * sh.rank * 2 * sh.block / ((th - tl) * 1e-6) / 1e9}}
             del rh
+        out["cfg1"] = small_step_leg(1, max(args.steps, 20))
+        out["cfg4_sampling_select"] = sampling_select_leg(peaks, max(args.steps, 20))
+        out["cache_append"] = cache_append_leg(wl, peaks, max(args.steps, 20))
+        out["parity_spot_check"] = parity_spot_check(run)
         if not args.no_cpu_baseline:
             t, est, desc = oracle_sample(wl, wl.seed, 0, wl.verify.batch, run.inp, run.ver)
             out["cpu_baseline"] = {"value": est * 1e6, "unit": "us", "cores": oracle_threads(), "kind": "oracle", "sample": desc,

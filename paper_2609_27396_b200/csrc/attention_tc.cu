@@ -45,6 +45,7 @@ constexpr float kRescaleLog2 = 8.0f;
 constexpr int kMaxOrdered = 128;
 constexpr int kMaxSched = 3072;  // items a host-built schedule can hold (kernel parameter space)
 constexpr int kMaxHeadBlocks = 4;  // G <= 16: at most four binary digits unless G == 16 (one block)
+constexpr int kMaxSeg = 224;       // segments of the cut schedule (groups + teams)
 constexpr int kMaxPairs = 256;     // 64 boundaries x 64 slots in tiles of 8 (j, i) rows = 512 tiles
 }  // namespace
 
@@ -84,6 +85,20 @@ struct TcParams {
   // time first, each item to the least loaded CTA); a ragged batch has few items per CTA (about five at the
   // benchmark shape), so handing them out round-robin leaves the most loaded CTA ~20 % above the mean.
   int use_sched;
+  // Cut schedule.  The X tile pairs of one (request, KV head) read the same K/V stream; run by X CTAs side by side (a
+  // TEAM: CTAs team * X .. team * X + X - 1, member x takes pair x) they stay in step and every K/V tile comes from HBM
+  // once and from L2 for the other members.  The host cuts the groups' key-tile ranges into CONTIGUOUS SEGMENTS of
+  // near-equal cost, one run of segments per team (team_first), so that all teams finish together whatever the number of
+  // groups (32 groups do not fill 37 teams otherwise, and a ragged batch does not balance).  A cut group's pieces leave
+  // unnormalised rows in scratch; when a CTA has finished its run it takes a ticket for each of its cut items, and
+  // whoever draws an item's last ticket merges the pieces and writes the output (no waiting).
+  int use_seg, seg_X, seg_teams;
+  struct Seg {
+    uint16_t group, t0, t1, slot0;  // (request, KV head) group; context tiles [t0, t1); scratch slot base of the group's piece 0
+    uint8_t piece, npieces, pad[2];
+  } seg[kMaxSeg];
+  uint16_t team_first[kNumSM + 1];
+  unsigned int *seg_count;  // [items] tickets, zeroed before the launch
   uint16_t cta_first[kNumSM + 1];
   uint16_t sched[kMaxSched];
 };
@@ -103,6 +118,7 @@ struct TcCfg {
 // One unit of work of a persistent CTA.
 struct Item {
   int n, g, pair, split, ntq, L, t0, t1, nctx, n_ctx_it, n_tail, n_iter, jb0, slot;
+  int npieces, slot0, item;    // KV pieces of the item (1: whole), scratch slot of piece 0, item id
   int blk, hs, h0, ji_t, ji0;  // head block, log2(heads per row group), first head, (j, i) rows per tile, first (j, i) row
   long long c0;
 };
@@ -166,7 +182,128 @@ __device__ __forceinline__ Item decode_item(const TcParams &P, int id) {
   I.n_tail = I.split == (1 << P.nsplit_log2) - 1 ? pi.n_tail : 0;
   I.n_iter = I.n_ctx_it + I.n_tail;
   I.slot = (((I.n * A.Hkv + I.g) * P.n_pairs + I.pair) << P.nsplit_log2) + I.split;
+  I.npieces = 1 << P.nsplit_log2;
+  I.slot0 = I.slot - I.split;
+  I.item = id;
   return I;
+}
+
+// Entry qi of this CTA's work list: a whole item (or one of its cluster splits), or a segment of a cut group.
+__device__ __forceinline__ Item fetch_item(const TcParams &P, int qi) {
+  if (!P.use_seg) return decode_item(P, P.use_sched ? (int)P.sched[qi] : qi);
+  const TcParams::Seg e = P.seg[qi];
+  const int x = (int)blockIdx.x % P.seg_X;  // this CTA's tile pair within its team
+  Item I = decode_item(P, (int)e.group * P.seg_X + x);
+  I.t0 = e.t0;
+  I.t1 = e.t1;
+  I.n_ctx_it = e.t1 - e.t0;
+  if (e.piece + 1 != e.npieces) I.n_tail = 0;  // the tail tiles go with the last piece
+  I.n_iter = I.n_ctx_it + I.n_tail;
+  I.split = e.piece;
+  I.npieces = e.npieces;
+  I.slot0 = (int)e.slot0 * P.seg_X + x * e.npieces;
+  I.slot = I.slot0 + e.piece;
+  return I;
+}
+
+// Merge of the KV pieces of an item: rows [row_begin, row_begin + n_rows) of the item's 256 (two tiles of 128; n_rows
+// divides 256).  Every piece has left its unnormalised rows and (max, sum) in its scratch slot (slot0 + piece); the caller
+// has made them visible.  A thread owns one row (its weights are worked out once) and walks over that row's 16-column
+// parts.  kNp = compile-time bound on the pieces (2, 4 or 8): every loop over pieces is fully unrolled and predicated, so
+// the loads of a part (of two parts when kNp = 2) are all in flight together.
+template <int D, int kNp>
+__device__ __forceinline__ void merge_pieces_n(const TcParams &P, const Item &I, int np, int row_begin, int n_rows, int tid) {
+  const AttnParams &A = P.a;
+  const float c = P.c_log2;
+  const size_t slot0 = (size_t)I.slot0;
+  constexpr int kParts = D / 16;
+  constexpr int kUnroll = kNp == 2 ? 2 : 1;  // parts whose loads are in flight together
+  const int R = row_begin + tid % n_rows;
+  const int t = R >> 7, r = R & 127;
+  const int ji = I.ji0 + t * I.ji_t + (r >> I.hs);
+  if (t >= I.ntq || ji >= P.n_rows) return;
+  const int h = I.g * A.G + I.h0 + (r & ((1 << I.hs) - 1));
+  const size_t orow = ((size_t)I.n * A.q_req_rows + A.lo * A.Bq + ji) * A.Hq + h;
+  // weights of the pieces for this row: exp2((m_piece - m) c) / sum; a piece without visible keys wrote no rows (its slot
+  // may hold anything) and gets weight 0
+  float2 ml[kNp];
+#pragma unroll
+  for (int sp = 0; sp < kNp; ++sp)
+    ml[sp] = sp < np ? __ldcg(P.part_ml + ((slot0 + sp) * 2 + t) * 128 + r) : make_float2(-INFINITY, 0.f);
+  float mmax = -INFINITY, lsum = 0.f, wgt[kNp];
+#pragma unroll
+  for (int sp = 0; sp < kNp; ++sp) if (ml[sp].y > 0.f) mmax = fmaxf(mmax, ml[sp].x);
+#pragma unroll
+  for (int sp = 0; sp < kNp; ++sp) {
+    wgt[sp] = ml[sp].y > 0.f ? ex2((ml[sp].x - mmax) * c) : 0.f;
+    lsum = fmaf(wgt[sp], ml[sp].y, lsum);
+  }
+  const float inv = lsum > 0.f ? 1.0f / lsum : 0.f;
+#pragma unroll
+  for (int sp = 0; sp < kNp; ++sp) wgt[sp] *= inv;
+  const int step = 256 / n_rows;
+  const float4 *po = reinterpret_cast<const float4 *>(P.part_o) + ((slot0 * 2 + t) * (D / 4)) * 128 + r;
+  constexpr size_t kPieceStride = (size_t)2 * (D / 4) * 128;  // float4 from one piece's tile to the next piece's
+  for (int part0 = tid / n_rows; part0 < kParts; part0 += step * kUnroll) {
+    float4 x[kUnroll][kNp < 4 ? kNp : 4][4];
+    float acc[kUnroll][16];
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u)
+#pragma unroll
+      for (int e = 0; e < 16; ++e) acc[u][e] = 0.f;
+#pragma unroll
+    for (int sp0 = 0; sp0 < kNp; sp0 += 4) {
+#pragma unroll
+      for (int u = 0; u < kUnroll; ++u) {
+        const int part = part0 + u * step;
+#pragma unroll
+        for (int q = 0; q < (kNp < 4 ? kNp : 4); ++q)
+#pragma unroll
+          for (int v = 0; v < 4; ++v)
+            x[u][q][v] = (sp0 + q < np && part < kParts) ? __ldcg(po + (size_t)(sp0 + q) * kPieceStride + (size_t)(part * 4 + v) * 128)
+                                                        : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+#pragma unroll
+      for (int u = 0; u < kUnroll; ++u)
+#pragma unroll
+        for (int q = 0; q < (kNp < 4 ? kNp : 4); ++q) {
+          const float w = wgt[sp0 + q];   // 0 for a piece that does not exist or saw no key: its (undefined) rows are not read above or weigh nothing
+#pragma unroll
+          for (int v = 0; v < 4; ++v) {
+            if (w > 0.f) {
+              acc[u][4 * v] = fmaf(w, x[u][q][v].x, acc[u][4 * v]);
+              acc[u][4 * v + 1] = fmaf(w, x[u][q][v].y, acc[u][4 * v + 1]);
+              acc[u][4 * v + 2] = fmaf(w, x[u][q][v].z, acc[u][4 * v + 2]);
+              acc[u][4 * v + 3] = fmaf(w, x[u][q][v].w, acc[u][4 * v + 3]);
+            }
+          }
+        }
+    }
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      const int part = part0 + u * step;
+      if (part >= kParts) break;
+      if (A.out_f32) {
+        float4 *dst = reinterpret_cast<float4 *>(static_cast<float *>(A.out) + orow * D + part * 16);
+#pragma unroll
+        for (int v = 0; v < 4; ++v) dst[v] = make_float4(acc[u][4 * v], acc[u][4 * v + 1], acc[u][4 * v + 2], acc[u][4 * v + 3]);
+      } else {
+        uint4 *dst = reinterpret_cast<uint4 *>(static_cast<uint16_t *>(A.out) + orow * D + part * 16);
+#pragma unroll
+        for (int v = 0; v < 2; ++v)
+          dst[v] = make_uint4(pack_bf16(acc[u][8 * v], acc[u][8 * v + 1]), pack_bf16(acc[u][8 * v + 2], acc[u][8 * v + 3]),
+                              pack_bf16(acc[u][8 * v + 4], acc[u][8 * v + 5]), pack_bf16(acc[u][8 * v + 6], acc[u][8 * v + 7]));
+      }
+    }
+  }
+  if (A.out_lse && tid / n_rows == 0) A.out_lse[orow] = lsum > 0.f ? (mmax * c + log2f(lsum)) * 0.6931471805599453f : -INFINITY;
+}
+
+template <int D>
+__device__ __forceinline__ void merge_pieces(const TcParams &P, const Item &I, int np, int row_begin, int n_rows, int tid) {
+  if (np <= 2) merge_pieces_n<D, 2>(P, I, np, row_begin, n_rows, tid);
+  else if (np <= 4) merge_pieces_n<D, 4>(P, I, np, row_begin, n_rows, tid);
+  else merge_pieces_n<D, 8>(P, I, np, row_begin, n_rows, tid);
 }
 
 // Persistent kernel: CTA c works through items c, c + gridDim.x, ... of the (longest request first) item
@@ -186,12 +323,14 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
            *p_full = q_full + 4, *pv_done = q_full + 6, *sf_a = q_full + 8, *sf_b = q_full + 9;
   uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(q_full + 10);
   volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+  volatile int *merge_flag = reinterpret_cast<volatile int *>(tmem_slot + 2);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // this CTA's items: its slice of the host-built schedule, else items blockIdx.x, blockIdx.x + gridDim.x, ...
-  const int q_begin = P.use_sched ? (int)P.cta_first[blockIdx.x] : (int)blockIdx.x;
-  const int q_end = P.use_sched ? (int)P.cta_first[blockIdx.x + 1] : P.n_items;
-  const int q_step = P.use_sched ? 1 : (int)gridDim.x;
+  const int team = P.use_seg ? (int)blockIdx.x / P.seg_X : 0;  // (CTAs behind the last whole team have no work)
+  const int q_begin = P.use_seg ? (team < P.seg_teams ? (int)P.team_first[team] : 0) : (P.use_sched ? (int)P.cta_first[blockIdx.x] : (int)blockIdx.x);
+  const int q_end = P.use_seg ? (team < P.seg_teams ? (int)P.team_first[team + 1] : 0) : (P.use_sched ? (int)P.cta_first[blockIdx.x + 1] : P.n_items);
+  const int q_step = (P.use_seg || P.use_sched) ? 1 : (int)gridDim.x;
   // (a CTA of a cluster must not leave early: its peers meet it at the cluster barriers below)
   if (P.nsplit == 1 && A.status_word && (*reinterpret_cast<volatile int32_t *>(A.status_word) & (int32_t)DPARA_STATUS_TIMEOUT)) return;
 
@@ -226,8 +365,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
     int ld = 0, k = 0;  // running K/V load counter, processed-item counter
     bool ok = true;
     for (int qi = q_begin; qi < q_end && ok; qi += q_step) {
-      const int id = P.use_sched ? (int)P.sched[qi] : qi;
-      const Item I = decode_item(P, id);
+      const Item I = fetch_item(P, qi);
       if (I.n_iter == 0) continue;
       // the Q buffer is free once the previous item's last QK has completed
       ok = __all_sync(0xffffffffu, mbar_wait(q_empty, (k & 1) ^ 1u, abort_flag));
@@ -342,8 +480,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
         mma_commit(kv_empty + vslot);
       };
       for (int qi = q_begin; qi < q_end && ok; qi += q_step) {
-      const int id = P.use_sched ? (int)P.sched[qi] : qi;
-        const Item I = decode_item(P, id);
+      const Item I = fetch_item(P, qi);
         if (I.n_iter == 0) continue;
         const int n_iter = I.n_iter;
         int kslot = 0, vslot = 0;
@@ -395,33 +532,24 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
     uint32_t ph_pv = 0;  // pv_done[t] completes once per (item, iteration); every phase is waited for exactly once, in order
     bool ok = true;
     for (int qi = q_begin; qi < q_end && ok; qi += q_step) {
-      const int id = P.use_sched ? (int)P.sched[qi] : qi;
-      const Item I = decode_item(P, id);
-      const int ji = I.ji0 + t * I.ji_t + (r >> I.hs);
-      const bool valid = (t < I.ntq) && (ji < P.n_rows);
-      const int h = I.g * A.G + I.h0 + (r & ((1 << I.hs) - 1));
-      const size_t orow = ((size_t)I.n * A.q_req_rows + A.lo * A.Bq + ji) * A.Hq + h;
-      // split-KV: this CTA's partial rows go to an L2-resident scratch slot and are merged after a cluster barrier
-      const size_t pslot = ((size_t)I.slot * 2 + t) * 128 + r;
-      if (I.n_iter == 0 || t >= I.ntq) {
-        // nothing visible to this work item, or no second tile in the last pair
-        if (P.nsplit > 1) {
-          __stcg(P.part_ml + pslot, make_float2(-INFINITY, 0.f));
-        } else if (valid) {
-          for (int d = 0; d < D; ++d) {
-            if (A.out_f32) static_cast<float *>(A.out)[orow * D + d] = 0.f;
-            else static_cast<uint16_t *>(A.out)[orow * D + d] = 0;
-          }
-          if (A.out_lse) A.out_lse[orow] = -INFINITY;
-        }
-        continue;
+      // ---- what the iteration loop needs, in as few registers as possible (the score row takes 128 of them); the item
+      // is decoded again after the loop for the output addresses
+      int n_iter, n_ctx_it, ragged_nv, jrel, na_row;
+      bool two_tiles, skip;
+      {
+        const Item I = fetch_item(P, qi);
+        skip = I.n_iter == 0 || t >= I.ntq;  // nothing visible to this work item, or no second tile in the last pair
+        n_iter = skip ? 0 : I.n_iter;
+        n_ctx_it = I.n_ctx_it;
+        two_tiles = I.ntq == 2;
+        ragged_nv = (I.t1 == I.nctx) ? (I.L & 127) : 0;  // valid keys of a part-filled last context tile (0: it is full or not ours)
+        // a mask-slot row: its boundary, counted from the first one whose block sits in the tail tiles, and its anchor
+        // prefix; a spine row (an anchor as a query): no own block (-1), and anchors 0 .. itself
+        const int ji = I.ji0 + t * I.ji_t + (r >> I.hs);
+        const bool is_spine = ji >= P.n_ji;
+        jrel = is_spine ? -1 : A.lo + ji / A.Bq - I.jb0;
+        na_row = is_spine ? ji - P.n_ji + 1 : max(0, min(A.lo + ji / A.Bq + A.pb, A.S));
       }
-      const int n_iter = I.n_iter;
-      // a mask-slot row: its boundary, counted from the first one whose block sits in the tail tiles, and its anchor
-      // prefix; a spine row (an anchor as a query): no own block (-1), and anchors 0 .. itself
-      const bool is_spine = ji >= P.n_ji;
-      const int jrel = is_spine ? -1 : A.lo + ji / A.Bq - I.jb0;
-      const int na_row = is_spine ? ji - P.n_ji + 1 : max(0, min(A.lo + ji / A.Bq + A.pb, A.S));
       float m_used = -INFINITY, l = 0.f;
 
       for (int it = 0; it < n_iter; ++it) {
@@ -429,8 +557,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
         // (worked out before the score row occupies the registers)
         // The visible keys of the tile as a 128-bit mask (four words), so that masking a score is one bit test.
         uint32_t vis[4] = {0u, 0u, 0u, 0u};
-        if (it >= I.n_ctx_it) {
-          const int tk = it - I.n_ctx_it;
+        if (it >= n_ctx_it) {
+          const int tk = it - n_ctx_it;
           const int kt = (!P.has_blk || jrel < 0) ? -1 : (jrel < P.cap0 ? 0 : 1 + (jrel - P.cap0) / P.cap);
           const int boff = jrel < P.cap0 ? P.S8 + jrel * A.Bq : ((jrel - P.cap0) % P.cap) * A.Bq;
           const int na_t = tk == 0 ? na_row : 0;
@@ -448,16 +576,16 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
         // the scores are in registers: hand the S buffer to the next QK product
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive((t == 0 && I.ntq == 2) ? sf_b : sf_a);  // next user: tile 1 of this iteration, else tile 0
+        if (lane == 0) mbar_arrive((t == 0 && two_tiles) ? sf_b : sf_a);  // next user: tile 1 of this iteration, else tile 0
         bool pv_waited = (it == 0);  // PV(t, it-1) must be complete before O_t is rescaled or P_t overwritten
         float s[128];
 #pragma unroll
         for (int kx = 0; kx < 128; ++kx) s[kx] = __uint_as_float(su[kx]);
-        if (it >= I.n_ctx_it) {
+        if (it >= n_ctx_it) {
 #pragma unroll
           for (int kx = 0; kx < 128; ++kx) s[kx] = ((vis[kx >> 5] >> (kx & 31)) & 1u) ? s[kx] : -INFINITY;
-        } else if (it == I.n_ctx_it - 1 && I.t1 == I.nctx && (I.L & 127)) {
-          const int nv = I.L & 127;
+        } else if (it == n_ctx_it - 1 && ragged_nv) {
+          const int nv = ragged_nv;
 #pragma unroll
           for (int kx = 0; kx < 128; ++kx) s[kx] = kx < nv ? s[kx] : -INFINITY;
         }
@@ -525,11 +653,30 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
         if (lane == 0) mbar_arrive(p_full + t);
       }
 
-      // ---- epilogue of this item (the MMA issuer cannot touch O_t again before this tile's next p_full arrive)
-      if (ok) {
-        ok = __all_sync(0xffffffffu, mbar_wait(pv_done + t, ph_pv, abort_flag, 9));
-        ph_pv ^= 1u;
+      // ---- output of this item (the MMA issuer cannot touch O_t again before this tile's next p_full arrive)
+      if (!ok) break;
+      const Item I = fetch_item(P, qi);
+      const int ji = I.ji0 + t * I.ji_t + (r >> I.hs);
+      const bool valid = (t < I.ntq) && (ji < P.n_rows);
+      const int h = I.g * A.G + I.h0 + (r & ((1 << I.hs) - 1));
+      const size_t orow = ((size_t)I.n * A.q_req_rows + A.lo * A.Bq + ji) * A.Hq + h;
+      // split-KV: this CTA's partial rows go to an L2-resident scratch slot and are merged later
+      const size_t pslot = ((size_t)I.slot * 2 + t) * 128 + r;
+      const bool partial = I.npieces > 1;  // one KV piece of several: unnormalised rows to scratch
+      if (skip) {
+        if (partial) {
+          __stcg(P.part_ml + pslot, make_float2(-INFINITY, 0.f));
+        } else if (valid) {
+          for (int d = 0; d < D; ++d) {
+            if (A.out_f32) static_cast<float *>(A.out)[orow * D + d] = 0.f;
+            else static_cast<uint16_t *>(A.out)[orow * D + d] = 0;
+          }
+          if (A.out_lse) A.out_lse[orow] = -INFINITY;
+        }
+        continue;
       }
+      ok = __all_sync(0xffffffffu, mbar_wait(pv_done + t, ph_pv, abort_flag, 9));
+      ph_pv ^= 1u;
       if (!ok) break;
       tc_fence_after();
       const float inv = l > 0.f ? 1.0f / l : 0.f;
@@ -543,7 +690,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
         uint32_t o[32];
         tmem_ld32(lane_addr + Cfg::kColO + t * 128 + cc * 32, o);
         tmem_wait_ld();
-        if (P.nsplit > 1) {
+        if (partial) {
           float4 *dst = reinterpret_cast<float4 *>(P.part_o) + (((size_t)I.slot * 2 + t) * (D / 4) + cc * 8) * 128 + r;
 #pragma unroll
           for (int v = 0; v < 8; ++v)
@@ -558,7 +705,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
                                    __uint_as_float(o[4 * v + 2]) * inv, __uint_as_float(o[4 * v + 3]) * inv);
           }
         }
-        if (P.nsplit == 1 && !A.out_f32) {
+        if (!partial && !A.out_f32) {
           // bf16 output: the thread's 32 columns are four 16-byte pieces of its row.  Written as they are, one store
           // instruction of a warp touches 32 rows (32 partial sectors).  The four lanes of a quad swap pieces (a 4 x 4
           // transpose by two butterfly steps) so that store v of a quad is 64 contiguous bytes of row 4q + v.
@@ -577,7 +724,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
         }
       }
       tc_fence_before();  // the O_t reads above are ordered before this warp's next p_full arrive
-      if (P.nsplit > 1) {
+      if (partial) {
         __stcg(P.part_ml + pslot, make_float2(m_used, l));
       } else if (valid && A.out_lse) {
         A.out_lse[orow] = l > 0.f ? (m_used * c + log2f(l)) * 0.6931471805599453f : -INFINITY;
@@ -598,74 +745,34 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
       const Item I = decode_item(P, blockIdx.x);
       const uint32_t rank = cluster_ctarank();
       const int rows_per = 256 / P.nsplit;
-      const float c = P.c_log2;
-      const size_t slot0 = (size_t)(I.slot - I.split);  // scratch slot of split 0 of this item
-      // unit of work: 16 output elements of one row; a warp's lanes take consecutive rows (contiguous loads);
-      // the loads of four splits are issued before their first use
-      constexpr int kParts = D / 16;
-      for (int u = threadIdx.x; u < rows_per * kParts; u += 256) {
-        const int R = (int)rank * rows_per + u % rows_per, part = u / rows_per;
-        const int t = R >> 7, r = R & 127;
-        const int ji = I.ji0 + t * I.ji_t + (r >> I.hs);
-        if (t >= I.ntq || ji >= P.n_rows) continue;
-        const int h = I.g * A.G + I.h0 + (r & ((1 << I.hs) - 1));
-        const size_t orow = ((size_t)I.n * A.q_req_rows + A.lo * A.Bq + ji) * A.Hq + h;
-        float2 ml[8];
-#pragma unroll
-        for (int sp = 0; sp < 8; ++sp)
-          ml[sp] = sp < P.nsplit ? __ldcg(P.part_ml + ((slot0 + sp) * 2 + t) * 128 + r) : make_float2(-INFINITY, 0.f);
-        float acc[16], lsum = 0.f;
-#pragma unroll
-        for (int e = 0; e < 16; ++e) acc[e] = 0.f;
-        float mmax = -INFINITY;
-        bool have_max = false;
-#pragma unroll
-        for (int sp0 = 0; sp0 < 8; sp0 += 4) {
-          if (sp0 >= P.nsplit) break;
-          float4 x[4][4];
-#pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            if (sp0 + q < P.nsplit) {
-              const float4 *src = reinterpret_cast<const float4 *>(P.part_o) + (((slot0 + sp0 + q) * 2 + t) * (D / 4) + part * 4) * 128 + r;
-#pragma unroll
-              for (int v = 0; v < 4; ++v) x[q][v] = __ldcg(src + v * 128);
-            }
-          }
-          if (!have_max) {
-#pragma unroll
-            for (int sp = 0; sp < 8; ++sp) if (ml[sp].y > 0.f) mmax = fmaxf(mmax, ml[sp].x);
-            have_max = true;
-          }
-#pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            // a peer without visible keys wrote no rows (its slot may hold anything): weight 0 skips it
-            const float wgt = (sp0 + q < P.nsplit && ml[sp0 + q].y > 0.f) ? ex2((ml[sp0 + q].x - mmax) * c) : 0.f;
-            lsum = fmaf(wgt, ml[sp0 + q].y, lsum);
-            if (wgt > 0.f) {
-#pragma unroll
-              for (int v = 0; v < 4; ++v) {
-                acc[4 * v] = fmaf(wgt, x[q][v].x, acc[4 * v]);
-                acc[4 * v + 1] = fmaf(wgt, x[q][v].y, acc[4 * v + 1]);
-                acc[4 * v + 2] = fmaf(wgt, x[q][v].z, acc[4 * v + 2]);
-                acc[4 * v + 3] = fmaf(wgt, x[q][v].w, acc[4 * v + 3]);
-              }
-            }
-          }
-        }
-        const float inv = lsum > 0.f ? 1.0f / lsum : 0.f;
-        if (A.out_f32) {
-          float4 *dst = reinterpret_cast<float4 *>(static_cast<float *>(A.out) + orow * D + part * 16);
-#pragma unroll
-          for (int v = 0; v < 4; ++v) dst[v] = make_float4(acc[4 * v] * inv, acc[4 * v + 1] * inv, acc[4 * v + 2] * inv, acc[4 * v + 3] * inv);
-        } else {
-          uint4 *dst = reinterpret_cast<uint4 *>(static_cast<uint16_t *>(A.out) + orow * D + part * 16);
-#pragma unroll
-          for (int v = 0; v < 2; ++v)
-            dst[v] = make_uint4(pack_bf16(acc[8 * v] * inv, acc[8 * v + 1] * inv), pack_bf16(acc[8 * v + 2] * inv, acc[8 * v + 3] * inv),
-                                pack_bf16(acc[8 * v + 4] * inv, acc[8 * v + 5] * inv), pack_bf16(acc[8 * v + 6] * inv, acc[8 * v + 7] * inv));
-        }
-        if (A.out_lse && part == 0) A.out_lse[orow] = lsum > 0.f ? (mmax * c + log2f(lsum)) * 0.6931471805599453f : -INFINITY;
+      merge_pieces<D>(P, I, P.nsplit, (int)rank * rows_per, rows_per, threadIdx.x);
+    }
+  }
+
+  // ------------------------------------------------------------------ cut schedule: tickets and merges
+  if (P.use_seg && q_end > q_begin) {
+    // The pieces written early in the kernel have long left L2 (the K/V stream passed through it since): ask for every
+    // cut item's scratch rows now, so that a merge finds them in L2 instead of paying an HBM round trip per dependent load.
+    for (int qi = q_begin; qi < q_end; ++qi) {
+      const Item I = fetch_item(P, qi);
+      if (I.npieces <= 1) continue;
+      const char *base = reinterpret_cast<const char *>(P.part_o) + (size_t)I.slot0 * 2 * 128 * D * 4;
+      const int lines = I.npieces * 2 * 128 * D * 4 / 128;
+      for (int k = threadIdx.x; k < lines; k += kThreads) prefetch_l2(base + (size_t)k * 128);
+      if (threadIdx.x < I.npieces * 2 * 8) prefetch_l2(reinterpret_cast<const char *>(P.part_ml + (size_t)I.slot0 * 2 * 128) + threadIdx.x * 128);
+    }
+    __threadfence();
+    __syncthreads();  // every partial row of this CTA is written
+    for (int qi = q_begin; qi < q_end; ++qi) {
+      const Item I = fetch_item(P, qi);
+      if (I.npieces <= 1) continue;
+      if (threadIdx.x == 0) *merge_flag = !*abort_flag && atomicAdd(P.seg_count + I.item, 1u) == (unsigned)I.npieces - 1u;
+      __syncthreads();
+      if (*merge_flag && warp < 8) {
+        __threadfence();
+        merge_pieces<D>(P, I, I.npieces, 0, 256, threadIdx.x);
       }
+      __syncthreads();
     }
   }
 
@@ -728,6 +835,10 @@ TcPlan plan_attention_tc(const dpara_shape *s, const int64_t *host_off, const in
   p.items = items;
   p.workspace_bytes = nsplit > 1 ? (size_t)items * nsplit * 256 * ((size_t)s->head_dim + 2) * 4 : 0;
   p.workspace_max_bytes = items < 96 ? (size_t)items * 8 * 256 * ((size_t)s->head_dim + 2) * 4 : 0;
+  // the cut schedule (items >= 96): at most two pieces per team and member plus seven per group of a degenerate cut,
+  // bounded here by 2 * SMs piece slots; plus one ticket per item
+  if (items >= 96 && p.n_pairs <= 16)
+    p.workspace_max_bytes = (size_t)(2 * kNumSM) * 256 * ((size_t)s->head_dim + 2) * 4 + align_up((size_t)items * 4, 256);
   p.eligible = true;
   return p;
 }
@@ -753,7 +864,7 @@ static dpara_status launch_tc_d(const TcParams &P, const TcPlan &plan, cudaStrea
     cfg.attrs = attr;
     cfg.numAttrs = 1;
   } else {
-    cfg.gridDim = dim3(P.n_items < sms ? P.n_items : sms);  // persistent: at most one CTA per SM
+    cfg.gridDim = dim3(P.use_seg || P.n_items >= sms ? sms : P.n_items);  // persistent: at most one CTA per SM
   }
   if (cudaLaunchKernelEx(&cfg, attn_tc_kernel<D>, P) != cudaSuccess) {
     cudaGetLastError();
@@ -869,6 +980,86 @@ dpara_status launch_attention_tc(const AttnParams &A, const TcPlan &plan, const 
   if (plan.nsplit > 1) {
     P.part_o = static_cast<float *>(workspace);
     P.part_ml = reinterpret_cast<float2 *>(P.part_o + (size_t)plan.items * plan.nsplit * 256 * D);
+  }
+  const int X = plan.n_pairs, n_groups = A.b * A.Hkv, teams = X > 0 ? sms / X : 0;
+  // Used for few, long items (up to 2.5 per SM): with more, handing whole items to the least loaded CTA balances as well
+  // and averages out the pairs' different tail-tile counts, which a team pays in full (measured at 640 items of ~22 key
+  // tiles: 207 us against 255 us).
+  if (plan.nsplit == 1 && P.n_items >= 96 && 2 * P.n_items <= 5 * sms && X <= 16 && teams >= 2 && n_groups + teams <= kMaxSeg &&
+      sms <= kNumSM && workspace) {
+    // ---- cut schedule: the groups' key tiles laid end to end (each group counted with its tail tiles and a fixed
+    // cost of ~3 tiles), cut at the multiples of total / teams; a cut snaps to the nearest allowed place -- a group
+    // boundary, or inside a group at least kMinPiece context tiles from either end
+    const int kFixedTiles = 3, kMinPiece = 4;
+    int max_tail = 0;
+    for (int x = 0; x < X; ++x) max_tail = std::max(max_tail, (int)P.pair[x].n_tail);
+    std::vector<int> nctx(n_groups);
+    std::vector<long long> pre(n_groups + 1, 0);
+    int longest = 0;
+    for (int gr = 0; gr < n_groups; ++gr) {
+      const int z = gr / A.Hkv, n = P.use_order ? (int)P.req_order[z] : z;
+      nctx[gr] = (int)((len_of(n) + 127) >> 7);
+      pre[gr + 1] = pre[gr] + nctx[gr] + max_tail + kFixedTiles;
+      longest = std::max(longest, nctx[gr]);
+    }
+    if (longest >= 4 * kMinPiece && longest < 65536) {
+      struct Piece { int group, t0, t1, team; };
+      std::vector<Piece> pieces;
+      // cut k (k = 1 .. teams - 1) as a position (group, tile): tile 0 = the group's start
+      int cg = 0, ct = 0, team = 0, cuts_in_group = 0;  // current start position, team under construction
+      auto emit_until = [&](int g1, int t1) {             // pieces of `team` from (cg, ct) up to (g1, t1), t1 == 0: the group's start
+        while (cg < g1 || (cg == g1 && ct < t1)) {
+          const int end = cg < g1 ? nctx[cg] : t1;
+          if (end > ct || nctx[cg] == 0) pieces.push_back({cg, ct, end, team});
+          if (cg < g1) { ++cg; ct = 0; cuts_in_group = 0; } else { ct = t1; }
+        }
+      };
+      for (int k = 1; k < teams; ++k) {
+        const long long target = pre[n_groups] * k / teams;
+        int g = cg;
+        while (g < n_groups && pre[g + 1] <= target) ++g;
+        if (g >= n_groups) break;
+        const long long off = target - pre[g];           // units into group g
+        // candidates: the start of g, the start of g + 1, a place inside g
+        long long best = off;                            // distance to the start of g
+        int bg = g, bt = 0;
+        if (pre[g + 1] - target < best) { best = pre[g + 1] - target; bg = g + 1; bt = 0; }
+        if (nctx[g] >= 2 * kMinPiece && cuts_in_group + (g == cg ? 0 : -cuts_in_group) < 7) {
+          long long t = std::min<long long>(std::max<long long>(off, kMinPiece), nctx[g] - kMinPiece);
+          if (g == cg) t = std::max<long long>(t, (long long)ct + kMinPiece);
+          if (t <= nctx[g] - kMinPiece && std::llabs(t - off) + 1 < best) { best = std::llabs(t - off); bg = g; bt = (int)t; }
+        }
+        if (bg < cg || (bg == cg && bt <= ct)) continue;  // nothing between the previous cut and this one: the team stays empty
+        emit_until(bg, bt);
+        if (bt > 0) ++cuts_in_group;
+        ++team;
+      }
+      team = std::min(team, teams - 1);
+      emit_until(n_groups, 0);
+      if ((int)pieces.size() <= kMaxSeg) {
+        std::vector<int> np(n_groups, 0), slot0(n_groups, 0), seen(n_groups, 0);
+        for (const Piece &pc : pieces) ++np[pc.group];
+        int slots = 0;  // per team member
+        for (int gr = 0; gr < n_groups; ++gr) { slot0[gr] = slots; slots += np[gr] > 1 ? np[gr] : 0; }
+        const size_t part_bytes = (size_t)slots * X * 256 * ((size_t)D + 2) * 4;
+        if (slots < 65536 && part_bytes + align_up((size_t)P.n_items * 4, 256) <= plan.workspace_max_bytes) {
+          int q = 0, c = 0;
+          for (const Piece &pc : pieces) {
+            while (c <= pc.team) P.team_first[c++] = (uint16_t)q;
+            TcParams::Seg &e = P.seg[q++];
+            e.group = (uint16_t)pc.group; e.t0 = (uint16_t)pc.t0; e.t1 = (uint16_t)pc.t1; e.slot0 = (uint16_t)slot0[pc.group];
+            e.piece = (uint8_t)seen[pc.group]++; e.npieces = (uint8_t)np[pc.group];
+          }
+          while (c <= kNumSM) P.team_first[c++] = (uint16_t)q;
+          P.use_seg = 1; P.seg_X = X; P.seg_teams = teams;
+          P.use_sched = 0;
+          P.part_o = static_cast<float *>(workspace);
+          P.part_ml = reinterpret_cast<float2 *>(P.part_o + (size_t)slots * X * 256 * D);
+          P.seg_count = reinterpret_cast<unsigned int *>(static_cast<uint8_t *>(workspace) + align_up(part_bytes, 256));
+          if (cudaMemsetAsync(P.seg_count, 0, (size_t)P.n_items * 4, st) != cudaSuccess) return DPARA_ERR_CUDA;
+        }
+      }
+    }
   }
   return D == 128 ? launch_tc_d<128>(P, plan, st) : launch_tc_d<64>(P, plan, st);
 }

@@ -196,6 +196,14 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 
+// Asks for the 128-byte line at `p` in L2 (no register, no wait).
+__device__ __forceinline__ void prefetch_l2(const void *p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
+
+// Barrier `id` (1..15; 0 is __syncthreads) among `nthreads` threads of the CTA (a multiple of 32; whole warps).
+__device__ __forceinline__ void named_bar_sync(int id, int nthreads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+
 // ---------------------------------------------------------------------------------------------- thread-block clusters
 __device__ __forceinline__ uint32_t cluster_ctarank() {
   uint32_t r;

@@ -193,3 +193,42 @@ def test_spine_tokens_as_query_rows(shape):
                                            [int(x) for x in inp.ctx_offsets], dev_bf16(inp.k_spine), dev_bf16(inp.v_spine),
                                            dev_bf16(inp.k_blk), dev_bf16(inp.v_blk))
     assert np.all(np.abs(out16.float().cpu().numpy()[:, J * Bq:] - ref_spine) <= tol[:, J * Bq:])
+
+
+@pytest.mark.parametrize("shape,spine", [
+    (W.AttnShape((4000, 5100, 3000, 4500), 32, 8, 128, 16, 16), False),      # 128 items of 24..40 key tiles: cut into segments
+    (W.AttnShape((2100, 4500, 3300), 40, 8, 128, 16, 16), False),            # group size 5: 120 items, part of them with 3 tail tiles
+    (W.AttnShape((3000, 5000, 2048, 4100), 32, 8, 128, 16, 16), True),       # spine rows: 160 items, every fifth a one-tile item
+])
+def test_cut_item_schedule(shape, spine):
+    """Between ~100 and a few hundred long items the host cuts the items' key ranges into per-CTA segments; a cut item's
+    pieces are merged by the CTA that finishes last.  Checked on seeded rows against the oracle (outputs and LSE)."""
+    import paper_2609_27396_b200 as dp
+    from gpu_util import dev_bf16
+    inp = W.make_attn_inputs(shape, 55)
+    b, J, Bq, Hq, D, S = shape.batch, shape.n_boundaries, shape.block, shape.n_q_heads, shape.head_dim, shape.spine
+    rng = np.random.default_rng(9)
+    rows = [(int(rng.integers(b)), int(rng.integers(J)), int(rng.integers(Bq)), int(rng.integers(Hq))) for _ in range(600)]
+    # every request x KV head at both ends of the row range (first and last tile pair)
+    rows += [(n, jj, ii, g * (Hq // shape.n_kv_heads)) for n in range(b) for g in range(shape.n_kv_heads) for (jj, ii) in ((0, 0), (J - 1, Bq - 1))]
+    ref = OA.draft_rows(inp.q, inp.k_ctx, inp.v_ctx, inp.ctx_offsets, inp.k_spine, inp.v_spine, inp.k_blk, inp.v_blk, rows)
+    args = (dev_bf16(inp.k_ctx), dev_bf16(inp.v_ctx), [int(x) for x in inp.ctx_offsets], dev_bf16(inp.k_spine), dev_bf16(inp.v_spine),
+            dev_bf16(inp.k_blk), dev_bf16(inp.v_blk))
+    if spine:
+        q_spine = W.make_attn_inputs(W.AttnShape(shape.ctx_lens, Hq, shape.n_kv_heads, D, S, 1), 56).q.reshape(b, S, Hq, D)
+        q_rows = np.concatenate([inp.q.reshape(b, J * Bq, Hq, D), q_spine], axis=1)
+        out, lse, status = dp.draft_with_spine_queries(dev_bf16(q_rows), J, Bq, *args, out_dtype=torch.float32, want_lse=True)
+        o = out.cpu().numpy()
+        got = np.stack([o[n, j * Bq + i, h] for (n, j, i, h) in rows])
+        srows = [(int(rng.integers(b)), int(rng.integers(S)), int(rng.integers(Hq))) for _ in range(64)]
+        sref = OA.spine_rows(q_spine, inp.k_ctx, inp.v_ctx, inp.ctx_offsets, inp.k_spine, inp.v_spine)
+        assert max(float(np.abs(o[n, J * Bq + s_, h] - sref[n, s_, h]).max()) for (n, s_, h) in srows) <= TOL
+    else:
+        out, lse, status = dp.draft_all_boundaries(dev_bf16(inp.q), *args, out_dtype=torch.float32, want_lse=True)
+        o = out.cpu().numpy()
+        got = np.stack([o[n, j, i, h] for (n, j, i, h) in rows])
+    torch.cuda.synchronize()
+    assert np.abs(got.astype(np.float64) - ref).max() <= TOL
+    assert np.isfinite(o).all() and np.isfinite(lse.cpu().numpy()).all() and int(status.item()) == 0
+    out16 = (dp.draft_with_spine_queries(dev_bf16(q_rows), J, Bq, *args)[0] if spine else dp.draft_all_boundaries(dev_bf16(inp.q), *args)[0])
+    assert np.abs(out16.float().cpu().numpy() - o).max() <= 2.0 ** -8 * np.abs(o).max() + 1e-6      # the bf16 output is the rounded fp32 one
