@@ -275,8 +275,34 @@ def _layer_attention_only_us(self, k: int) -> float:
     return _median_us(lambda: plan(q=q, **self.kv, k_blk=kb, v_blk=vb, out=out), k, self.flush)
 
 
-def _layer_gemm_legs(self, peaks, k: int):
-    """Each projection of the block on its own (dpara_gemm_bf16 at the block's shapes)."""
+def _graph_us(fn, flush, k: int = 10) -> float:
+    """Device time of fn() per call: k x (L2 flush, fn) replayed from one CUDA graph, minus k x flush."""
+    import torch
+
+    def timed(body):
+        s = torch.cuda.Stream()
+        with torch.cuda.stream(s):
+            for _ in range(2):
+                body()
+            torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=s):
+                for _ in range(k):
+                    flush.zero_(); body()
+            ts = []
+            for _ in range(5):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(s); g.replay(); e1.record(s)
+                torch.cuda.synchronize()
+                ts.append(e0.elapsed_time(e1) * 1e3 / k)
+        return statistics.median(ts)
+    return timed(fn) - timed(lambda: None)
+
+
+def _layer_gemm_legs(self, peaks, k: int, only=None):
+    """Each projection of the block on its own (dpara_gemm_bf16 at the block's shapes, buffers allocated up front, calls
+    replayed from a CUDA graph so that no host time is in the figure)."""
+    import ctypes as C
     import torch
     import paper_2609_27396_b200 as dp
     a, l = self.attn, self.layer
@@ -284,12 +310,22 @@ def _layer_gemm_legs(self, peaks, k: int):
     qd, kd = a.n_q_heads * a.head_dim, a.n_kv_heads * a.head_dim
     g = torch.Generator(device="cuda").manual_seed(2)
     act = lambda K: torch.randn(M, K, device="cuda", generator=g).to(torch.bfloat16)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
     res = {}
     for name, w, K, N, epi in (("qkv", self.t["w_qkv"], l.hidden, qd + 2 * kd, 0), ("o", self.t["w_o"], qd, l.hidden, 1),
                                ("gate_up", self.t["w_gate_up"], l.hidden, l.intermediate, 2), ("down", self.t["w_down"], l.intermediate, l.hidden, 1)):
+        if only is not None and name != only:
+            continue
         x = act(K)
-        resid = torch.zeros(M, N, dtype=torch.float32, device="cuda") if epi == 1 else None
-        us = _median_us(lambda: dp.gemm_bf16(x, w, epilogue=epi, resid=resid), k, self.flush)
+        resid = torch.zeros(M, N, dtype=torch.bfloat16 if name == "o" else torch.float32, device="cuda") if epi == 1 else None
+        out = torch.empty(M, N, dtype=torch.float32 if epi == 1 else torch.bfloat16, device="cuda")
+        io = dp.GemmIO(x.data_ptr(), w.data_ptr(), M, N, K, epi, resid.data_ptr() if resid is not None else None,
+                       dp.BF16 if name == "o" else dp.F32, out.data_ptr(), None)
+
+        def call():
+            rc = dp.lib.dpara_gemm_bf16(C.byref(io), status.data_ptr(), torch.cuda.current_stream().cuda_stream)
+            assert rc == 0
+        us = _graph_us(call, self.flush, k)
         fl = 2.0 * M * K * N * (2 if epi == 2 else 1)
         res[name] = {"M": M, "N": N, "K": K, "us": us, "tflops": fl / (us * 1e-6) / 1e12, "frac_of_measured_burst": fl / (us * 1e-6) / 1e12 / peaks["bf16_tflops"]}
     return res
@@ -339,6 +375,33 @@ def backbone_leg(w5: W.Workload, peaks, k: int):
     fl = n_layers * (rows_fl + 2.0 * M * (l.hidden * (qd + 2 * kd) + qd * l.hidden + 3 * l.hidden * l.intermediate))
     return {"workload": f"{n_layers} blocks, spine tokens as query rows, {w5.name} shapes: M = {M} rows per block", "us": us, "us_per_block": us / n_layers,
             "flops": fl, "tflops": fl / (us * 1e-6) / 1e12, "tensor_frac_of_measured_burst": fl / (us * 1e-6) / 1e12 / peaks["bf16_tflops"]}
+
+
+def graph_timed_b1(r: "StepRunner", k: int = 20):
+    """The b = 1 step replayed from ONE CUDA graph (k x (L2 flush, attention, verify/select) minus k x flush): what the
+    device spends when the launches come from a captured graph, as the paper's single-GPU deployment does, instead of
+    from Python.  Both calls capture as they are (fixed addresses, no allocation)."""
+    import torch
+
+    def timed(fn):
+        s = torch.cuda.Stream()
+        with torch.cuda.stream(s):
+            torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=s):
+                for _ in range(k):
+                    r.flush.zero_(); fn()
+            ts = []
+            for _ in range(5):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(s); g.replay(); e1.record(s)
+                torch.cuda.synchronize()
+                ts.append(e0.elapsed_time(e1) * 1e3 / k)
+        return statistics.median(ts)
+    base = timed(lambda: None)
+    return {"graph_replay": {"step_us": timed(r.step) - base, "attention_us": timed(r.attention) - base,
+                             "verify_select_us": timed(r.verify) - base, "single_boundary_attention_us": timed(lambda: r.attention(r.plan1)) - base,
+                             "note": "k x (flush, calls) replayed from one CUDA graph, minus k x flush"}}
 
 
 def small_step_leg(index: int, k: int):
@@ -526,6 +589,53 @@ def oracle_threads() -> int:
     return len(os.sched_getaffinity(0))
 
 
+# ----------------------------------------------------------------------------- single targets for a profiler
+ONLY_TARGETS = {"attention_cfg2", "attention_cfg3", "attention_cfg5", "verify_cfg2", "verify_cfg3", "verify_cfg4", "layer_cfg5", "gemm_qkv", "gemm_o",
+                "gemm_gate_up", "gemm_down", "head", "cache_append", "backbone_cfg5"}
+
+
+def run_only(target: str, reps: int):
+    """Runs the kernels of one leg `reps` times on cuda:0 (inputs as in the timed legs) and returns."""
+    import torch
+    torch.cuda.set_device(0)
+    peaks = measured_peaks()
+    if target.startswith("attention_cfg") and target != "attention_cfg5":
+        w = W.workload(int(target[-1]))
+        r = StepRunner(w, w.seed)
+        fn = r.attention
+    elif target.startswith("verify_cfg") and target != "verify_cfg4":
+        w = W.workload(int(target[-1]))
+        r = StepRunner(w, w.seed)
+        fn = r.verify
+    elif target == "verify_cfg4":
+        sampling_select_leg(peaks, reps)
+        return
+    elif target in ("attention_cfg5", "layer_cfg5") or target.startswith("gemm_"):
+        w5 = W.workload(5)
+        r = LayerRunner(w5, w5.seed)
+        if target == "layer_cfg5":
+            fn = lambda: r.plan(**r.kv)
+        elif target == "attention_cfg5":
+            r.attention_only_us(reps)
+            return
+        else:
+            r.gemm_legs(peaks, 2, only=target[5:])
+            return
+    elif target == "head":
+        w = W.workload(3)
+        r = HeadRunner(w, w.seed)
+        fn = r.step
+    elif target == "cache_append":
+        cache_append_leg(W.workload(3), peaks, reps)
+        return
+    else:
+        backbone_leg(W.workload(5), peaks, reps)
+        return
+    for _ in range(reps):
+        fn()
+    torch.cuda.synchronize()
+
+
 # ----------------------------------------------------------------------------- main
 def main():
     ap = argparse.ArgumentParser()
@@ -537,7 +647,13 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-layer", action="store_true", help="skip the full-layer (cfg5) leg")
     ap.add_argument("--no-head", action="store_true", help="skip the LM head + autoregressive head loop (T_Head) leg")
+    ap.add_argument("--only", default=None, choices=sorted(ONLY_TARGETS), help="run ONE kernel family a few times and exit (no timing, "
+                    "no JSON line): the small command a profiler is pointed at")
+    ap.add_argument("--only-reps", type=int, default=3)
     args = ap.parse_args()
+    if args.only:
+        run_only(args.only, args.only_reps)
+        return
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "ours":
         # started without a launcher: become one -- N ranks of this script, one per GPU; rank 0 prints the line
         from paper_2609_27396_b200.dist_util import launch_ranks
@@ -654,6 +770,7 @@ def main():
                      "single_boundary_attention_us": statistics.median(p[1] for p in s2) * 1e3,
                      "all_over_single": a2 / (statistics.median(p[1] for p in s2) * 1e3), "allowance": w2.attn.n_boundaries,
                      "attention_gbs": attention_bytes(w2.attn) / (a2 * 1e-6) / 1e9, "attention_tflops": attention_flops(w2.attn) / (a2 * 1e-6) / 1e12}
+        out["b1"].update(graph_timed_b1(r2))
         del r2
         if not args.no_layer:
             w5 = W.workload(5)
