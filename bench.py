@@ -469,6 +469,109 @@ def cache_append_leg(wl: W.Workload, peaks, k: int, n_layers: int = 5):
             "frac_of_measured_hbm": by / (us * 1e-6) / 1e9 / peaks["hbm_gbs"]}
 
 
+def colocation_leg(peaks, n_layers: int = 2, standin_gb: float = 3.0):
+    """One round on ONE GPU the way the paper's single-GPU deployment runs it (Sec. 3.3: T_step ~ max(T_verify, T_precompute) +
+    T_Head; App. D, single-GPU paragraph: verification and backbone precomputation on two streams, everything captured in one CUDA
+    graph).  Stream A: a STAND-IN for the target's verification forward (there is no target model here): a chain of library matmuls
+    of the verified rows against `standin_gb` GB of bf16 weights, i.e. a weight-streaming load like a decoder forward.  Stream B: the
+    all-boundary backbone pass (dpara_draft_backbone, spine tokens as query rows, the paper's main draft length d = 7).  After the
+    join: verify/select, cache append, LM head + head loop.  Reported: each part alone, both together, and how much of the
+    precompute the overlap hides."""
+    import torch
+    import paper_2609_27396_b200 as dp
+    w3 = W.workload(3)
+    a = W.AttnShape(w3.attn.ctx_lens, 40, 8, 128, 8, 8)           # b = 16 ragged contexts, d = 7: 8 boundaries x 8 slots
+    hidden, inter, V = 5120, 17408, w3.verify.vocab
+    b, J, Bq, S = a.batch, a.n_boundaries, a.block, a.spine
+    R = J * Bq + S
+    g = torch.Generator(device="cuda").manual_seed(5)
+    mk = lambda sig, *sh: (torch.randn(*sh, device="cuda", generator=g) * sig).to(torch.bfloat16)
+    ones = lambda n: torch.ones(n, dtype=torch.bfloat16, device="cuda")
+    # caches with slack, one per layer
+    cap = [L + 4 * J for L in a.ctx_lens]
+    start = [0]
+    for c in cap:
+        start.append(start[-1] + c)
+    kc = [mk(1.0, start[-1], a.n_kv_heads, a.head_dim) for _ in range(n_layers)]
+    vc = [mk(1.0, start[-1], a.n_kv_heads, a.head_dim) for _ in range(n_layers)]
+    lens = torch.tensor(list(a.ctx_lens), dtype=torch.int64, device="cuda")
+    lens0 = lens.clone()
+    qd, kd = a.n_q_heads * a.head_dim, a.n_kv_heads * a.head_dim
+    x = mk(1.0, b, R, hidden)
+    y = torch.zeros(b, R, hidden, dtype=torch.float32, device="cuda")
+    y16 = torch.zeros(b, R, hidden, dtype=torch.bfloat16, device="cuda")
+    keep, layers = [], []
+    for _ in range(n_layers):
+        t = dict(w_qkv=mk(0.02, qd + 2 * kd, hidden), w_o=mk(0.02, hidden, qd), w_gate_up=mk(0.02, 2 * inter, hidden), w_down=mk(0.02, hidden, inter),
+                 rms1_w=ones(hidden), rms2_w=ones(hidden), qnorm_w=ones(a.head_dim), knorm_w=ones(a.head_dim))
+        keep.append(t)
+        layers.append(dp.make_layer_io(x=x, **t, y_f32=y, y_bf16=y16))
+    bplan = dp.BackbonePlan(ctx_offsets=start, n_boundaries=J, block=Bq, n_q_heads=a.n_q_heads, n_kv_heads=a.n_kv_heads, head_dim=a.head_dim,
+                            layers=layers, k_ctx=kc, v_ctx=vc, n_spine=S, ctx_lens=list(a.ctx_lens))
+    # verification side: stand-in forward, then the real select / append / head calls
+    n_mats = max(1, int(standin_gb * 1e9 / (8192 * 8192 * 2)))
+    wt = [mk(0.01, 8192, 8192) for _ in range(n_mats)]
+    xt = mk(1.0, b * J, 8192)
+    ver = W.make_verify_inputs(W.VerifyShape(b, J, V, Bq, hidden, "greedy", 0.75, 2.0), w3.seed, reps=np.zeros((1,), np.uint16))
+    target, tokens = torch.from_numpy(ver.target).cuda(), torch.from_numpy(ver.draft_tokens).cuda()
+    vplan = dp.VerifyPlan(batch=b, n_boundaries=J, vocab=V, block=Bq, hidden=hidden, mode=0, rep_req_rows=R)
+    cplan = dp.CachePlan(batch=b, n_rows=J, w_kv=[mk(0.02, 2 * kd, hidden) for _ in range(n_layers)], k_ctx=kc, v_ctx=vc,
+                         row_start=torch.tensor(start[:-1], dtype=torch.int64, device="cuda"), capacity=torch.tensor(cap, dtype=torch.int64, device="cuda"),
+                         ctx_len=lens, norm_w=[ones(hidden)] * n_layers, knorm_w=[ones(a.head_dim) for _ in range(n_layers)])
+    feats = mk(1.0, b, J, hidden)
+    hplan = dp.HeadPlan(b, Bq, hidden, V, 256)
+    w_lm, ar_w, ar_e = mk(0.02, V, hidden), mk(1.0, V, 256), mk(0.05, V, 256)
+
+    def standin():
+        h = xt
+        for wm in wt:
+            h = torch.mm(h, wm)
+        return h
+
+    def tail():
+        vplan(target=target, draft_tokens=tokens, reps=y16)
+        lens.copy_(lens0)
+        cplan.run(feats, vplan.accept_len)
+        hplan.run(vplan.selected, w_lm, ar_w, ar_e, vplan.bonus)
+
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device="cuda")
+    s_main, s_b = torch.cuda.Stream(), torch.cuda.Stream()
+
+    def graph_us(body, k=3):
+        with torch.cuda.stream(s_main):
+            body(); body()
+            torch.cuda.synchronize()
+            gr = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(gr, stream=s_main):
+                for _ in range(k):
+                    flush.zero_(); body()
+            ts = []
+            for _ in range(5):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(s_main); gr.replay(); e1.record(s_main)
+                torch.cuda.synchronize()
+                ts.append(e0.elapsed_time(e1) * 1e3 / k)
+        return statistics.median(ts)
+
+    def both():
+        s_b.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(s_b):
+            bplan()
+        standin()
+        torch.cuda.current_stream().wait_stream(s_b)
+
+    base = graph_us(lambda: None)
+    t_v, t_p, t_both = graph_us(standin) - base, graph_us(lambda: bplan()) - base, graph_us(both) - base
+    t_tail = graph_us(tail) - base
+    t_round = graph_us(lambda: (both(), tail())) - base
+    return {"workload": f"one round on one GPU: b={b} ragged contexts (sum {sum(a.ctx_lens)}), d=7 ({J} boundaries x {Bq} slots + {S} spine rows = {b * R} rows), "
+                        f"{n_layers} backbone blocks (hidden {hidden}, inter {inter}); verification = STAND-IN: {n_mats} library matmuls of {b * J} rows against {n_mats * 0.134:.1f} GB of bf16 weights",
+            "verify_standin_us": t_v, "precompute_us": t_p, "both_streams_us": t_both, "serial_us": t_v + t_p,
+            "precompute_hidden_frac": (t_v + t_p - t_both) / t_p if t_p > 0 else None,
+            "select_append_head_us": t_tail, "round_us": t_round, "round_serial_us": t_v + t_p + t_tail,
+            "note": "CUDA graph replay, L2 flushed before every round; T_step ~ max(T_verify, T_precompute) + T_Head of Sec. 3.3 is both_streams_us + select_append_head_us"}
+
+
 def parity_spot_check(run: "StepRunner", n_rows: int = 64):
     """max |delta| of the timed attention output against the oracle on a few seeded rows of the bench workload (the
     GPU tests check 4096 rows; this ties the timed configuration to the oracle inside the bench run itself)."""
@@ -590,7 +693,7 @@ def oracle_threads() -> int:
 
 
 # ----------------------------------------------------------------------------- single targets for a profiler
-ONLY_TARGETS = {"attention_cfg2", "attention_cfg3", "attention_cfg5", "verify_cfg2", "verify_cfg3", "verify_cfg4", "layer_cfg5", "gemm_qkv", "gemm_o",
+ONLY_TARGETS = {"colocation", "attention_cfg2", "attention_cfg3", "attention_cfg5", "verify_cfg2", "verify_cfg3", "verify_cfg4", "layer_cfg5", "gemm_qkv", "gemm_o",
                 "gemm_gate_up", "gemm_down", "head", "cache_append", "backbone_cfg5"}
 
 
@@ -627,6 +730,9 @@ def run_only(target: str, reps: int):
         fn = r.step
     elif target == "cache_append":
         cache_append_leg(W.workload(3), peaks, reps)
+        return
+    elif target == "colocation":
+        print(json.dumps(colocation_leg(peaks)))
         return
     else:
         backbone_leg(W.workload(5), peaks, reps)
@@ -811,6 +917,8 @@ def main():
         out["cfg4_sampling_select"] = sampling_select_leg(peaks, max(args.steps, 20))
         out["cache_append"] = cache_append_leg(wl, peaks, max(args.steps, 20))
         out["parity_spot_check"] = parity_spot_check(run)
+        if not args.no_layer and not args.no_head:
+            out["colocation"] = colocation_leg(peaks)
         if not args.no_cpu_baseline:
             t, est, desc = oracle_sample(wl, wl.seed, 0, wl.verify.batch, run.inp, run.ver)
             out["cpu_baseline"] = {"value": est * 1e6, "unit": "us", "cores": oracle_threads(), "kind": "oracle", "sample": desc,
