@@ -90,3 +90,59 @@ def test_draft_head_matches_composition_and_bf16_inputs_are_taken_exactly():
     # the generator's correction really matters: without it some token differs
     base_only = np.stack([np.argmax(wl @ h[n].T, axis=0) for n in range(3)])
     assert (base_only != got).any()
+
+
+# ----------------------------------------------------------------------------- sampling head loop (App. C setting: T = 1, top-p = 1)
+def test_sample_from_logits_closed_forms():
+    """Two tokens with logits (0, ln 3): probabilities 1/4 and 3/4 -- token 0 iff u < 1/4.  A one-hot row always gives its
+    token.  Adding a constant to every logit changes nothing.  NaN logits are never drawn."""
+    z = np.array([0.0, np.log(3.0)])
+    assert H.sample_from_logits(z, 0.0) == 0 and H.sample_from_logits(z, 0.2499) == 0
+    assert H.sample_from_logits(z, 0.25) == 1 and H.sample_from_logits(z, 0.999999) == 1
+    one_hot = np.array([-np.inf, -np.inf, 2.0, -np.inf])
+    assert all(H.sample_from_logits(one_hot, u) == 2 for u in (0.0, 0.5, 1 - 2.0 ** -24))
+    rng = np.random.default_rng(0)
+    z = rng.standard_normal(50)
+    for u in rng.random(20):
+        assert H.sample_from_logits(z, u) == H.sample_from_logits(z + 7.5, u)
+    z[3] = np.nan
+    assert all(H.sample_from_logits(z, u) != 3 for u in np.linspace(0, 0.9999, 200))
+    assert H.sample_from_logits(np.full(5, np.nan), 0.3) == 0
+    # monotone in u: the draw is the inverse of a non-decreasing function
+    draws = [H.sample_from_logits(z, u) for u in np.linspace(0, 0.9999, 300)]
+    assert draws == sorted(draws)
+
+
+def test_sampling_reproduces_softmax_chi_square():
+    """2e5 seeded uniforms m * 2^-24 over a 16-token vocabulary: the draws follow softmax(z) (15 dof, p > 0.001 <=> chi2 < 37.7)."""
+    rng = np.random.default_rng(4)
+    z = rng.standard_normal(16) * 1.5
+    p = np.exp(z - z.max()); p /= p.sum()
+    m = rng.integers(0, 1 << 24, size=200000)
+    c = np.cumsum(np.exp(z - z.max()))
+    toks = np.searchsorted(c, m * 2.0 ** -24 * c[-1], side="right")         # vectorised copy of the definition ...
+    assert all(H.sample_from_logits(z, mm * 2.0 ** -24) == t for mm, t in zip(m[:500], toks[:500]))   # ... checked against the function
+    counts = np.bincount(toks, minlength=16)
+    chi2 = float(((counts - p * len(m)) ** 2 / (p * len(m))).sum())
+    assert chi2 < 37.7, chi2
+
+
+def test_sampling_chain_feeds_the_previous_token():
+    """Same construction as the greedy chain: a +30 correction on (y + 1) mod V makes softmax a point mass, so the sampled
+    chain walks bonus + 1, bonus + 2, ... whatever the uniforms; with zero correction the draws depend on the uniforms only
+    and equal independent draws from the base rows."""
+    V, d = 9, 5
+    E = np.eye(V)
+    Wm = np.zeros((V, V))
+    for y in range(V):
+        Wm[(y + 1) % V][y] = 30.0
+    u = np.random.default_rng(1).random(d)
+    got = H.ar_head_sampling(np.zeros((d, V)), _bits(Wm), _bits(E), 6, u)
+    assert got.tolist() == [(6 + i + 1) % V for i in range(d)]
+    base = np.random.default_rng(2).standard_normal((d, V))
+    got = H.ar_head_sampling(base, _bits(np.zeros((V, V))), _bits(E), 3, u)
+    assert got.tolist() == [H.sample_from_logits(base[i], u[i]) for i in range(d)]
+    # a very peaked distribution: sampling equals greedy
+    sharp = base * 200.0
+    assert np.array_equal(H.ar_head_sampling(sharp, _bits(np.zeros((V, V))), _bits(E), 3, u),
+                          H.ar_head_greedy(sharp, _bits(np.zeros((V, V))), _bits(E), 3))
