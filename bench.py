@@ -606,14 +606,18 @@ class HeadRunner:
         self.plan = dp.HeadPlan(sh.batch, sh.block, sh.hidden, sh.vocab, sh.rank)
         self.flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device="cuda")
 
-    def step(self):
-        self.plan.run(*self.t, self.bonus)
+    def step(self, sampling: bool = False):
+        if sampling and not hasattr(self, "uniforms"):
+            g = self.torch.Generator(device="cuda").manual_seed(11)
+            sh = self.shape
+            self.uniforms = (self.torch.randint(0, 1 << 24, (sh.batch, sh.block), generator=g, device="cuda").float() * 2.0 ** -24)
+        self.plan.run(*self.t, self.bonus, uniforms=self.uniforms if sampling else None)
 
     def lm_head_only(self):
         sh = self.shape
         return self.dp.gemm_bf16(self.t[0].view(sh.batch * sh.block, sh.hidden), self.t[1], epilogue=3, status=self.plan.status)
 
-    def timed(self, k: int, lm_only: bool = False):
+    def timed(self, k: int, lm_only: bool = False, sampling: bool = False):
         torch = self.torch
         ev = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(k)]
         for s in range(k):
@@ -622,7 +626,7 @@ class HeadRunner:
             if lm_only:
                 self.lm_head_only()
             else:
-                self.step()
+                self.step(sampling)
             ev[s][1].record()
         torch.cuda.synchronize()
         return [e[0].elapsed_time(e[1]) for e in ev]
@@ -903,10 +907,14 @@ def main():
                 rh.step()
             th = statistics.median(rh.timed(max(5, min(args.steps, 10)))) * 1e3
             tl = statistics.median(rh.timed(max(5, min(args.steps, 10)), lm_only=True)) * 1e3
+            rh.step(sampling=True)
+            ts = statistics.median(rh.timed(max(5, min(args.steps, 10)), sampling=True)) * 1e3
             lmb, arb = head_bytes(rh.shape)
             sh = rh.shape
             out["head"] = {"workload": "T_Head at %s: b=%d, d=%d, hidden=%d, vocab=%d, head rank=%d (greedy)" % (wl.name, sh.batch, sh.block, sh.hidden, sh.vocab, sh.rank),
                            "head_us": th, "lm_head_us": tl, "ar_loop_us": th - tl, "ar_step_us": (th - tl) / sh.block,
+                           "sampling": {"head_us": ts, "ar_loop_us": ts - tl, "ar_step_us": (ts - tl) / sh.block,
+                                        "note": "y_i ~ softmax(z_i) from supplied uniforms (temperature 1): per step one GEMM that writes z_i and one inverse-CDF kernel"},
                            "lm_head": {"bound": "hbm", "achieved": lmb / (tl * 1e-6) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                                        "frac": lmb / (tl * 1e-6) / 1e9 / peaks["hbm_gbs"], "bytes": lmb,
                                        "tflops": 2.0 * sh.batch * sh.block * sh.hidden * sh.vocab / (tl * 1e-6) / 1e12},

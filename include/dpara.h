@@ -254,8 +254,11 @@ dpara_status dpara_verify_select_static(const dpara_verify_io *io, int32_t *stat
  * and picks the next token; Sec. 3.2 "Loss" gives the formula: the head has its own low-rank token embedding E and
  * a projection W of it to the vocabulary, and reads only the preceding token).  The base
  * logits l_i are the language-model head applied to the selected branch's final hidden states (App. D runs the
- * language-model head on shipped hidden states right before the head loop).  Greedy decoding (Table 1): y_i is the
- * lowest index holding the maximum of z_i; NaN ranks below every number.
+ * language-model head on shipped hidden states right before the head loop).  uniforms == NULL: greedy decoding (Table 1),
+ * y_i is the lowest index holding the maximum of z_i; NaN ranks below every number.  uniforms != NULL: sampling (App. C:
+ * temperature 1, top-p 1), y_i is drawn from softmax(z_i) by the inverse CDF in vocabulary order with the supplied
+ * uniform u = uniforms[n][i-1] = m * 2^-24: the lowest v with sum_{v' <= v} w_v' > u * sum w, w_v = exp(z_v - max z)
+ * (exponentials and sums in double precision; NaN logits weigh nothing).
  *   sel_reps     device [b][block][hidden] bf16: the selected branches (the `selected` output of dpara_verify_select)
  *   w_lm         device [vocab][hidden] bf16 (weights stored [out][in])
  *   ar_w, ar_e   device [vocab][rank] bf16: W (one row per vocabulary entry) and E (one row per token)
@@ -264,7 +267,9 @@ dpara_status dpara_verify_select_static(const dpara_verify_io *io, int32_t *stat
  *   next_tokens  device [b][block] int32 out: y_1 .. y_d
  * bf16 products with fp32 accumulation; z_i = (fp32 base logit) + (fp32 correction), compared in fp32.
  * Workspace: dpara_head_workspace_bytes(b, block, vocab) bytes of device memory, 16-byte aligned, owned by the
- * caller and private to the call while it runs (it holds the fp32 base logits [b * block][vocab]).
+ * caller and private to the call while it runs (it holds the fp32 base logits [b * block][vocab] and, for sampling, one
+ * step's logits z [b][vocab]).  The greedy loop is ONE persistent kernel; the sampling loop is two launches per step
+ * (the skinny product with the base logits added, then one CTA per request that draws the token).
  * All work is queued on `stream`; nothing is allocated.  Errors: INVALID_ARG (null or misaligned pointer,
  * non-positive size), UNSUPPORTED (b > 32, block > 64, rank not a multiple of 64 or > 256, hidden % 64 != 0,
  * vocab % 8 != 0), CUDA.  A device-side wait that runs out sets DPARA_STATUS_TIMEOUT in *status_word. */
@@ -276,6 +281,7 @@ typedef struct {
   const int32_t *bonus;
   int32_t *next_tokens;
   int32_t b, block, hidden, vocab, rank;
+  const float *uniforms;      /* device [b][block] fp32 or NULL (greedy) */
 } dpara_head_io;
 size_t dpara_head_workspace_bytes(int32_t b, int32_t block, int32_t vocab);
 dpara_status dpara_draft_head(const dpara_head_io *io, void *workspace, size_t workspace_bytes, int32_t *status_word, void *stream);

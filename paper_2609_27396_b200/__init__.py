@@ -322,7 +322,7 @@ def verify_select(target, draft_tokens, reps=None, *, mode: int = 0, draft_probs
 class HeadIO(C.Structure):
     _fields_ = [("sel_reps", C.c_void_p), ("w_lm", C.c_void_p), ("ar_w", C.c_void_p), ("ar_e", C.c_void_p),
                 ("bonus", C.c_void_p), ("next_tokens", C.c_void_p), ("b", C.c_int32), ("block", C.c_int32),
-                ("hidden", C.c_int32), ("vocab", C.c_int32), ("rank", C.c_int32)]
+                ("hidden", C.c_int32), ("vocab", C.c_int32), ("rank", C.c_int32), ("uniforms", C.c_void_p)]
 
 
 lib.dpara_head_workspace_bytes.restype = C.c_size_t
@@ -349,9 +349,10 @@ class HeadPlan:
         return self.workspace[: n * 4].view(torch.float32).view(self.block, self.b, self.vocab).permute(1, 0, 2).reshape(
             self.b * self.block, self.vocab)
 
-    def run(self, sel_reps, w_lm, ar_w, ar_e, bonus, stream=None):
+    def run(self, sel_reps, w_lm, ar_w, ar_e, bonus, uniforms=None, stream=None):
+        """uniforms [b][block] fp32 (each m * 2^-24): sample y_i from softmax(z_i); None: greedy."""
         io = HeadIO(_ptr(sel_reps), _ptr(w_lm), _ptr(ar_w), _ptr(ar_e), _ptr(bonus), _ptr(self.next_tokens),
-                    self.b, self.block, self.hidden, self.vocab, self.rank)
+                    self.b, self.block, self.hidden, self.vocab, self.rank, _ptr(uniforms))
         rc = lib.dpara_draft_head(C.byref(io), self.workspace.data_ptr(), self.workspace_bytes, self.status.data_ptr(),
                                   _stream_ptr(stream))
         if rc != OK:
@@ -359,12 +360,12 @@ class HeadPlan:
         return self.next_tokens
 
 
-def draft_head(sel_reps, w_lm, ar_w, ar_e, bonus, stream=None):
+def draft_head(sel_reps, w_lm, ar_w, ar_e, bonus, uniforms=None, stream=None):
     """dpara_draft_head: sel_reps [b][block][hidden], w_lm [vocab][hidden], ar_w / ar_e [vocab][rank] (bf16 CUDA
     tensors), bonus [b] int32.  Returns (next_tokens [b][block] int32, plan)."""
     b, block, hidden = sel_reps.shape
     plan = HeadPlan(b, block, hidden, w_lm.shape[0], ar_w.shape[1], sel_reps.device)
-    plan.run(sel_reps, w_lm, ar_w, ar_e, bonus, stream)
+    plan.run(sel_reps, w_lm, ar_w, ar_e, bonus, uniforms, stream)
     return plan.next_tokens, plan
 
 

@@ -162,5 +162,6 @@ extern "C" dpara_status dpara_draft_head(const dpara_head_io *io, void *workspac
   HeadArgs h;
   h.sel_reps = io->sel_reps; h.w_lm = io->w_lm; h.ar_w = io->ar_w; h.ar_e = io->ar_e; h.bonus = io->bonus;
   h.next_tokens = io->next_tokens; h.b = io->b; h.block = io->block; h.hidden = io->hidden; h.vocab = io->vocab; h.rank = io->rank;
+  h.uniforms = io->uniforms;
   return launch_head(h, workspace, status_word, static_cast<cudaStream_t>(stream));
 }

@@ -54,8 +54,15 @@ struct ArParams {
   unsigned int *barrier;      // zeroed before the launch
   int32_t *status;
   int b, block, vocab, rank, n_tiles, nb, stages;
+  float *z_out;               // sampling: [b][vocab] fp32, the logits z of step `step0`
+  int step0;                  // sampling: the one step this launch computes
 };
 
+// kSample = false: the whole greedy loop in one cooperative launch.  kSample = true: ONE step (P.step0) of the sampling
+// loop -- the same producer / MMA / epilogue pipeline, but the epilogue writes z = l + W E(y_prev) to P.z_out instead of
+// tracking maxima, the previous tokens come from P.next_tokens (written by the draw of the step before), and there is no
+// grid barrier (the draw is a launch of its own).
+template <bool kSample>
 __global__ void __launch_bounds__(kThreads, 1) ar_head_kernel(const __grid_constant__ ArParams P) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -88,6 +95,7 @@ __global__ void __launch_bounds__(kThreads, 1) ar_head_kernel(const __grid_const
   const uint32_t tmem = *tmem_slot;
   // this CTA's tiles: blockIdx.x, blockIdx.x + gridDim.x, ... (the same in every step)
   const int my_tiles = (P.n_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+  const int step_begin = kSample ? P.step0 : 0, step_end = kSample ? P.step0 + 1 : P.block;
 
   if (warp == kProducerWarp) {
     // ------------------------------------------------------------------ producer
@@ -96,7 +104,7 @@ __global__ void __launch_bounds__(kThreads, 1) ar_head_kernel(const __grid_const
       int stage = 0;
       uint32_t ph = 0;
       bool ok = true;
-      for (int step = 0; step < P.block && ok; ++step) {
+      for (int step = step_begin; step < step_end && ok; ++step) {
         for (int k = 0; k < my_tiles; ++k) {
           ok = mbar_wait(empty + stage, ph ^ 1u, abort_flag, 2);
           if (!ok) break;
@@ -117,8 +125,8 @@ __global__ void __launch_bounds__(kThreads, 1) ar_head_kernel(const __grid_const
       int stage = 0, kt = 0;
       uint32_t ph = 0;
       bool ok = true;
-      for (int step = 0; step < P.block && ok; ++step) {
-        ok = mbar_wait(e_ready, step & 1, abort_flag, 3);   // Ey of this step is in shared memory
+      for (int step = step_begin; step < step_end && ok; ++step) {
+        ok = mbar_wait(e_ready, (step - step_begin) & 1, abort_flag, 3);   // Ey of this step is in shared memory
         for (int k = 0; k < my_tiles && ok; ++k, ++kt) {
           const int buf = kt & 1;
           ok = mbar_wait(acc_empty + buf, ((kt >> 1) & 1) ^ 1u, abort_flag, 4) && mbar_wait(full + stage, ph, abort_flag, 5);
@@ -151,7 +159,7 @@ __global__ void __launch_bounds__(kThreads, 1) ar_head_kernel(const __grid_const
       ph_epi ^= 1u;
       return r;
     };
-    for (int step = 0; step < P.block && ok; ++step) {
+    for (int step = step_begin; step < step_end && ok; ++step) {
       // previous tokens: the bonus for the first step, else the winners of the previous step
       if (threadIdx.x < kMaxBatch) {
         int tok = 0;
@@ -162,6 +170,9 @@ __global__ void __launch_bounds__(kThreads, 1) ar_head_kernel(const __grid_const
               if (P.status) atomicOr(reinterpret_cast<unsigned int *>(P.status), DPARA_STATUS_BAD_TOKEN);
               tok = 0;
             }
+          } else if (kSample) {
+            tok = __ldcg(P.next_tokens + (size_t)threadIdx.x * P.block + (step - 1));
+            if (tok < 0 || tok >= P.vocab) tok = 0;
           } else {
             const unsigned long long w = __ldcg(P.best + ((size_t)(step - 1) * kMaxBatch + threadIdx.x) * kBestStride);
             tok = (int)(0xffffffffu - (uint32_t)(w & 0xffffffffull));
@@ -214,15 +225,19 @@ __global__ void __launch_bounds__(kThreads, 1) ar_head_kernel(const __grid_const
           const int n = 2 * j + nh;
           if (n < P.b) {
             const float z = __uint_as_float(nh ? acc[2 * j + 1] : acc[2 * j]) + sl[n * 128];
-            // larger, or the first number this thread sees (NaN never wins; -inf can, at the lowest index)
-            if (live && (z > bz[j] || (bv[j] < 0 && z == z))) { bz[j] = z; bv[j] = v; }
+            if (kSample) {
+              if (live) P.z_out[(size_t)n * P.vocab + v] = z;       // a warp writes 32 consecutive entries of one row
+            } else if (live && (z > bz[j] || (bv[j] < 0 && z == z))) {
+              // larger, or the first number this thread sees (NaN never wins; -inf can, at the lowest index)
+              bz[j] = z; bv[j] = v;
+            }
           }
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(empty + stage);
         if (++stage == P.stages) { stage = 0; ph_full ^= 1u; }
       }
-      if (!ok) break;
+      if (!ok || kSample) break;
       // step maximum: warp reduction, CTA reduction through shared memory, then ONE atomic per request and CTA,
       // each request on its own 128-byte line (atomics on one line are serialised by a single L2 unit)
 #pragma unroll
@@ -262,7 +277,7 @@ __global__ void __launch_bounds__(kThreads, 1) ar_head_kernel(const __grid_const
       ok = epi_sync() && !*abort_flag;
     }
     // the last step's winners
-    if (ok && blockIdx.x == 0 && (int)threadIdx.x < P.b) {
+    if (!kSample && ok && blockIdx.x == 0 && (int)threadIdx.x < P.b) {
       const unsigned long long w = __ldcg(P.best + ((size_t)(P.block - 1) * kMaxBatch + threadIdx.x) * kBestStride);
       P.next_tokens[(size_t)threadIdx.x * P.block + (P.block - 1)] = w == 0ull ? 0 : (int)(0xffffffffu - (uint32_t)(w & 0xffffffffull));
     }
@@ -281,10 +296,194 @@ __global__ void __launch_bounds__(kThreads, 1) ar_head_kernel(const __grid_const
   if (warp == kMmaWarp) tmem_dealloc(tmem, 64);
 }
 
+// ------------------------------------------------------------------------------------------------ sampling head loop
+// y_i ~ softmax(z_i) with a supplied uniform (App. C: temperature 1, top-p 1).  Two launches per step: the head kernel
+// above in its one-step form writes z = l_i + W E(y_{i-1}) (fp32, [b][vocab]), then the draw, spread over
+// (vocabulary chunk, request) CTAs: each CTA leaves its chunk's maximum m_c and weight sum s_c = sum exp(z - m_c) and
+// takes a ticket; the CTA that takes a request's last ticket (no CTA ever waits) rescales the chunk sums to the row
+// maximum, finds the chunk the threshold u * total falls into, rescans that one chunk in vocabulary order for the
+// crossing element, writes the token and puts the ticket back to zero.
+// Exponentials are fp32 (relative error ~1e-7, far below the fp32 logits' own), every sum is fp64.
+namespace {
+constexpr int kPickThreads = 256;
+constexpr int kPickMaxChunks = 256;          // one chunk per thread in the finishing CTA
+
+struct PickPart { float m; float pad; double s; };
+
+__host__ __device__ inline int pick_chunk_elems(int vocab) {
+  int chunk = 2048;
+  while ((vocab + chunk - 1) / chunk > kPickMaxChunks) chunk *= 2;
+  return chunk;
+}
+
+__device__ __forceinline__ double warp_sum(double x) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+  return x;
+}
+
+// inclusive block scan of one double per thread (kPickThreads threads); returns the inclusive value, total in *total
+__device__ __forceinline__ double block_scan(double x, double *s_warp, double *total) {
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  double inc = x;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const double t = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += t;
+  }
+  __syncthreads();                       // s_warp free again
+  if (lane == 31) s_warp[w] = inc;
+  __syncthreads();
+  double before = 0.0, tot = 0.0;
+#pragma unroll
+  for (int k = 0; k < kPickThreads / 32; ++k) { if (k < w) before += s_warp[k]; tot += s_warp[k]; }
+  *total = tot;
+  return before + inc;
+}
+
+__global__ void __launch_bounds__(kPickThreads) head_sample_kernel(const float *__restrict__ z, const float *__restrict__ uniforms,
+                                                                   int32_t *__restrict__ next_tokens, PickPart *__restrict__ part,
+                                                                   unsigned int *__restrict__ tick, int vocab, int block,
+                                                                   int step, int chunk) {
+  const int n = blockIdx.y, c = blockIdx.x, n_chunks = gridDim.x, tid = threadIdx.x;
+  const float *row = z + (size_t)n * vocab;
+  __shared__ float s_max[kPickThreads / 32];
+  __shared__ double s_warp[kPickThreads / 32];
+  __shared__ int s_flag;
+  __shared__ int s_tok;
+  __shared__ double s_base;
+
+  // ---- phase 1: this chunk's maximum and weight sum (vocab % 8 == 0 and chunk % 1024 == 0: float4 loads never straddle)
+  const int c0 = c * chunk, c1 = min(vocab, c0 + chunk);
+  float mx = -INFINITY;
+  for (int v = c0 + tid * 4; v < c1; v += kPickThreads * 4) {
+    const float4 x = __ldcg(reinterpret_cast<const float4 *>(row + v));
+    mx = fmaxf(mx, fmaxf(fmaxf(x.x, x.y), fmaxf(x.z, x.w)));          // fmaxf drops NaN operands
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+  if ((tid & 31) == 0) s_max[tid >> 5] = mx;
+  __syncthreads();
+  mx = s_max[0];
+#pragma unroll
+  for (int w = 1; w < kPickThreads / 32; ++w) mx = fmaxf(mx, s_max[w]);
+  double loc = 0.0;
+  if (mx > -INFINITY && mx < INFINITY) {
+    for (int v = c0 + tid * 4; v < c1; v += kPickThreads * 4) {
+      const float4 x = __ldcg(reinterpret_cast<const float4 *>(row + v));
+      if (x.x == x.x) loc += (double)expf(x.x - mx);
+      if (x.y == x.y) loc += (double)expf(x.y - mx);
+      if (x.z == x.z) loc += (double)expf(x.z - mx);
+      if (x.w == x.w) loc += (double)expf(x.w - mx);
+    }
+  }
+  loc = warp_sum(loc);
+  if ((tid & 31) == 0) s_warp[tid >> 5] = loc;
+  __syncthreads();
+  if (tid == 0) {
+    double s = 0.0;
+    for (int w = 0; w < kPickThreads / 32; ++w) s += s_warp[w];
+    PickPart pp; pp.m = mx; pp.pad = 0.f; pp.s = s;
+    part[(size_t)n * kPickMaxChunks + c] = pp;
+    __threadfence();
+    s_flag = atomicAdd(tick + n, 1u) == (unsigned)(n_chunks - 1);
+  }
+  __syncthreads();
+  if (!s_flag) return;
+  __threadfence();
+
+  // ---- phase 2 (the CTA that took the request's last ticket): thread t holds chunk t
+  float m_c = -INFINITY;
+  double s_c = 0.0;
+  if (tid < n_chunks) {
+    const uint4 raw = __ldcg(reinterpret_cast<const uint4 *>(part + (size_t)n * kPickMaxChunks + tid));
+    m_c = __uint_as_float(raw.x);
+    s_c = __hiloint2double((int)raw.w, (int)raw.z);
+  }
+  float M = m_c;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+  __syncthreads();
+  if ((tid & 31) == 0) s_max[tid >> 5] = M;
+  if (tid == 0) { s_tok = -1; s_flag = -1; }
+  __syncthreads();
+  M = s_max[0];
+#pragma unroll
+  for (int w = 1; w < kPickThreads / 32; ++w) M = fmaxf(M, s_max[w]);
+  int tok = 0;
+  if (M > -INFINITY && M < INFINITY) {
+    const double scale = (m_c > -INFINITY) ? exp((double)m_c - (double)M) : 0.0;
+    const double S = s_c * scale;
+    double total;
+    const double inc = block_scan(S, s_warp, &total);
+    const double T = (double)uniforms[(size_t)n * block + step] * total;
+    // the chunk the threshold falls into; when rounding puts the threshold at or past the total, the last chunk with weight
+    if (S > 0.0 && inc - S <= T && T < inc) { s_flag = tid; s_base = inc - S; }
+    __syncthreads();
+    if (s_flag < 0) {
+      if (S > 0.0) atomicMax(&s_flag, tid);
+      __syncthreads();
+      if (tid == s_flag) s_base = inc - S;
+      __syncthreads();
+    }
+    const int cs = s_flag;                               // >= 0: total > 0 because the row maximum is finite
+    __syncthreads();
+    if (tid == cs) { s_max[0] = m_c; s_warp[0] = scale; }
+    __syncthreads();
+    const float mcs = s_max[0];
+    const double scs = s_warp[0];
+    double running = s_base;
+    const int r0 = cs * chunk, r1 = min(vocab, r0 + chunk);
+    int last_w = -1;                                     // the last element with weight seen by this thread
+    for (int v0 = r0; v0 < r1; v0 += kPickThreads * 4) {
+      const int v = v0 + tid * 4;
+      double w[4] = {0.0, 0.0, 0.0, 0.0};
+      if (v < r1) {
+        const float4 x = __ldcg(reinterpret_cast<const float4 *>(row + v));
+        if (x.x == x.x) w[0] = (double)expf(x.x - mcs) * scs;
+        if (x.y == x.y) w[1] = (double)expf(x.y - mcs) * scs;
+        if (x.z == x.z) w[2] = (double)expf(x.z - mcs) * scs;
+        if (x.w == x.w) w[3] = (double)expf(x.w - mcs) * scs;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) if (w[k] > 0.0) last_w = v + k;
+      }
+      const double l4 = (w[0] + w[1]) + (w[2] + w[3]);
+      double sub_total;
+      const double inc4 = block_scan(l4, s_warp, &sub_total);
+      double acc = running + inc4 - l4;
+      if (l4 > 0.0 && acc <= T && T < acc + l4) {
+        int pick = -1;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          if (pick < 0 && w[k] > 0.0) { acc += w[k]; if (acc > T) pick = v + k; }
+        }
+        if (pick < 0) pick = last_w;                     // rounding inside the four: their last with weight
+        s_tok = pick;
+      }
+      __syncthreads();
+      if (s_tok >= 0) break;
+      running += sub_total;
+    }
+    if (s_tok < 0) {
+      // summation order put the threshold past this chunk's end: its last element with weight
+      atomicMax(&s_tok, last_w);
+      __syncthreads();
+    }
+    tok = s_tok < 0 ? 0 : s_tok;
+  }
+  if (tid == 0) {
+    next_tokens[(size_t)n * block + step] = tok;
+    tick[n] = 0u;                                        // the next step finds the ticket at zero
+  }
+}
+}  // namespace
+
 size_t head_workspace_bytes(int b, int block, int vocab) {
   if (b <= 0 || block <= 0 || vocab <= 0) return 0;
   const size_t logits = (((size_t)b * block * vocab * sizeof(float)) + 255) & ~size_t(255);
-  return logits + (size_t)block * kMaxBatch * kBestStride * sizeof(unsigned long long) + 256;
+  const size_t zstep = (((size_t)b * vocab * sizeof(float)) + 255) & ~size_t(255);   // sampling: one step's logits
+  return logits + (size_t)block * kMaxBatch * kBestStride * sizeof(unsigned long long) + 256 + zstep +
+         (size_t)kMaxBatch * kPickMaxChunks * sizeof(PickPart);
 }
 
 dpara_status launch_head(const HeadArgs &h, void *workspace, int32_t *status, cudaStream_t st) {
@@ -297,6 +496,7 @@ dpara_status launch_head(const HeadArgs &h, void *workspace, int32_t *status, cu
   const size_t logits_bytes = (((size_t)h.b * h.block * h.vocab * sizeof(float)) + 255) & ~size_t(255);
   unsigned long long *best = reinterpret_cast<unsigned long long *>(ws + logits_bytes);
   unsigned int *barrier = reinterpret_cast<unsigned int *>(best + (size_t)h.block * kMaxBatch * kBestStride);
+  float *zstep = reinterpret_cast<float *>(reinterpret_cast<uint8_t *>(barrier) + 256);
   if (cudaMemsetAsync(best, 0, (size_t)h.block * kMaxBatch * kBestStride * sizeof(unsigned long long) + 256, st) != cudaSuccess) return DPARA_ERR_CUDA;
 
   // base logits of the selected branches, fp32, stored step-major [block][b][vocab] (GEMM row n * block + i goes
@@ -321,13 +521,31 @@ dpara_status launch_head(const HeadArgs &h, void *workspace, int32_t *status, cu
   const int fixed = (h.rank / 64) * P.nb * 128 + 1024 + 2048;   // Ey, alignment slack, barriers and reduction scratch
   P.stages = (227 * 1024 - fixed) / stage_bytes > 4 ? 4 : (227 * 1024 - fixed) / stage_bytes;
   const int smem = P.stages * stage_bytes + fixed;
-  if (cudaFuncSetAttribute(ar_head_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return DPARA_ERR_CUDA;
+  if (cudaFuncSetAttribute(ar_head_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
+      cudaFuncSetAttribute(ar_head_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return DPARA_ERR_CUDA;
   int dev = 0, sms = kNumSM;
   if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  // cooperative launch: the grid barrier needs every CTA resident (one CTA per SM fits by construction)
   const int grid = P.n_tiles < sms ? P.n_tiles : sms;
+  if (h.uniforms) {
+    // ---- sampling: per step the logits z (one-step head kernel), then the draw.  The tickets live in the zeroed 256 bytes
+    // after the greedy path's barrier word (kMaxBatch words from byte 128).
+    unsigned int *tick = barrier + 32;
+    PickPart *part = reinterpret_cast<PickPart *>(reinterpret_cast<uint8_t *>(zstep) + ((((size_t)h.b * h.vocab * sizeof(float)) + 255) & ~size_t(255)));
+    const int chunk = pick_chunk_elems(h.vocab), n_chunks = (h.vocab + chunk - 1) / chunk;
+    P.z_out = zstep;
+    for (int i = 0; i < h.block; ++i) {
+      P.step0 = i;
+      ar_head_kernel<true><<<grid, kThreads, smem, st>>>(P);
+      DPARA_CHECK_LAUNCH();
+      head_sample_kernel<<<dim3(n_chunks, h.b), kPickThreads, 0, st>>>(zstep, h.uniforms, h.next_tokens, part, tick, h.vocab, h.block, i, chunk);
+      DPARA_CHECK_LAUNCH();
+      count_launches(2);
+    }
+    return DPARA_OK;
+  }
+  // cooperative launch: the grid barrier needs every CTA resident (one CTA per SM fits by construction)
   void *args[] = {&P};
-  if (cudaLaunchCooperativeKernel(reinterpret_cast<void *>(ar_head_kernel), dim3(grid), dim3(kThreads), args, smem, st) != cudaSuccess) {
+  if (cudaLaunchCooperativeKernel(reinterpret_cast<void *>(ar_head_kernel<false>), dim3(grid), dim3(kThreads), args, smem, st) != cudaSuccess) {
     cudaGetLastError();
     return DPARA_ERR_CUDA;
   }

@@ -12,6 +12,7 @@ struct HeadArgs {
   const int32_t *bonus;      // [b]
   int32_t *next_tokens;      // [b][block]
   int b, block, hidden, vocab, rank;
+  const float *uniforms;     // [b][block] or null: null = greedy, else y_i is drawn from softmax(z_i) with uniforms[n][i-1]
 };
 
 size_t head_workspace_bytes(int b, int block, int vocab);

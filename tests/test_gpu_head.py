@@ -127,3 +127,69 @@ def test_head_full_size_sampled():
         z = H.ar_logits(row, inp.ar_w, inp.ar_e, y_prev)
         want, got = int(np.argmax(z)), int(toks[n, i])
         assert got == want or z[got] >= z[want] - TIE * max(1.0, float(np.abs(z).max())), (n, i, got, want)
+
+
+# ----------------------------------------------------------------------------- sampling head loop
+def _check_sampling(inp, toks, logits, uniforms, eps=2e-5):
+    """Step by step with the kernel's own previous token: the kernel's token v must satisfy the oracle's inverse-CDF rule
+    up to rounding -- u inside [C(v-1) - eps, C(v) + eps] of the oracle's float64 cumulative softmax (the kernel's logits are
+    fp32 accumulations, relative error ~3e-6, which moves every cumulative value by about that much)."""
+    sh = inp.shape
+    exact = 0
+    for n in range(sh.batch):
+        y = int(inp.bonus[n])
+        base = H.lm_head(inp.sel_reps[n], inp.w_lm)
+        for i in range(sh.block):
+            assert np.abs(logits[n * sh.block + i] - base[i]).max() <= TIE * max(1.0, float(np.abs(base[i]).max()))
+            z = H.ar_logits(base[i], inp.ar_w, inp.ar_e, y)
+            u = float(uniforms[n, i])
+            want = H.sample_from_logits(z, u)
+            got = int(toks[n, i])
+            assert 0 <= got < sh.vocab
+            w = np.exp(z - z.max())
+            c = np.cumsum(w) / w.sum()
+            lo = c[got - 1] if got > 0 else 0.0
+            assert lo - eps <= u <= c[got] + eps, (n, i, got, want, u, lo, c[got])
+            exact += got == want
+            y = got
+    return exact
+
+
+@pytest.mark.parametrize("shape", [
+    W.HeadShape(3, 4, 128, 1000, 64),
+    W.HeadShape(16, 8, 512, 20000 + 8, 256),
+    W.HeadShape(20, 5, 256, 4096, 128),
+    W.HeadShape(2, 6, 1024, 151936, 256),      # the full vocabulary
+])
+def test_head_sampling_parity(shape):
+    inp = W.make_head_inputs(shape, 31)
+    rng = np.random.default_rng(8)
+    uniforms = (rng.integers(0, 1 << 24, size=(shape.batch, shape.block)) * 2.0 ** -24).astype(np.float32)
+    uniforms[0, 0] = 0.0
+    uniforms[-1, -1] = np.float32(1 - 2.0 ** -24)
+    t = [dev_bf16(x) for x in (inp.sel_reps, inp.w_lm, inp.ar_w, inp.ar_e)]
+    toks, plan = dp.draft_head(t[0], t[1], t[2], t[3], torch.from_numpy(inp.bonus).cuda(), uniforms=torch.from_numpy(uniforms).cuda())
+    torch.cuda.synchronize()
+    assert plan.status.item() == 0
+    exact = _check_sampling(inp, toks.cpu().numpy(), plan.base_logits().cpu().numpy().astype(np.float64), uniforms)
+    assert exact >= 0.98 * shape.batch * shape.block        # a different token than the oracle's is the rare boundary case
+
+
+def test_head_sampling_repeats_and_leaves_greedy_unchanged():
+    """Two runs with the same uniforms give the same tokens, and a greedy run on the same plan's workspace after a sampling
+    run gives what it gave before (the sampling path leaves no state behind)."""
+    sh = W.HeadShape(4, 6, 256, 8192, 64)
+    inp = W.make_head_inputs(sh, 5)
+    t = [dev_bf16(x) for x in (inp.sel_reps, inp.w_lm, inp.ar_w, inp.ar_e)]
+    bonus = torch.from_numpy(inp.bonus).cuda()
+    u = torch.rand(4, 6, device="cuda") * (1 - 2.0 ** -20)
+    g, plan = dp.draft_head(t[0], t[1], t[2], t[3], bonus)
+    g = g.clone()
+    s1 = plan.run(t[0], t[1], t[2], t[3], bonus, uniforms=u).clone()
+    s2 = plan.run(t[0], t[1], t[2], t[3], bonus, uniforms=u).clone()
+    g2 = plan.run(t[0], t[1], t[2], t[3], bonus).clone()
+    torch.cuda.synchronize()
+    assert plan.status.item() == 0
+    assert torch.equal(s1, s2)
+    assert torch.equal(g, g2)
+    assert not torch.equal(s1, g)
