@@ -16,8 +16,10 @@
  * Conventions
  *   - Every pointer is a DEVICE pointer unless its name starts with host_.  The caller owns every
  *     buffer; the library allocates nothing.  The only state it keeps between calls is a process-wide
- *     launch counter (dpara_kernel_launches) and, for the fixed-scratch entry point, that entry's
- *     scratch array and its cached device address.
+ *     launch counter (dpara_kernel_launches), the last attention work schedule with the key-tile counts
+ *     it was built for (a pure function of those counts, kept in host memory to save host time when they
+ *     repeat) and, for the fixed-scratch entry point, that entry's scratch array and its cached device
+ *     address.
  *   - Calls enqueue kernels on `stream` (a cudaStream_t passed as void*) and return without
  *     synchronising.  Outputs are valid once the stream has reached the end of the call's work.
  *   - The return code reports host-detectable errors.  Argument errors (INVALID_ARG, UNSUPPORTED,
