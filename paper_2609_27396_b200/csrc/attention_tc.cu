@@ -745,7 +745,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
     if (warp < 8 && !*abort_flag) {
       const Item I = decode_item(P, blockIdx.x);
       const uint32_t rank = cluster_ctarank();
-      const int rows_per = 256 / P.nsplit;
+      const int rows_per = I.ntq * 128 / P.nsplit;  // the item's rows (one tile or two), shared out over the cluster
       merge_pieces<D>(P, I, P.nsplit, (int)rank * rows_per, rows_per, threadIdx.x);
     }
   }
@@ -794,6 +794,35 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
 }
 
 // ------------------------------------------------------------------------------------------------ host
+// Clusters of `size` CTAs of this kernel that the device runs at the same time (one CTA per SM, a cluster inside one
+// GPC: fewer than SMs / size).  Asked once per (head dim, size); without a device, a careful guess.
+static int max_active_clusters(int D, int size) {
+  static std::mutex mu;
+  static int cached[2][4] = {{0, 0, 0, 0}, {0, 0, 0, 0}};
+  const int di = D == 128 ? 1 : 0, si = size == 8 ? 3 : (size == 4 ? 2 : (size == 2 ? 1 : 0));
+  std::lock_guard<std::mutex> lock(mu);
+  if (cached[di][si] > 0) return cached[di][si];
+  int n = 0;
+  cudaLaunchConfig_t cfg = {};
+  cudaLaunchAttribute attr[1];
+  cfg.gridDim = dim3(size * kNumSM);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = D == 128 ? TcCfg<128>::kSmemBytes : TcCfg<64>::kSmemBytes;
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = size; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  cudaError_t e = D == 128 ? cudaFuncSetAttribute(attn_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)cfg.dynamicSmemBytes)
+                           : cudaFuncSetAttribute(attn_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)cfg.dynamicSmemBytes);
+  if (e == cudaSuccess)
+    e = D == 128 ? cudaOccupancyMaxActiveClusters(&n, attn_tc_kernel<128>, &cfg) : cudaOccupancyMaxActiveClusters(&n, attn_tc_kernel<64>, &cfg);
+  if (e != cudaSuccess || n <= 0) {
+    cudaGetLastError();
+    return (kNumSM * 3 / 4) / size;   // not cached: a later call with a device asks again
+  }
+  cached[di][si] = n;
+  return n;
+}
+
 TcPlan plan_attention_tc(const dpara_shape *s, const int64_t *host_off, const int64_t *host_lens) {
   auto len_of = [&](int n) { return host_lens ? host_lens[n] : host_off[n + 1] - host_off[n]; };
   TcPlan p{};
@@ -804,33 +833,49 @@ TcPlan plan_attention_tc(const dpara_shape *s, const int64_t *host_off, const in
   p.n_ji = nb * s->block;
   p.n_rows = p.n_ji + (s->spine_queries ? s->n_spine : 0);
   // head blocks = binary digits of G, widest first; block k's tiles hold 128 / hb (j, i) rows
-  p.n_hblk = 0;
-  p.n_pairs = 0;
-  for (int bit = 4, h0 = 0; bit >= 0; --bit) {
-    if (!(G & (1 << bit))) continue;
-    const int ji_t = 128 >> bit, tiles = (p.n_rows + ji_t - 1) / ji_t;
-    p.hb_log2[p.n_hblk] = bit;
-    p.h0[p.n_hblk] = h0;
+  auto lay_out_items = [&](int tiles_per_item) {
+    p.tiles_per_item = tiles_per_item;
+    p.n_hblk = 0;
+    p.n_pairs = 0;
+    for (int bit = 4, h0 = 0; bit >= 0; --bit) {
+      if (!(G & (1 << bit))) continue;
+      const int ji_t = 128 >> bit, tiles = (p.n_rows + ji_t - 1) / ji_t;
+      p.hb_log2[p.n_hblk] = bit;
+      p.h0[p.n_hblk] = h0;
+      p.pair_start[p.n_hblk] = p.n_pairs;
+      p.n_pairs += (tiles + tiles_per_item - 1) / tiles_per_item;
+      h0 += 1 << bit;
+      ++p.n_hblk;
+    }
     p.pair_start[p.n_hblk] = p.n_pairs;
-    p.n_pairs += (tiles + 1) / 2;
-    h0 += 1 << bit;
-    ++p.n_hblk;
-  }
-  p.pair_start[p.n_hblk] = p.n_pairs;
+  };
+  lay_out_items(2);
   p.S8 = (s->n_spine + 7) & ~7;
   p.cap = 128 / s->block;
   p.cap0 = (128 - p.S8) / s->block;  // >= 1: S8 <= 64 and block <= 64
   long long max_l = 0, tot = host_off[s->batch] - host_off[0];
   for (int n = 0; n < s->batch; ++n) max_l = len_of(n) > max_l ? len_of(n) : max_l;
   if (tot + 128 >= (1ll << 31) || (long long)s->batch * s->n_boundaries * s->block >= (1ll << 31)) return p;
-  const long long items = (long long)s->batch * s->n_kv_heads * p.n_pairs;
   const int max_tiles = (int)((max_l + 127) / 128);
+  // A small batch is latency-bound: when one-tile items with their splits still fit the GPU in a single wave, an item is
+  // ONE query tile instead of two -- twice the CTAs, each with half the Q load, half the partial rows and half the merge
+  int split_cap = 8;  // largest cluster size whose clusters all run at once
+  {
+    const int pairs2 = p.n_pairs;
+    lay_out_items(1);
+    const long long items1 = (long long)s->batch * s->n_kv_heads * p.n_pairs;
+    int split1 = 0;
+    for (int c = 8; c >= 2 && !split1; c >>= 1)
+      if (c <= max_tiles && items1 <= max_active_clusters(s->head_dim, c)) split1 = c;
+    if (p.n_pairs == pairs2 || items1 >= 96 || split1 < 4) lay_out_items(2); else split_cap = split1;
+  }
+  const long long items = (long long)s->batch * s->n_kv_heads * p.n_pairs;
   // split the KV range over a cluster of 2, 4 or 8 CTAs when the batch alone cannot fill the GPU
   int nsplit = 1;
   if (items < 96 && max_tiles > 1) {
     const long long want = (kNumSM + items - 1) / items;
     for (int c = 8; c >= 2; c >>= 1)
-      if (c <= want && c <= max_tiles) { nsplit = c; break; }
+      if (c <= want && c <= max_tiles && c <= split_cap) { nsplit = c; break; }
   }
   p.nsplit = nsplit;
   p.items = items;
@@ -900,9 +945,10 @@ dpara_status launch_attention_tc(const AttnParams &A, const TcPlan &plan, const 
     int blk = 0;
     while (blk + 1 < plan.n_hblk && x >= plan.pair_start[blk + 1]) ++blk;
     const int ji_t = 128 >> plan.hb_log2[blk], pl = x - plan.pair_start[blk];
-    const int ntq = std::min(2, (plan.n_rows + ji_t - 1) / ji_t - pl * 2);
+    const int tpi = plan.tiles_per_item;
+    const int ntq = std::min(tpi, (plan.n_rows + ji_t - 1) / ji_t - pl * tpi);
     // boundaries whose own blocks the pair's mask-slot rows need (none if the pair holds spine rows only)
-    const int ji0 = pl * 2 * ji_t, ji_last = std::min(ji0 + ntq * ji_t, plan.n_ji) - 1;
+    const int ji0 = pl * tpi * ji_t, ji_last = std::min(ji0 + ntq * ji_t, plan.n_ji) - 1;
     TcParams::PairInfo &pi = P.pair[x];
     pi.ji0 = (int16_t)ji0;
     pi.jb0_rel = (int16_t)(ji0 / A.Bq);

@@ -6,7 +6,8 @@ namespace dpara {
 
 struct TcPlan {
   bool eligible;        // false: shape outside what the tensor-core kernel handles (use the general kernel)
-  int n_ji, n_pairs;    // (boundary, slot) rows per request; tile pairs per (request, KV head), all head blocks
+  int n_ji, n_pairs;    // (boundary, slot) rows per request; items (tile pairs, or single tiles) per (request, KV head), all head blocks
+  int tiles_per_item;   // 2: an item is a pair of 128-row query tiles; 1: a single tile (small batches)
   int n_rows;           // query rows per request and head: n_ji, plus the spine rows when they are queries
   int n_hblk, hb_log2[4], h0[4], pair_start[5];  // head blocks (binary digits of the group size) and their tile pairs
   int nsplit;           // KV splits per (request, KV head, tile pair)

@@ -22,13 +22,15 @@ constexpr int kBM = 128, kBN = 256, kBK = 64, kStages = 4;
 constexpr int kABytes = kBM * kBK * 2;         // 16 KB
 constexpr int kBBytes = kBN * kBK * 2;         // 32 KB (two 128-row boxes)
 constexpr int kStageBytes = kABytes + kBBytes;  // 48 KB
-constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*align*/ + 256 /*barriers*/;
+constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*align*/ + 256 /*barriers*/ + 4 * 32 * 36 * 4 /*epilogue staging*/;
 constexpr int kThreads = 192;                   // warps 0-3 epilogue, 4 TMA, 5 MMA
 }  // namespace
 
 struct GemmKernelParams {
-  CUtensorMap map_a;
-  CUtensorMap map_b;
+  CUtensorMap map_a[kGemmMaxGroups];   // one entry per product of a grouped launch (a plain launch uses entry 0)
+  CUtensorMap map_b[kGemmMaxGroups];
+  void *out_g[kGemmMaxGroups];         // grouped launch: the products' outputs
+  int n_groups;
   int M, N, K;
   int epi;
   int up_row_offset;
@@ -38,88 +40,83 @@ struct GemmKernelParams {
   void *out_bf16;
   int32_t *status;
   int perm_block, perm_b;
+  int split_k;   // > 1 (fp32 store only, CTA pairs): the K range in split_k parts, part s writes plane s of [split_k][M][N] partial sums
 };
 
 __device__ __forceinline__ float silu_f(float g) { return g / (1.0f + __expf(-g)); }
 
-// Epilogue of one accumulator tile: thread = one accumulator row (`row` of the output), `taddr` = this warp's lanes
-// of the accumulator buffer.
-__device__ __forceinline__ void gemm_epilogue(const GemmKernelParams &P, uint32_t taddr, int row, int n_tile) {
-      if (P.epi == 2) {
-        const int col0 = n_tile * 128;
+// Epilogue of one accumulator tile.  A thread reads one accumulator ROW from tensor memory (lane = row), 32 columns at
+// a time; stored like that, one warp instruction would touch 32 rows x 16 bytes -- 32 cache lines for 512 bytes.  Each
+// 32 x 32 block therefore goes through a per-warp shared-memory buffer (row pitch 36 floats: conflict-free both ways)
+// and comes back with 8 lanes on one row: an instruction then covers 4 rows x 128 contiguous bytes, for the residual
+// read as well as for the stores.  `row_base` = output row of lane 0, `stage` = this warp's 32 x 36 floats.
+constexpr int kEpiPitch = 36;
+
+__device__ __forceinline__ void gemm_epilogue(const GemmKernelParams &P, uint32_t taddr, int row_base, int n_tile, float *stage, int lane, int ks,
+                                              int grp) {
+  // fp32 output of this product; split K (fp32 store only): plane ks of the partial sums
+  float *out_f32 = static_cast<float *>(P.n_groups > 1 ? P.out_g[grp] : P.out) + (size_t)ks * P.M * P.N;
+  const int n_chunks = P.epi == 2 ? 4 : kBN / 32;
+  const int col0 = n_tile * (P.epi == 2 ? 128 : kBN);
+  const int sub_row = lane >> 3, piece = lane & 7;
 #pragma unroll 1
-        for (int c = 0; c < 4; ++c) {
-          uint32_t g[32], u[32];
-          tmem_ld32(taddr + c * 32, g);
-          tmem_ld32(taddr + 128 + c * 32, u);
-          tmem_wait_ld();
-          if (row < P.M) {
-            uint16_t *o = static_cast<uint16_t *>(P.out) + (size_t)row * P.N + col0 + c * 32;
+  for (int c = 0; c < n_chunks; ++c) {
+    uint32_t r[32];
+    tmem_ld32(taddr + c * 32, r);
+    if (P.epi == 2) {
+      uint32_t u[32];
+      tmem_ld32(taddr + 128 + c * 32, u);
+      tmem_wait_ld();
 #pragma unroll
-            for (int v = 0; v < 4; ++v) {
-              if (col0 + c * 32 + v * 8 < P.N) {
-                uint32_t w[4];
+      for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(silu_f(__uint_as_float(r[e])) * __uint_as_float(u[e]));
+    } else {
+      tmem_wait_ld();
+    }
+    float4 *mine = reinterpret_cast<float4 *>(stage + lane * kEpiPitch);
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                  float a0 = silu_f(__uint_as_float(g[v * 8 + 2 * e])) * __uint_as_float(u[v * 8 + 2 * e]);
-                  float a1 = silu_f(__uint_as_float(g[v * 8 + 2 * e + 1])) * __uint_as_float(u[v * 8 + 2 * e + 1]);
-                  w[e] = pack_bf16(a0, a1);
-                }
-                *reinterpret_cast<uint4 *>(o + v * 8) = make_uint4(w[0], w[1], w[2], w[3]);
-              }
-            }
-          }
+    for (int v = 0; v < 8; ++v)
+      mine[v] = make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]), __uint_as_float(r[4 * v + 2]), __uint_as_float(r[4 * v + 3]));
+    __syncwarp();
+    const int col = col0 + c * 32 + piece * 4;
+    if (col < P.N) {
+      // the residual rows first, all in flight together
+      float4 rr[8];
+      if (P.epi == 1) {
+        // (rows past M read row M - 1: an unconditional load the compiler can issue early; the value is not used)
+        if (P.resid_bf16) {
+          uint2 q[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i)
+            q[i] = *reinterpret_cast<const uint2 *>(static_cast<const uint16_t *>(P.resid) + (size_t)min(row_base + i * 4 + sub_row, P.M - 1) * P.N + col);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) rr[i] = make_float4(bf16lo(q[i].x), bf16hi(q[i].x), bf16lo(q[i].y), bf16hi(q[i].y));
+        } else {
+#pragma unroll
+          for (int i = 0; i < 8; ++i)
+            rr[i] = *reinterpret_cast<const float4 *>(static_cast<const float *>(P.resid) + (size_t)min(row_base + i * 4 + sub_row, P.M - 1) * P.N + col);
         }
-      } else {
-        const int col0 = n_tile * kBN;
-#pragma unroll 1
-        for (int c = 0; c < kBN / 32; ++c) {
-          uint32_t r[32];
-          tmem_ld32(taddr + c * 32, r);
-          tmem_wait_ld();
-          if (row < P.M) {
-            const int cb = col0 + c * 32;
-            if (P.epi == 0) {
-              uint16_t *o = static_cast<uint16_t *>(P.out) + (size_t)row * P.N + cb;
+      }
 #pragma unroll
-              for (int v = 0; v < 4; ++v) {
-                if (cb + v * 8 < P.N) {
-                  uint32_t w[4];
-#pragma unroll
-                  for (int e = 0; e < 4; ++e)
-                    w[e] = pack_bf16(__uint_as_float(r[v * 8 + 2 * e]), __uint_as_float(r[v * 8 + 2 * e + 1]));
-                  *reinterpret_cast<uint4 *>(o + v * 8) = make_uint4(w[0], w[1], w[2], w[3]);
-                }
-              }
-            } else {
-              const int orow = P.perm_block ? (row % P.perm_block) * P.perm_b + row / P.perm_block : row;
-              float *o = static_cast<float *>(P.out) + (size_t)orow * P.N + cb;
-#pragma unroll
-              for (int v = 0; v < 8; ++v) {
-                if (cb + v * 4 < P.N) {
-                  float x[4];
-                  if (P.epi == 3) {
-                    x[0] = x[1] = x[2] = x[3] = 0.f;
-                  } else if (P.resid_bf16) {
-                    uint2 rr = *reinterpret_cast<const uint2 *>(static_cast<const uint16_t *>(P.resid) + (size_t)row * P.N + cb + v * 4);
-                    x[0] = bf16lo(rr.x); x[1] = bf16hi(rr.x); x[2] = bf16lo(rr.y); x[3] = bf16hi(rr.y);
-                  } else {
-                    float4 rr = *reinterpret_cast<const float4 *>(static_cast<const float *>(P.resid) + (size_t)row * P.N + cb + v * 4);
-                    x[0] = rr.x; x[1] = rr.y; x[2] = rr.z; x[3] = rr.w;
-                  }
-#pragma unroll
-                  for (int e = 0; e < 4; ++e) x[e] += __uint_as_float(r[v * 4 + e]);
-                  *reinterpret_cast<float4 *>(o + v * 4) = make_float4(x[0], x[1], x[2], x[3]);
-                  if (P.out_bf16) {
-                    uint16_t *ob = static_cast<uint16_t *>(P.out_bf16) + (size_t)row * P.N + cb + v * 4;
-                    *reinterpret_cast<uint2 *>(ob) = make_uint2(pack_bf16(x[0], x[1]), pack_bf16(x[2], x[3]));
-                  }
-                }
-              }
-            }
+      for (int i = 0; i < 8; ++i) {
+        const int rl = i * 4 + sub_row, row = row_base + rl;
+        const float4 a = *reinterpret_cast<const float4 *>(stage + rl * kEpiPitch + piece * 4);
+        if (row < P.M) {
+          if (P.epi == 0 || P.epi == 2) {
+            uint16_t *o = static_cast<uint16_t *>(P.out) + (size_t)row * P.N + col;
+            *reinterpret_cast<uint2 *>(o) = make_uint2(pack_bf16(a.x, a.y), pack_bf16(a.z, a.w));
+          } else {
+            const int orow = P.perm_block ? (row % P.perm_block) * P.perm_b + row / P.perm_block : row;
+            float4 x = a;
+            if (P.epi == 1) { x.x += rr[i].x; x.y += rr[i].y; x.z += rr[i].z; x.w += rr[i].w; }
+            *reinterpret_cast<float4 *>(out_f32 + (size_t)orow * P.N + col) = x;
+            if (P.out_bf16)
+              *reinterpret_cast<uint2 *>(static_cast<uint16_t *>(P.out_bf16) + (size_t)row * P.N + col) = make_uint2(pack_bf16(x.x, x.y), pack_bf16(x.z, x.w));
           }
         }
       }
+    }
+    __syncwarp();
+  }
 }
 
 __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_constant__ GemmKernelParams P) {
@@ -164,8 +161,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
   // Two accumulator buffers in TMEM let the epilogue of one tile overlap the main loop of the next.
   if (warp == 4) {
     if (lane == 0) {
-      prefetch_tensormap(&P.map_a);
-      prefetch_tensormap(&P.map_b);
+      prefetch_tensormap(&P.map_a[0]);
+      prefetch_tensormap(&P.map_b[0]);
       int stage = 0;
       uint32_t ph = 0;
       bool ok = true;
@@ -178,9 +175,9 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
           if (!ok) break;
           uint8_t *sa = smem + stage * kStageBytes;
           mbar_arrive_expect_tx(full + stage, kStageBytes);
-          tma_load_2d(sa, &P.map_a, full + stage, kb * kBK, m_tile * kBM);
-          tma_load_2d(sa + kABytes, &P.map_b, full + stage, kb * kBK, brow0);
-          tma_load_2d(sa + kABytes + 128 * kBK * 2, &P.map_b, full + stage, kb * kBK, brow1);
+          tma_load_2d(sa, &P.map_a[0], full + stage, kb * kBK, m_tile * kBM);
+          tma_load_2d(sa + kABytes, &P.map_b[0], full + stage, kb * kBK, brow0);
+          tma_load_2d(sa + kABytes + 128 * kBK * 2, &P.map_b[0], full + stage, kb * kBK, brow1);
           if (++stage == kStages) { stage = 0; ph ^= 1u; }
         }
       }
@@ -223,11 +220,11 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
     // ---------------- epilogue: thread = one accumulator row
     const bool ok = __all_sync(0xffffffffu, mbar_wait(acc_full + buf, (k >> 1) & 1, abort_flag));  // warp-uniform: tcgen05.ld is warp-wide
     tc_fence_after();
-    const int row = m_tile * kBM + warp * 32 + lane;
+    const int row_base = m_tile * kBM + warp * 32;
     const uint32_t taddr = tmem + buf * kBN + ((uint32_t)(warp * 32) << 16);
     live = ok;
     if (ok) {
-      gemm_epilogue(P, taddr, row, n_tile);
+      gemm_epilogue(P, taddr, row_base, n_tile, reinterpret_cast<float *>(smem + kStages * kStageBytes + 256) + warp * 32 * kEpiPitch, lane, 0, 0);
     }
     // this warp has read its part of the accumulator: hand the buffer back to the MMA issuer
     tc_fence_before();
@@ -254,7 +251,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
 namespace {
 constexpr int kStages2 = 6;
 constexpr int kStageBytes2 = kABytes + 128 * kBK * 2;  // 32 KB: 128 activation rows + 128 weight rows
-constexpr int kSmemBytes2 = kStages2 * kStageBytes2 + 1024 + 256;
+constexpr int kSmemBytes2 = kStages2 * kStageBytes2 + 1024 + 256 + 4 * 32 * 36 * 4;
 }  // namespace
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1) gemm_tc2_kernel(const __grid_constant__ GemmKernelParams P) {
@@ -273,7 +270,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1) gemm_tc
   const int nkb = P.K / kBK;
   const int tile_cols = P.epi == 2 ? 128 : kBN;
   const int m_pairs = (P.M + 2 * kBM - 1) / (2 * kBM), n_tiles = (P.N + tile_cols - 1) / tile_cols;
-  const int total_tiles = m_pairs * n_tiles;
+  const int group_units = m_pairs * n_tiles * P.split_k;   // work units of one product: (tile, K part), the parts of a tile adjacent
+  const int total_tiles = group_units * P.n_groups;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages2; ++s) {
@@ -299,23 +297,28 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1) gemm_tc
 
   if (warp == 4) {
     if (lane == 0) {
-      prefetch_tensormap(&P.map_a);
-      prefetch_tensormap(&P.map_b);
+      for (int gi = 0; gi < P.n_groups; ++gi) {
+        prefetch_tensormap(&P.map_a[gi]);
+        prefetch_tensormap(&P.map_b[gi]);
+      }
       int stage = 0;
       uint32_t ph = 0;
       bool ok = true;
-      for (int tile = pair; tile < total_tiles && ok; tile += n_pairs) {
+      for (int unit0 = pair; unit0 < total_tiles && ok; unit0 += n_pairs) {
+        const int grp = unit0 / group_units, unit = unit0 - grp * group_units;
+        const int tile = unit / P.split_k, ks = unit - tile * P.split_k;
         const int m_pair = tile % m_pairs, n_tile = tile / m_pairs;
+        const int kb0 = ks * nkb / P.split_k, kb1 = (ks + 1) * nkb / P.split_k;
         // this CTA's half of the weight tile: rows [rank * 128, +128) of the tile (SwiGLU: gate rows / up rows)
         const int brow = P.epi == 2 ? (rank == 0 ? n_tile * 128 : P.up_row_offset + n_tile * 128) : n_tile * kBN + (int)rank * 128;
         const int arow = (m_pair * 2 + (int)rank) * kBM;
-        for (int kb = 0; kb < nkb; ++kb) {
+        for (int kb = kb0; kb < kb1; ++kb) {
           ok = mbar_wait(empty + stage, ph ^ 1u, abort_flag, 2);
           if (!ok) break;
           uint8_t *sa = smem + stage * kStageBytes2;
           if (rank == 0) mbar_arrive_expect_tx(full + stage, 2u * kStageBytes2);
-          tma_load_2d_pair(sa, &P.map_a, full + stage, kb * kBK, arow);
-          tma_load_2d_pair(sa + kABytes, &P.map_b, full + stage, kb * kBK, brow);
+          tma_load_2d_pair(sa, &P.map_a[grp], full + stage, kb * kBK, arow);
+          tma_load_2d_pair(sa + kABytes, &P.map_b[grp], full + stage, kb * kBK, brow);
           if (++stage == kStages2) { stage = 0; ph ^= 1u; }
         }
       }
@@ -328,18 +331,20 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1) gemm_tc
       int stage = 0, k = 0;
       uint32_t ph = 0;
       bool ok = true;
-      for (int tile = pair; tile < total_tiles && ok; tile += n_pairs, ++k) {
+      for (int unit0 = pair; unit0 < total_tiles && ok; unit0 += n_pairs, ++k) {
+        const int ks = (unit0 % group_units) % P.split_k;
+        const int kb0 = ks * nkb / P.split_k, kb1 = (ks + 1) * nkb / P.split_k;
         const int buf = k & 1;
         ok = mbar_wait(acc_empty + buf, ((k >> 1) & 1) ^ 1u, abort_flag, 3);  // both CTAs' epilogues of tile k - 2 are done
         if (!ok) break;
         tc_fence_after();
         const uint32_t acc = tmem + buf * kBN;
-        for (int kb = 0; kb < nkb; ++kb) {
+        for (int kb = kb0; kb < kb1; ++kb) {
           ok = mbar_wait(full + stage, ph, abort_flag, 4);
           if (!ok) break;
           tc_fence_after();
           const uint64_t so = (uint64_t)(stage * (kStageBytes2 >> 4));
-          mma2_ss(acc, adesc0 + so, bdesc0 + so, idesc, kb != 0);
+          mma2_ss(acc, adesc0 + so, bdesc0 + so, idesc, kb != kb0);
 #pragma unroll
           for (int kk = 1; kk < kBK / 16; ++kk) mma2_ss_c<true>(acc, adesc0 + so + 2 * kk, bdesc0 + so + 2 * kk, idesc);
           mma2_commit_both(empty + stage);
@@ -351,15 +356,17 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1) gemm_tc
   } else {
     int k = 0;
     bool live = true;
-    for (int tile = pair; tile < total_tiles && live; tile += n_pairs, ++k) {
+    for (int unit0 = pair; unit0 < total_tiles && live; unit0 += n_pairs, ++k) {
+      const int grp = unit0 / group_units, unit = unit0 - grp * group_units;
+      const int tile = unit / P.split_k, ks = unit - tile * P.split_k;
       const int m_pair = tile % m_pairs, n_tile = tile / m_pairs;
       const int buf = k & 1;
       const bool ok = __all_sync(0xffffffffu, mbar_wait(acc_full + buf, (k >> 1) & 1, abort_flag, 5));
       tc_fence_after();
-      const int row = (m_pair * 2 + (int)rank) * kBM + warp * 32 + lane;
+      const int row_base = (m_pair * 2 + (int)rank) * kBM + warp * 32;
       const uint32_t taddr = tmem + buf * kBN + ((uint32_t)(warp * 32) << 16);
       live = ok;
-      if (ok) gemm_epilogue(P, taddr, row, n_tile);
+      if (ok) gemm_epilogue(P, taddr, row_base, n_tile, reinterpret_cast<float *>(smem + kStages2 * kStageBytes2 + 256) + warp * 32 * kEpiPitch, lane, ks, grp);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_leader(acc_empty + buf);
@@ -380,11 +387,28 @@ dpara_status launch_gemm_tc(const GemmArgs &g, int32_t *status, cudaStream_t st)
   if (!aligned16(g.a) || !aligned16(g.w) || !aligned16(g.out) || !aligned16(g.resid) || !aligned16(g.out_bf16)) return DPARA_ERR_INVALID_ARG;
   GemmKernelParams P;
   const int w_rows = g.epi == 2 ? 2 * g.N : g.N;
-  if (!make_tmap_bf16_2d(&P.map_a, g.a, g.K, g.M, (uint64_t)g.K * 2, kBK, kBM)) return DPARA_ERR_CUDA;
-  if (!make_tmap_bf16_2d(&P.map_b, g.w, g.K, w_rows, (uint64_t)g.K * 2, kBK, 128)) return DPARA_ERR_CUDA;
+  P.n_groups = 1;
+  if (g.n_groups > 1) {
+    // several products of one shape in one launch (fp32 stores, CTA pairs): entry 0 of the lists is (a, w, out)
+    if (g.epi != 3 || g.M <= kBM || g.n_groups > kGemmMaxGroups || g.perm_block) return DPARA_ERR_UNSUPPORTED;
+    P.n_groups = g.n_groups;
+  }
+  for (int gi = 0; gi < P.n_groups; ++gi) {
+    const void *a = gi ? g.a_g[gi] : g.a, *w = gi ? g.w_g[gi] : g.w;
+    void *o = gi ? g.out_g[gi] : g.out;
+    if (!a || !w || !o || !aligned16(a) || !aligned16(w) || !aligned16(o)) return DPARA_ERR_INVALID_ARG;
+    if (!make_tmap_bf16_2d(&P.map_a[gi], a, g.K, g.M, (uint64_t)g.K * 2, kBK, kBM)) return DPARA_ERR_CUDA;
+    if (!make_tmap_bf16_2d(&P.map_b[gi], w, g.K, w_rows, (uint64_t)g.K * 2, kBK, 128)) return DPARA_ERR_CUDA;
+    P.out_g[gi] = o;
+  }
   P.M = g.M; P.N = g.N; P.K = g.K; P.epi = g.epi; P.up_row_offset = g.N;
   P.out = g.out; P.resid = g.resid; P.resid_bf16 = g.resid_bf16; P.out_bf16 = g.out_bf16; P.status = status;
   P.perm_block = g.epi == 3 ? g.perm_block : 0; P.perm_b = g.perm_b;
+  P.split_k = 1;
+  if (g.split_k > 1) {
+    if (g.epi != 3 || g.M <= kBM || g.split_k > g.K / kBK) return DPARA_ERR_UNSUPPORTED;
+    P.split_k = g.split_k;
+  }
   if (cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess) return DPARA_ERR_CUDA;
   const int tile_cols = g.epi == 2 ? 128 : kBN;
   const int tiles = ((g.N + tile_cols - 1) / tile_cols) * ((g.M + kBM - 1) / kBM);
@@ -393,7 +417,7 @@ dpara_status launch_gemm_tc(const GemmArgs &g, int32_t *status, cudaStream_t st)
   if (g.M > kBM) {
     // more than one 128-row tile of activations: CTA pairs (one 256 x 256 tile per pair and round)
     if (cudaFuncSetAttribute(gemm_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes2) != cudaSuccess) return DPARA_ERR_CUDA;
-    const int pair_tiles = ((g.N + tile_cols - 1) / tile_cols) * ((g.M + 2 * kBM - 1) / (2 * kBM));
+    const int pair_tiles = ((g.N + tile_cols - 1) / tile_cols) * ((g.M + 2 * kBM - 1) / (2 * kBM)) * P.split_k * P.n_groups;
     const int pairs = pair_tiles < sms / 2 ? pair_tiles : sms / 2;
     gemm_tc2_kernel<<<2 * pairs, kThreads, kSmemBytes2, st>>>(P);
     DPARA_CHECK_LAUNCH();

@@ -69,6 +69,8 @@ def _check(ci, use_rope=True, knorm=True, capacity=None):
     ((37, 0, 5, 130), 4, 256, 2, 64, 2),
     ((300, 12, 77), 8, 512, 8, 128, 3),
     ((64,) * 20, 16, 320, 4, 128, 1),          # 320 candidate rows: several GEMM row tiles
+    ((50, 9, 31) * 6, 9, 512, 4, 128, 10),     # 162 rows x 10 layers: two grouped launches (8 + 2 layers), K ranges in parts
+    ((40,) * 33, 8, 1024, 2, 64, 3),           # 264 rows: two row pairs per layer, three layers in one launch
 ])
 def test_append_parity(lens, J, F, Hkv, D, layers):
     ci = W.make_cache_inputs(lens, J, F, Hkv, D, layers, 21)
