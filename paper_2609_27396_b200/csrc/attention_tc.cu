@@ -332,6 +332,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
   const int q_begin = P.use_seg ? (team < P.seg_teams ? (int)P.team_first[team] : 0) : (P.use_sched ? (int)P.cta_first[blockIdx.x] : (int)blockIdx.x);
   const int q_end = P.use_seg ? (team < P.seg_teams ? (int)P.team_first[team + 1] : 0) : (P.use_sched ? (int)P.cta_first[blockIdx.x + 1] : P.n_items);
   const int q_step = (P.use_seg || P.use_sched) ? 1 : (int)gridDim.x;
+  pdl_launch_dependents();
+  pdl_wait();  // nothing above touches global memory
   // (a CTA of a cluster must not leave early: its peers meet it at the cluster barriers below)
   if (P.nsplit == 1 && A.status_word && (*reinterpret_cast<volatile int32_t *>(A.status_word) & (int32_t)DPARA_STATUS_TIMEOUT)) return;
 
@@ -896,19 +898,22 @@ static dpara_status launch_tc_d(const TcParams &P, const TcPlan &plan, cudaStrea
   int dev = 0, sms = kNumSM;
   if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   cudaLaunchConfig_t cfg = {};
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   cfg.blockDim = dim3(kThreads);
   cfg.dynamicSmemBytes = Cfg::kSmemBytes;
   cfg.stream = st;
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
   if (P.nsplit > 1) {
     // one CTA per (item, split); the splits of an item are consecutive CTAs = one cluster
     cfg.gridDim = dim3(P.n_items);
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = P.nsplit;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = P.nsplit;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
+    cfg.numAttrs = 2;
   } else {
     cfg.gridDim = dim3(P.use_seg || P.n_items >= sms ? sms : P.n_items);  // persistent: at most one CTA per SM
   }

@@ -37,6 +37,8 @@ struct AppendParams {
 __global__ void __launch_bounds__(128) append_rows_kernel(const AppendParams P) {
   extern __shared__ float s_cs[];  // cos[D/2], sin[D/2]
   const int n = blockIdx.x / P.J, i = blockIdx.x % P.J, tid = threadIdx.x, g = blockIdx.y;
+  pdl_launch_dependents();
+  pdl_wait();
   const uint16_t *knorm_w = P.knorm_w[g];
   const float *kv_parts = P.kv_parts + (size_t)g * P.n_parts * P.part_stride;
   const int r = P.accept_len[n];
@@ -118,6 +120,8 @@ __global__ void __launch_bounds__(128) append_rows_kernel(const AppendParams P) 
 
 // After every layer has read the old lengths: L_n += r_n + 1 for the requests that fitted.
 __global__ void append_commit_kernel(int64_t *ctx_len, const int64_t *capacity, const int32_t *accept_len, int b, int J) {
+  pdl_launch_dependents();
+  pdl_wait();
   for (int n = blockIdx.x * blockDim.x + threadIdx.x; n < b; n += gridDim.x * blockDim.x) {
     const int r = accept_len[n];
     const long long L = ctx_len[n];
@@ -213,12 +217,12 @@ dpara_status launch_cache_append(const dpara_cache_io *io, void *workspace, int3
     if (s != DPARA_OK) return s;
     P.kv = kv;
     P.kv_parts = reinterpret_cast<const float *>(kv); P.n_parts = parts;
-    append_rows_kernel<<<dim3(M, group), 128, io->head_dim * sizeof(float), st>>>(P);
+    launch_pdl(append_rows_kernel, dim3(M, group), dim3(128), io->head_dim * sizeof(float), st, P);
     DPARA_CHECK_LAUNCH();
     count_launches(1);
     l0 += group;
   }
-  append_commit_kernel<<<(io->batch + 127) / 128, 128, 0, st>>>(io->ctx_len, io->capacity, io->accept_len, io->batch, io->n_rows);
+  launch_pdl(append_commit_kernel, dim3((io->batch + 127) / 128), dim3(128), 0, st, io->ctx_len, io->capacity, io->accept_len, io->batch, io->n_rows);
   DPARA_CHECK_LAUNCH();
   count_launches(1);
   return DPARA_OK;

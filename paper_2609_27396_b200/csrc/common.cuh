@@ -31,6 +31,29 @@ inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 
     if (e_ != cudaSuccess) return DPARA_ERR_CUDA;              \
   } while (0)
 
+// Programmatic dependent launch.  Every kernel of this library starts with pdl_launch_dependents() (the next kernel on the
+// stream may be set up and its CTAs made resident as SMs free up) followed by pdl_wait() (blocks until the kernels before it
+// have completed and their writes are visible) BEFORE it reads or writes any global memory; launched through launch_pdl
+// the kernel's launch latency and prologue then overlap the tail of its predecessor.  Without the launch attribute both
+// instructions do nothing.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args &&...args) {
+  cudaLaunchConfig_t cfg = {};
+  cudaLaunchAttribute attr[1];
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // Process-wide count of kernels this library has launched (evidence for benchmarks; relaxed atomic).
 void count_launches(int n);
 

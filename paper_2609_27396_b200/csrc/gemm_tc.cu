@@ -147,6 +147,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
     *abort_flag = 0;
     fence_barrier_init();
   }
+  pdl_launch_dependents();
   if (warp == 5) {
     tmem_alloc(tmem_slot, 512);
     tmem_relinquish();
@@ -155,6 +156,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
+  pdl_wait();  // nothing above touches global memory: the set-up overlaps the tail of the kernel before
 
   // Persistent: CTA c computes tiles c, c + gridDim.x, ...; tile id = n_tile * m_tiles + m_tile, so the CTAs
   // running together cover all M rows of a few weight tiles (A stays in L2, each weight tile is read once).
@@ -285,6 +287,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1) gemm_tc
     *abort_flag = 0;
     fence_barrier_init();
   }
+  pdl_launch_dependents();
   if (warp == 5) {
     tmem_alloc_pair(tmem_slot, 512);
     tmem_relinquish_pair();
@@ -294,6 +297,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1) gemm_tc
   cluster_sync_all();  // both CTAs' barriers exist before anything signals across the pair
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
+  pdl_wait();  // nothing above touches global memory: the set-up overlaps the tail of the kernel before
 
   if (warp == 4) {
     if (lane == 0) {
@@ -419,12 +423,12 @@ dpara_status launch_gemm_tc(const GemmArgs &g, int32_t *status, cudaStream_t st)
     if (cudaFuncSetAttribute(gemm_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes2) != cudaSuccess) return DPARA_ERR_CUDA;
     const int pair_tiles = ((g.N + tile_cols - 1) / tile_cols) * ((g.M + 2 * kBM - 1) / (2 * kBM)) * P.split_k * P.n_groups;
     const int pairs = pair_tiles < sms / 2 ? pair_tiles : sms / 2;
-    gemm_tc2_kernel<<<2 * pairs, kThreads, kSmemBytes2, st>>>(P);
+    launch_pdl(gemm_tc2_kernel, dim3(2 * pairs), dim3(kThreads), kSmemBytes2, st, P);
     DPARA_CHECK_LAUNCH();
     count_launches(1);
     return DPARA_OK;
   }
-  gemm_tc_kernel<<<tiles < sms ? tiles : sms, kThreads, kSmemBytes, st>>>(P);
+  launch_pdl(gemm_tc_kernel, dim3(tiles < sms ? tiles : sms), dim3(kThreads), kSmemBytes, st, P);
   DPARA_CHECK_LAUNCH();
   count_launches(1);
   return DPARA_OK;

@@ -20,6 +20,8 @@ template <bool kF32In>
 __global__ void __launch_bounds__(128) rmsnorm_kernel(const void *__restrict__ x, const uint16_t *__restrict__ gain,
                                                       uint16_t *__restrict__ out, int H, float eps) {
   const int row = blockIdx.x, tid = threadIdx.x;
+  pdl_launch_dependents();
+  pdl_wait();
   float ss = 0.f;
   for (int c = tid * 8; c < H; c += 128 * 8) {
     float v[8];
@@ -91,6 +93,8 @@ __global__ void __launch_bounds__(128) qk_norm_rope_kernel(const QkParams P) {
   const int row = blockIdx.x, tid = threadIdx.x;
   const int half = P.D / 2;
   const int R = P.Bq * P.J + P.Sq;
+  pdl_launch_dependents();
+  pdl_wait();
   const int n = row / R, rr = row % R;
   if (P.use_rope) {
     const int rel = rr < P.Bq * P.J ? rr / P.Bq + 2 + rr % P.Bq : rr - P.Bq * P.J;  // mask slot (j, i): j + 2 + i; spine row s: s
@@ -184,7 +188,7 @@ void layer_workspace_offsets(const dpara_shape *shape, const dpara_layer_io *lay
 
 dpara_status launch_rmsnorm_bf16(const void *x, const void *gain, void *out, int M, int H, float eps, cudaStream_t st) {
   if (H % 8) return DPARA_ERR_UNSUPPORTED;
-  rmsnorm_kernel<false><<<M, 128, 0, st>>>(x, static_cast<const uint16_t *>(gain), static_cast<uint16_t *>(out), H, eps);
+  launch_pdl(rmsnorm_kernel<false>, dim3(M), dim3(128), 0, st, x, static_cast<const uint16_t *>(gain), static_cast<uint16_t *>(out), H, eps);
   DPARA_CHECK_LAUNCH();
   count_launches(1);
   return DPARA_OK;
@@ -217,7 +221,7 @@ dpara_status launch_layer(const dpara_shape *shape, const dpara_attn_io *io, con
   uint16_t *a = reinterpret_cast<uint16_t *>(lw + w.a), *hn = reinterpret_cast<uint16_t *>(lw + w.hn), *act = reinterpret_cast<uint16_t *>(lw + w.act);
   float *h1 = reinterpret_cast<float *>(lw + w.h1);
 
-  rmsnorm_kernel<false><<<M, 128, 0, st>>>(L->x, static_cast<const uint16_t *>(L->rms1_w), xn, H, L->rms_eps);
+  launch_pdl(rmsnorm_kernel<false>, dim3(M), dim3(128), 0, st, L->x, static_cast<const uint16_t *>(L->rms1_w), xn, H, L->rms_eps);
   DPARA_CHECK_LAUNCH();
   count_launches(1);
   GemmArgs g{};
@@ -230,7 +234,7 @@ dpara_status launch_layer(const dpara_shape *shape, const dpara_attn_io *io, con
   qp.q = q; qp.k = k; qp.v = v; qp.ctx_offsets = io->ctx_offsets; qp.ctx_lens = io->ctx_lens;
   qp.J = shape->n_boundaries; qp.Bq = shape->block; qp.Hq = shape->n_q_heads; qp.Hkv = shape->n_kv_heads; qp.D = D; qp.Sq = Sq;
   qp.use_rope = L->use_rope; qp.use_norm = L->qnorm_w != nullptr; qp.eps = L->rms_eps; qp.theta = L->rope_theta;
-  qk_norm_rope_kernel<<<M, 128, D * sizeof(float), st>>>(qp);
+  launch_pdl(qk_norm_rope_kernel, dim3(M), dim3(128), D * sizeof(float), st, qp);
   DPARA_CHECK_LAUNCH();
   count_launches(1);
 
@@ -248,7 +252,7 @@ dpara_status launch_layer(const dpara_shape *shape, const dpara_attn_io *io, con
   g.a = a; g.w = L->w_o; g.M = M; g.N = H; g.K = QD; g.epi = 1; g.resid = L->x; g.resid_bf16 = 1; g.out = h1;
   s = launch_gemm_tc(g, status_word, st);
   if (s != DPARA_OK) return s;
-  rmsnorm_kernel<true><<<M, 128, 0, st>>>(h1, static_cast<const uint16_t *>(L->rms2_w), hn, H, L->rms_eps);
+  launch_pdl(rmsnorm_kernel<true>, dim3(M), dim3(128), 0, st, static_cast<const void *>(h1), static_cast<const uint16_t *>(L->rms2_w), hn, H, L->rms_eps);
   DPARA_CHECK_LAUNCH();
   count_launches(1);
   g = GemmArgs{};

@@ -97,6 +97,8 @@ template <int kGreedyLoads>
 __global__ void __launch_bounds__(kVsThreads, kGreedyLoads >= 16 ? 3 : (kGreedyLoads >= 8 ? 4 : 6)) verify_greedy_kernel(const VerifyParams P) {
   constexpr int kGreedyChunk = kGreedyLoads * 1024;  // floats per CTA
   const int tid = threadIdx.x;
+  pdl_launch_dependents();
+  pdl_wait();
   // rows are handed out position-major (every request's row 0 first, then every row 1, ...): the early rows,
   // which decide the accepted length, finish early for ALL requests
   const int n = blockIdx.y % P.b;
@@ -259,6 +261,8 @@ __device__ __forceinline__ void weights_of(float p, float q, bool residual, unsi
 
 __global__ void __launch_bounds__(kVsThreads) verify_sampling_kernel(const VerifyParams P) {
   const int tid = threadIdx.x;
+  pdl_launch_dependents();
+  pdl_wait();
   const int n = blockIdx.y;
   const int c = blockIdx.x;
   const int g = P.J - 1;
@@ -529,16 +533,19 @@ dpara_status launch_verify(const dpara_verify_io *io, void *ws, int32_t *status_
   // keys, masks and counters are zero on entry (the previous call put them back); nothing is cleared here
   if (io->mode == 0) {
     dim3 grid(P.nchunks, io->batch * io->n_boundaries);
+    // The 16-load form is chosen when the grid is several waves deep (b = 16: 2560 CTAs): launched early behind a long
+    // kernel it measured 5 us SLOWER than a plain launch, so only the small-grid forms ask for the early launch
+    // (b = 1: 152 CTAs, 3 us faster).
     switch (greedy_loads_of(io)) {
       case 16: verify_greedy_kernel<16><<<grid, kVsThreads, 0, st>>>(P); break;
-      case 8: verify_greedy_kernel<8><<<grid, kVsThreads, 0, st>>>(P); break;
-      case 4: verify_greedy_kernel<4><<<grid, kVsThreads, 0, st>>>(P); break;
-      case 2: verify_greedy_kernel<2><<<grid, kVsThreads, 0, st>>>(P); break;
-      default: verify_greedy_kernel<1><<<grid, kVsThreads, 0, st>>>(P); break;
+      case 8: launch_pdl(verify_greedy_kernel<8>, dim3(grid), dim3(kVsThreads), 0, st, P); break;
+      case 4: launch_pdl(verify_greedy_kernel<4>, dim3(grid), dim3(kVsThreads), 0, st, P); break;
+      case 2: launch_pdl(verify_greedy_kernel<2>, dim3(grid), dim3(kVsThreads), 0, st, P); break;
+      default: launch_pdl(verify_greedy_kernel<1>, dim3(grid), dim3(kVsThreads), 0, st, P); break;
     }
   } else {
     dim3 grid(P.nchunks, io->batch);
-    verify_sampling_kernel<<<grid, kVsThreads, 0, st>>>(P);
+    launch_pdl(verify_sampling_kernel, dim3(grid), dim3(kVsThreads), 0, st, P);
   }
   DPARA_CHECK_LAUNCH();
   count_launches(1);
