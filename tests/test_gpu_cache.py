@@ -71,6 +71,7 @@ def _check(ci, use_rope=True, knorm=True, capacity=None):
     ((64,) * 20, 16, 320, 4, 128, 1),          # 320 candidate rows: several GEMM row tiles
     ((50, 9, 31) * 6, 9, 512, 4, 128, 10),     # 162 rows x 10 layers: two grouped launches (8 + 2 layers), K ranges in parts
     ((40,) * 33, 8, 1024, 2, 64, 3),           # 264 rows: two row pairs per layer, three layers in one launch
+    ((100, 37, 64, 12) * 4, 16, 5120, 8, 128, 5),   # the benchmark's shape: 256 candidate rows x 5120 features, 5 layers in one grouped launch
 ])
 def test_append_parity(lens, J, F, Hkv, D, layers):
     ci = W.make_cache_inputs(lens, J, F, Hkv, D, layers, 21)
