@@ -707,7 +707,7 @@ def oracle_threads() -> int:
 
 # ----------------------------------------------------------------------------- single targets for a profiler
 ONLY_TARGETS = {"colocation", "attention_cfg2", "attention_cfg3", "attention_cfg5", "verify_cfg2", "verify_cfg3", "verify_cfg4", "layer_cfg5", "gemm_qkv", "gemm_o",
-                "gemm_gate_up", "gemm_down", "head", "cache_append", "backbone_cfg5"}
+                "gemm_gate_up", "gemm_down", "head", "head_sampling", "cache_append", "backbone_cfg5"}
 
 
 def run_only(target: str, reps: int):
@@ -741,6 +741,10 @@ def run_only(target: str, reps: int):
         w = W.workload(3)
         r = HeadRunner(w, w.seed)
         fn = r.step
+    elif target == "head_sampling":
+        w = W.workload(3)
+        r = HeadRunner(w, w.seed)
+        fn = lambda: r.step(sampling=True)
     elif target == "cache_append":
         cache_append_leg(W.workload(3), peaks, reps)
         return
