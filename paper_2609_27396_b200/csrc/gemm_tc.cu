@@ -40,6 +40,7 @@ struct GemmKernelParams {
   void *out_bf16;
   int32_t *status;
   int perm_block, perm_b;
+  int bn;        // output columns per tile of the CTA-pair kernel: 256, or 192 where that fills the rounds better (bf16 / fp32 stores)
   int split_k;   // > 1 (fp32 store only, CTA pairs): the K range in split_k parts, part s writes plane s of [split_k][M][N] partial sums
 };
 
@@ -56,8 +57,8 @@ __device__ __forceinline__ void gemm_epilogue(const GemmKernelParams &P, uint32_
                                               int grp) {
   // fp32 output of this product; split K (fp32 store only): plane ks of the partial sums
   float *out_f32 = static_cast<float *>(P.n_groups > 1 ? P.out_g[grp] : P.out) + (size_t)ks * P.M * P.N;
-  const int n_chunks = P.epi == 2 ? 4 : kBN / 32;
-  const int col0 = n_tile * (P.epi == 2 ? 128 : kBN);
+  const int n_chunks = P.epi == 2 ? 4 : P.bn / 32;
+  const int col0 = n_tile * (P.epi == 2 ? 128 : P.bn);
   const int sub_row = lane >> 3, piece = lane & 7;
 #pragma unroll 1
   for (int c = 0; c < n_chunks; ++c) {
@@ -270,7 +271,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1) gemm_tc
   const uint32_t rank = cluster_ctarank();
   const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
   const int nkb = P.K / kBK;
-  const int tile_cols = P.epi == 2 ? 128 : kBN;
+  const int tile_cols = P.epi == 2 ? 128 : P.bn;
   const int m_pairs = (P.M + 2 * kBM - 1) / (2 * kBM), n_tiles = (P.N + tile_cols - 1) / tile_cols;
   const int group_units = m_pairs * n_tiles * P.split_k;   // work units of one product: (tile, K part), the parts of a tile adjacent
   const int total_tiles = group_units * P.n_groups;
@@ -314,13 +315,15 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1) gemm_tc
         const int m_pair = tile % m_pairs, n_tile = tile / m_pairs;
         const int kb0 = ks * nkb / P.split_k, kb1 = (ks + 1) * nkb / P.split_k;
         // this CTA's half of the weight tile: rows [rank * 128, +128) of the tile (SwiGLU: gate rows / up rows)
-        const int brow = P.epi == 2 ? (rank == 0 ? n_tile * 128 : P.up_row_offset + n_tile * 128) : n_tile * kBN + (int)rank * 128;
+        const int half = P.epi == 2 ? 128 : P.bn / 2;   // weight rows each CTA of the pair holds
+        const int brow = P.epi == 2 ? (rank == 0 ? n_tile * 128 : P.up_row_offset + n_tile * 128) : n_tile * P.bn + (int)rank * half;
+        const uint32_t tx = 2u * ((uint32_t)kABytes + (uint32_t)half * kBK * 2u);
         const int arow = (m_pair * 2 + (int)rank) * kBM;
         for (int kb = kb0; kb < kb1; ++kb) {
           ok = mbar_wait(empty + stage, ph ^ 1u, abort_flag, 2);
           if (!ok) break;
           uint8_t *sa = smem + stage * kStageBytes2;
-          if (rank == 0) mbar_arrive_expect_tx(full + stage, 2u * kStageBytes2);
+          if (rank == 0) mbar_arrive_expect_tx(full + stage, tx);
           tma_load_2d_pair(sa, &P.map_a[grp], full + stage, kb * kBK, arow);
           tma_load_2d_pair(sa + kABytes, &P.map_b[grp], full + stage, kb * kBK, brow);
           if (++stage == kStages2) { stage = 0; ph ^= 1u; }
@@ -329,7 +332,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1) gemm_tc
     }
   } else if (warp == 5) {
     if (rank == 0 && lane == 0) {
-      constexpr uint32_t idesc = idesc_bf16_f32(2 * kBM, kBN, false, false);
+      const uint32_t idesc = idesc_bf16_f32(2 * kBM, P.epi == 2 ? kBN : P.bn, false, false);
       const uint64_t adesc0 = smem_desc_sw128(smem_u32(smem), 16, 1024);
       const uint64_t bdesc0 = smem_desc_sw128(smem_u32(smem) + kABytes, 16, 1024);
       int stage = 0, k = 0;
@@ -391,6 +394,19 @@ dpara_status launch_gemm_tc(const GemmArgs &g, int32_t *status, cudaStream_t st)
   if (!aligned16(g.a) || !aligned16(g.w) || !aligned16(g.out) || !aligned16(g.resid) || !aligned16(g.out_bf16)) return DPARA_ERR_INVALID_ARG;
   GemmKernelParams P;
   const int w_rows = g.epi == 2 ? 2 * g.N : g.N;
+  int dev = 0, sms = kNumSM;
+  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int split = g.split_k > 1 ? g.split_k : 1, groups = g.n_groups > 1 ? g.n_groups : 1;
+  // Tile width of the pair kernel: 192 columns when that evens out the rounds (QKV at 1024 x 6144: 96 tiles of 256 are two
+  // rounds of the 74 pairs, the second a third full; 128 tiles of 192 are two rounds of 0.75 the length).  A 192-wide tile
+  // pulls 28 KB per CTA and K slab for 0.75 of the flops of a 256-wide one: its rounds are weighted 1.14x.
+  P.bn = kBN;
+  if (g.M > kBM && g.epi != 2) {
+    const long m_pairs = (g.M + 2 * kBM - 1) / (2 * kBM), pairs = sms / 2 > 0 ? sms / 2 : 1;
+    const long u256 = m_pairs * ((g.N + 255) / 256) * split * groups, u192 = m_pairs * ((g.N + 191) / 192) * split * groups;
+    const double c256 = (double)((u256 + pairs - 1) / pairs) * 256.0, c192 = (double)((u192 + pairs - 1) / pairs) * 192.0 * 1.14;
+    if (c192 < 0.95 * c256) P.bn = 192;
+  }
   P.n_groups = 1;
   if (g.n_groups > 1) {
     // several products of one shape in one launch (fp32 stores, CTA pairs): entry 0 of the lists is (a, w, out)
@@ -402,7 +418,7 @@ dpara_status launch_gemm_tc(const GemmArgs &g, int32_t *status, cudaStream_t st)
     void *o = gi ? g.out_g[gi] : g.out;
     if (!a || !w || !o || !aligned16(a) || !aligned16(w) || !aligned16(o)) return DPARA_ERR_INVALID_ARG;
     if (!make_tmap_bf16_2d(&P.map_a[gi], a, g.K, g.M, (uint64_t)g.K * 2, kBK, kBM)) return DPARA_ERR_CUDA;
-    if (!make_tmap_bf16_2d(&P.map_b[gi], w, g.K, w_rows, (uint64_t)g.K * 2, kBK, 128)) return DPARA_ERR_CUDA;
+    if (!make_tmap_bf16_2d(&P.map_b[gi], w, g.K, w_rows, (uint64_t)g.K * 2, kBK, P.bn == kBN ? 128 : P.bn / 2)) return DPARA_ERR_CUDA;
     P.out_g[gi] = o;
   }
   P.M = g.M; P.N = g.N; P.K = g.K; P.epi = g.epi; P.up_row_offset = g.N;
@@ -414,10 +430,8 @@ dpara_status launch_gemm_tc(const GemmArgs &g, int32_t *status, cudaStream_t st)
     P.split_k = g.split_k;
   }
   if (cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess) return DPARA_ERR_CUDA;
-  const int tile_cols = g.epi == 2 ? 128 : kBN;
+  const int tile_cols = g.epi == 2 ? 128 : P.bn;
   const int tiles = ((g.N + tile_cols - 1) / tile_cols) * ((g.M + kBM - 1) / kBM);
-  int dev = 0, sms = kNumSM;
-  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   if (g.M > kBM) {
     // more than one 128-row tile of activations: CTA pairs (one 256 x 256 tile per pair and round)
     if (cudaFuncSetAttribute(gemm_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes2) != cudaSuccess) return DPARA_ERR_CUDA;
