@@ -862,10 +862,11 @@ TcPlan plan_attention_tc(const dpara_shape *s, const int64_t *host_off, const in
   // A small batch is latency-bound: when one-tile items with their splits still fit the GPU in a single wave, an item is
   // ONE query tile instead of two -- twice the CTAs, each with half the Q load, half the partial rows and half the merge
   int split_cap = 8;  // largest cluster size whose clusters all run at once
+  long long items1 = 0;
   {
     const int pairs2 = p.n_pairs;
     lay_out_items(1);
-    const long long items1 = (long long)s->batch * s->n_kv_heads * p.n_pairs;
+    items1 = (long long)s->batch * s->n_kv_heads * p.n_pairs;
     int split1 = 0;
     for (int c = 8; c >= 2 && !split1; c >>= 1)
       if (c <= max_tiles && items1 <= max_active_clusters(s->head_dim, c)) split1 = c;
@@ -882,7 +883,9 @@ TcPlan plan_attention_tc(const dpara_shape *s, const int64_t *host_off, const in
   p.nsplit = nsplit;
   p.items = items;
   p.workspace_bytes = nsplit > 1 ? (size_t)items * nsplit * 256 * ((size_t)s->head_dim + 2) * 4 : 0;
-  p.workspace_max_bytes = items < 96 ? (size_t)items * 8 * 256 * ((size_t)s->head_dim + 2) * 4 : 0;
+  // (sized for the one-tile layout, the larger of the two: which layout is taken depends on how many clusters the device
+  //  runs at once, and the size must not)
+  p.workspace_max_bytes = items < 96 ? (size_t)std::max(items, items1) * 8 * 256 * ((size_t)s->head_dim + 2) * 4 : 0;
   // the cut schedule (items >= 96): at most two pieces per team and member plus seven per group of a degenerate cut,
   // bounded here by 2 * SMs piece slots; plus one ticket per item
   if (items >= 96 && p.n_pairs <= 16)

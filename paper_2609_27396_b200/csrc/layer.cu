@@ -110,41 +110,59 @@ __global__ void __launch_bounds__(128) qk_norm_rope_kernel(const QkParams P) {
   __syncthreads();
   const int warp = tid >> 5, lane = tid & 31;
   const size_t qkv_row = (size_t)row * (P.Hq + 2 * P.Hkv) * P.D;
-  const int E = P.D / 64;  // pairs (d, d + D/2) per lane: D = 64 -> 1, D = 128 -> 2
-  for (int hd = warp; hd < P.Hq + P.Hkv; hd += 4) {
-    const bool is_q = hd < P.Hq;
-    const uint16_t *src = P.qkv + qkv_row + (size_t)hd * P.D;
-    uint16_t *dst = is_q ? P.q + ((size_t)row * P.Hq + hd) * P.D : P.k + ((size_t)row * P.Hkv + (hd - P.Hq)) * P.D;
-    const uint16_t *gain = is_q ? P.qnorm_w : P.knorm_w;
-    float x1[2], x2[2];
-    float ss = 0.f;
-    for (int e = 0; e < E; ++e) {
-      const int d = lane + 32 * e;
-      x1[e] = bf16_bits_to_float(src[d]);
-      x2[e] = bf16_bits_to_float(src[d + half]);
-      ss += x1[e] * x1[e] + x2[e] * x2[e];
-    }
-    if (P.use_norm) {
+  // A lane owns the element pairs (2 lane, 2 lane + 1) of both halves of a head (one 4-byte load each); a warp takes heads
+  // warp, warp + 4, ... and fetches kChunk of them before it works on the first, so that a row costs a few global round
+  // trips instead of one per head.
+  constexpr int kChunk = 6;
+  const bool active = 2 * lane < half;
+  const int n_heads = P.Hq + P.Hkv;
+  for (int hd0 = warp; hd0 < n_heads; hd0 += 4 * kChunk) {
+    uint32_t lo[kChunk], hi[kChunk];
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-      const float rs = rsqrtf(ss / (float)P.D + P.eps);
-      for (int e = 0; e < E; ++e) {
-        const int d = lane + 32 * e;
-        const float g1 = gain ? bf16_bits_to_float(gain[d]) : 1.f, g2 = gain ? bf16_bits_to_float(gain[d + half]) : 1.f;
-        x1[e] = __bfloat162float(__float2bfloat16_rn(x1[e] * rs * g1));
-        x2[e] = __bfloat162float(__float2bfloat16_rn(x2[e] * rs * g2));
+    for (int c = 0; c < kChunk; ++c) {
+      const int hd = hd0 + 4 * c;
+      lo[c] = hi[c] = 0u;
+      if (hd < n_heads && active) {
+        const uint16_t *src = P.qkv + qkv_row + (size_t)hd * P.D;
+        lo[c] = *reinterpret_cast<const uint32_t *>(src + 2 * lane);
+        hi[c] = *reinterpret_cast<const uint32_t *>(src + half + 2 * lane);
       }
     }
-    for (int e = 0; e < E; ++e) {
-      const int d = lane + 32 * e;
-      float y1 = x1[e], y2 = x2[e];
-      if (P.use_rope) {
-        const float cs = s_cs[d], sn = s_cs[half + d];
-        y1 = x1[e] * cs - x2[e] * sn;
-        y2 = x2[e] * cs + x1[e] * sn;
+#pragma unroll
+    for (int c = 0; c < kChunk; ++c) {
+      const int hd = hd0 + 4 * c;
+      if (hd >= n_heads) break;
+      const bool is_q = hd < P.Hq;
+      uint16_t *dst = is_q ? P.q + ((size_t)row * P.Hq + hd) * P.D : P.k + ((size_t)row * P.Hkv + (hd - P.Hq)) * P.D;
+      const uint16_t *gain = is_q ? P.qnorm_w : P.knorm_w;
+      float x1[2] = {bf16lo(lo[c]), bf16hi(lo[c])}, x2[2] = {bf16lo(hi[c]), bf16hi(hi[c])};
+      if (P.use_norm) {
+        float ss = x1[0] * x1[0] + x2[0] * x2[0] + x1[1] * x1[1] + x2[1] * x2[1];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+        const float rs = rsqrtf(ss / (float)P.D + P.eps);
+        if (active) {
+          const uint32_t g1 = gain ? *reinterpret_cast<const uint32_t *>(gain + 2 * lane) : 0x3f803f80u;          // bf16 1.0 twice
+          const uint32_t g2 = gain ? *reinterpret_cast<const uint32_t *>(gain + half + 2 * lane) : 0x3f803f80u;
+          x1[0] = __bfloat162float(__float2bfloat16_rn(x1[0] * rs * bf16lo(g1)));
+          x1[1] = __bfloat162float(__float2bfloat16_rn(x1[1] * rs * bf16hi(g1)));
+          x2[0] = __bfloat162float(__float2bfloat16_rn(x2[0] * rs * bf16lo(g2)));
+          x2[1] = __bfloat162float(__float2bfloat16_rn(x2[1] * rs * bf16hi(g2)));
+        }
       }
-      dst[d] = __bfloat16_as_ushort(__float2bfloat16_rn(y1));
-      dst[d + half] = __bfloat16_as_ushort(__float2bfloat16_rn(y2));
+      if (active) {
+        float y1[2] = {x1[0], x1[1]}, y2[2] = {x2[0], x2[1]};
+        if (P.use_rope) {
+#pragma unroll
+          for (int e = 0; e < 2; ++e) {
+            const float cs = s_cs[2 * lane + e], sn = s_cs[half + 2 * lane + e];
+            y1[e] = x1[e] * cs - x2[e] * sn;
+            y2[e] = x2[e] * cs + x1[e] * sn;
+          }
+        }
+        *reinterpret_cast<uint32_t *>(dst + 2 * lane) = pack_bf16(y1[0], y1[1]);
+        *reinterpret_cast<uint32_t *>(dst + half + 2 * lane) = pack_bf16(y2[0], y2[1]);
+      }
     }
   }
   // v: plain copy into its own contiguous tensor
