@@ -31,6 +31,7 @@ struct AppendParams {
   int32_t *status_word;
   int J, Hkv, D, use_rope;
   float eps, theta;
+  double inv_freq[64];      // theta^(-2 d / D), d < D / 2, worked out on the host in double precision
 };
 
 // One CTA per (candidate row (request n, draft position i), layer of the launch); rows above the accepted length leave at once.
@@ -53,7 +54,7 @@ __global__ void __launch_bounds__(128) append_rows_kernel(const AppendParams P) 
     const double pos = (double)(L + i);
     for (int d = tid; d < half; d += 128) {
       double sn, cs;
-      sincos(pos * pow((double)P.theta, -2.0 * d / P.D), &sn, &cs);
+      sincos(pos * P.inv_freq[d], &sn, &cs);
       s_cs[d] = (float)cs;
       s_cs[half + d] = (float)sn;
     }
@@ -189,6 +190,7 @@ dpara_status launch_cache_append(const dpara_cache_io *io, void *workspace, int3
   P.status_word = status_word;
   P.J = io->n_rows; P.Hkv = io->n_kv_heads; P.D = io->head_dim; P.use_rope = io->use_rope;
   P.eps = io->rms_eps; P.theta = io->rope_theta;
+  for (int d = 0; d < io->head_dim / 2 && d < 64; ++d) P.inv_freq[d] = pow((double)io->rope_theta, -2.0 * d / io->head_dim);
   P.part_stride = (size_t)M * N;
   const void *prev_gain = nullptr;
   int slot = -1;

@@ -86,6 +86,7 @@ struct QkParams {
   int J, Bq, Hq, Hkv, D, Sq;
   int use_rope, use_norm;
   float eps, theta;
+  double inv_freq[64];   // theta^(-2 d / D), d < D / 2, worked out on the host in double precision
 };
 
 __global__ void __launch_bounds__(128) qk_norm_rope_kernel(const QkParams P) {
@@ -100,9 +101,8 @@ __global__ void __launch_bounds__(128) qk_norm_rope_kernel(const QkParams P) {
     const int rel = rr < P.Bq * P.J ? rr / P.Bq + 2 + rr % P.Bq : rr - P.Bq * P.J;  // mask slot (j, i): j + 2 + i; spine row s: s
     const double pos = (double)(P.ctx_lens ? P.ctx_lens[n] : P.ctx_offsets[n + 1] - P.ctx_offsets[n]) + rel;
     for (int d = tid; d < half; d += 128) {
-      const double inv = pow((double)P.theta, -2.0 * d / P.D);
       double sn, cs;
-      sincos(pos * inv, &sn, &cs);
+      sincos(pos * P.inv_freq[d], &sn, &cs);
       s_cs[d] = (float)cs;
       s_cs[half + d] = (float)sn;
     }
@@ -252,6 +252,7 @@ dpara_status launch_layer(const dpara_shape *shape, const dpara_attn_io *io, con
   qp.q = q; qp.k = k; qp.v = v; qp.ctx_offsets = io->ctx_offsets; qp.ctx_lens = io->ctx_lens;
   qp.J = shape->n_boundaries; qp.Bq = shape->block; qp.Hq = shape->n_q_heads; qp.Hkv = shape->n_kv_heads; qp.D = D; qp.Sq = Sq;
   qp.use_rope = L->use_rope; qp.use_norm = L->qnorm_w != nullptr; qp.eps = L->rms_eps; qp.theta = L->rope_theta;
+  for (int d = 0; d < D / 2 && d < 64; ++d) qp.inv_freq[d] = pow((double)L->rope_theta, -2.0 * d / D);
   launch_pdl(qk_norm_rope_kernel, dim3(M), dim3(128), D * sizeof(float), st, qp);
   DPARA_CHECK_LAUNCH();
   count_launches(1);
