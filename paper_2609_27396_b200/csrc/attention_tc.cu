@@ -58,10 +58,12 @@ struct TcParams {
   // 128 >> hb_log2[k] (j, i) rows; its tile pairs are pair_start[k] .. pair_start[k + 1] - 1
   int n_hblk, hb_log2[kMaxHeadBlocks], h0[kMaxHeadBlocks], pair_start[kMaxHeadBlocks + 1];
   // per tile pair, worked out on the host so that taking up an item costs a few loads, not a dozen divisions
+  // (the two tiles of an item may come from DIFFERENT head blocks: the odd last tiles of two blocks share one K/V stream)
   struct PairInfo {
-    int16_t ji0;      // first (j, i) row
+    int16_t ji0[2];   // first (j, i) row of each tile
     int16_t jb0_rel;  // first boundary whose block keys sit in the tail tiles, relative to boundary_lo
-    uint8_t blk, hs, h0, ntq, n_tail, pad[3];
+    uint8_t blk[2], hs[2], h0[2];  // per tile: head block, log2(heads per row group), first head
+    uint8_t ntq, n_tail;
   } pair[kMaxPairs];
   int nsplit_log2;
 
@@ -120,9 +122,16 @@ struct TcCfg {
 struct Item {
   int n, g, pair, split, ntq, L, t0, t1, nctx, n_ctx_it, n_tail, n_iter, jb0, slot;
   int npieces, slot0, item;    // KV pieces of the item (1: whole), scratch slot of piece 0, item id
-  int blk, hs, h0, ji_t, ji0;  // head block, log2(heads per row group), first head, (j, i) rows per tile, first (j, i) row
+  uint32_t geo0, geo1;  // per tile, packed (selected with a ternary, never indexed: the struct stays in registers):
+                        // first (j, i) row | log2(heads per row group) << 16 | first head << 20 | head block << 28
   long long c0;
 };
+
+__device__ __forceinline__ uint32_t tile_geo(const Item &I, int t) { return t ? I.geo1 : I.geo0; }
+__device__ __forceinline__ int geo_ji0(uint32_t g) { return (int)(g & 0xffffu); }
+__device__ __forceinline__ int geo_hs(uint32_t g) { return (int)((g >> 16) & 0xfu); }
+__device__ __forceinline__ int geo_h0(uint32_t g) { return (int)((g >> 20) & 0xffu); }
+__device__ __forceinline__ int geo_blk(uint32_t g) { return (int)(g >> 28); }
 
 // The low k bits set (k <= 0: none, k >= 32: all).
 __device__ __forceinline__ uint32_t bits_below(int k) { return k <= 0 ? 0u : (k >= 32 ? 0xffffffffu : ((1u << k) - 1u)); }
@@ -162,12 +171,9 @@ __device__ __forceinline__ Item decode_item(const TcParams &P, int id) {
   I.pair = (int)(x >> P.nsplit_log2);
   I.split = (int)(x & ((1u << P.nsplit_log2) - 1u));
   const TcParams::PairInfo pi = P.pair[I.pair];
-  I.blk = pi.blk;
-  I.hs = pi.hs;
-  I.h0 = pi.h0;
-  I.ji_t = 128 >> I.hs;
+  I.geo0 = (uint32_t)(uint16_t)pi.ji0[0] | ((uint32_t)pi.hs[0] << 16) | ((uint32_t)pi.h0[0] << 20) | ((uint32_t)pi.blk[0] << 28);
+  I.geo1 = (uint32_t)(uint16_t)pi.ji0[1] | ((uint32_t)pi.hs[1] << 16) | ((uint32_t)pi.h0[1] << 20) | ((uint32_t)pi.blk[1] << 28);
   I.ntq = pi.ntq;
-  I.ji0 = pi.ji0;
   if (P.use_ctx_p) {
     I.c0 = P.ctx_off_p[I.n];
     I.L = P.ctx_len_p[I.n];
@@ -221,9 +227,10 @@ __device__ __forceinline__ void merge_pieces_n(const TcParams &P, const Item &I,
   constexpr int kUnroll = kNp == 2 ? 2 : 1;  // parts whose loads are in flight together
   const int R = row_begin + tid % n_rows;
   const int t = R >> 7, r = R & 127;
-  const int ji = I.ji0 + t * I.ji_t + (r >> I.hs);
+  const uint32_t geo = tile_geo(I, t);
+  const int ji = geo_ji0(geo) + (r >> geo_hs(geo));
   if (t >= I.ntq || ji >= P.n_rows) return;
-  const int h = I.g * A.G + I.h0 + (r & ((1 << I.hs) - 1));
+  const int h = I.g * A.G + geo_h0(geo) + (r & ((1 << geo_hs(geo)) - 1));
   const size_t orow = ((size_t)I.n * A.q_req_rows + A.lo * A.Bq + ji) * A.Hq + h;
   // weights of the pieces for this row: exp2((m_piece - m) c) / sum; a piece without visible keys wrote no rows (its slot
   // may hold anything) and gets weight 0
@@ -374,12 +381,14 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
       ok = __all_sync(0xffffffffu, mbar_wait(q_empty, (k & 1) ^ 1u, abort_flag));
       if (!ok) break;
       if (lane == 0) {
-        const int qrow0 = I.n * A.q_req_rows + A.lo * A.Bq + I.ji0;
+        const int qrow0 = I.n * A.q_req_rows + A.lo * A.Bq;
         mbar_arrive_expect_tx(q_full, (uint32_t)(I.ntq * Cfg::kTileBytes));
-        for (int t = 0; t < I.ntq; ++t)
+        for (int t = 0; t < I.ntq; ++t) {
+          const uint32_t geo = tile_geo(I, t);
           for (int sb = 0; sb < Cfg::kSlabs; ++sb)
-            tma_load_3d(sQ + t * Cfg::kTileBytes + sb * Cfg::kSlabBytes, &P.map_q[I.blk], q_full, sb * 64, I.g * A.G + I.h0,
-                        qrow0 + t * I.ji_t);
+            tma_load_3d(sQ + t * Cfg::kTileBytes + sb * Cfg::kSlabBytes, &P.map_q[geo_blk(geo)], q_full, sb * 64, I.g * A.G + geo_h0(geo),
+                        qrow0 + geo_ji0(geo));
+        }
       }
       // load order K0 K1 V0 K2 V1 ... K(n-1) V(n-2) V(n-1): the order the MMA issuer consumes them in
       // (the scores of iteration it + 1 are issued before the PV product of iteration it); slot = (ld + q) % kSlots
@@ -548,7 +557,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
         ragged_nv = (I.t1 == I.nctx) ? (I.L & 127) : 0;  // valid keys of a part-filled last context tile (0: it is full or not ours)
         // a mask-slot row: its boundary, counted from the first one whose block sits in the tail tiles, and its anchor
         // prefix; a spine row (an anchor as a query): no own block (-1), and anchors 0 .. itself
-        const int ji = I.ji0 + t * I.ji_t + (r >> I.hs);
+        const int ji = geo_ji0(tile_geo(I, t)) + (r >> geo_hs(tile_geo(I, t)));
         const bool is_spine = ji >= P.n_ji;
         jrel = is_spine ? -1 : A.lo + ji / A.Bq - I.jb0;
         na_row = is_spine ? ji - P.n_ji + 1 : max(0, min(A.lo + ji / A.Bq + A.pb, A.S));
@@ -659,9 +668,10 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
       // ---- output of this item (the MMA issuer cannot touch O_t again before this tile's next p_full arrive)
       if (!ok) break;
       const Item I = fetch_item(P, qi);
-      const int ji = I.ji0 + t * I.ji_t + (r >> I.hs);
+      const uint32_t geo = tile_geo(I, t);
+      const int ji = geo_ji0(geo) + (r >> geo_hs(geo));
       const bool valid = (t < I.ntq) && (ji < P.n_rows);
-      const int h = I.g * A.G + I.h0 + (r & ((1 << I.hs) - 1));
+      const int h = I.g * A.G + geo_h0(geo) + (r & ((1 << geo_hs(geo)) - 1));
       const size_t orow = ((size_t)I.n * A.q_req_rows + A.lo * A.Bq + ji) * A.Hq + h;
       // split-KV: this CTA's partial rows go to an L2-resident scratch slot and are merged later
       const size_t pslot = ((size_t)I.slot * 2 + t) * 128 + r;
@@ -839,17 +849,20 @@ TcPlan plan_attention_tc(const dpara_shape *s, const int64_t *host_off, const in
     p.tiles_per_item = tiles_per_item;
     p.n_hblk = 0;
     p.n_pairs = 0;
+    int n_odd = 0;
     for (int bit = 4, h0 = 0; bit >= 0; --bit) {
       if (!(G & (1 << bit))) continue;
       const int ji_t = 128 >> bit, tiles = (p.n_rows + ji_t - 1) / ji_t;
       p.hb_log2[p.n_hblk] = bit;
       p.h0[p.n_hblk] = h0;
       p.pair_start[p.n_hblk] = p.n_pairs;
-      p.n_pairs += (tiles + tiles_per_item - 1) / tiles_per_item;
+      p.n_pairs += tiles / tiles_per_item;
+      n_odd += tiles_per_item == 2 ? (tiles & 1) : 0;
       h0 += 1 << bit;
       ++p.n_hblk;
     }
     p.pair_start[p.n_hblk] = p.n_pairs;
+    p.n_pairs += (n_odd + 1) / 2;   // the blocks' odd last tiles, two by two
   };
   lay_out_items(2);
   p.S8 = (s->n_spine + 7) & ~7;
@@ -949,19 +962,36 @@ dpara_status launch_attention_tc(const AttnParams &A, const TcPlan &plan, const 
   P.nsplit_log2 = plan.nsplit == 8 ? 3 : (plan.nsplit == 4 ? 2 : (plan.nsplit == 2 ? 1 : 0));
   P.has_tail = (A.S > 0) || P.has_blk;
   P.n_items = (int)(plan.items * plan.nsplit);
-  for (int x = 0; x < plan.n_pairs; ++x) {
-    int blk = 0;
-    while (blk + 1 < plan.n_hblk && x >= plan.pair_start[blk + 1]) ++blk;
-    const int ji_t = 128 >> plan.hb_log2[blk], pl = x - plan.pair_start[blk];
+  {
+    // the items of a (request, KV head): per head block its tiles two by two (or one by one); the odd last tiles of the
+    // blocks, which all cover the highest (j, i) rows, are paired with one another
+    struct Tile { int blk, idx; };
+    std::vector<std::vector<Tile>> items;
+    std::vector<Tile> odd;
     const int tpi = plan.tiles_per_item;
-    const int ntq = std::min(tpi, (plan.n_rows + ji_t - 1) / ji_t - pl * tpi);
-    // boundaries whose own blocks the pair's mask-slot rows need (none if the pair holds spine rows only)
-    const int ji0 = pl * tpi * ji_t, ji_last = std::min(ji0 + ntq * ji_t, plan.n_ji) - 1;
-    TcParams::PairInfo &pi = P.pair[x];
-    pi.ji0 = (int16_t)ji0;
-    pi.jb0_rel = (int16_t)(ji0 / A.Bq);
-    pi.blk = (uint8_t)blk; pi.hs = (uint8_t)plan.hb_log2[blk]; pi.h0 = (uint8_t)plan.h0[blk]; pi.ntq = (uint8_t)ntq;
-    pi.n_tail = (uint8_t)tail_tiles(P.has_tail, P.has_blk, ji_last >= ji0 ? ji_last / A.Bq - ji0 / A.Bq + 1 : 0, plan.cap0, plan.cap);
+    for (int blk = 0; blk < plan.n_hblk; ++blk) {
+      const int ji_t = 128 >> plan.hb_log2[blk], tiles = (plan.n_rows + ji_t - 1) / ji_t;
+      for (int i = 0; i + tpi <= tiles; i += tpi) items.push_back(tpi == 2 ? std::vector<Tile>{{blk, i}, {blk, i + 1}} : std::vector<Tile>{{blk, i}});
+      if (tpi == 2 && (tiles & 1)) odd.push_back({blk, tiles - 1});
+    }
+    for (size_t i = 0; i < odd.size(); i += 2) items.push_back(i + 1 < odd.size() ? std::vector<Tile>{odd[i], odd[i + 1]} : std::vector<Tile>{odd[i]});
+    if ((int)items.size() != plan.n_pairs) return DPARA_ERR_INVALID_ARG;   // (plan and table disagree: cannot happen)
+    for (int x = 0; x < plan.n_pairs; ++x) {
+      TcParams::PairInfo &pi = P.pair[x];
+      memset(&pi, 0, sizeof(pi));
+      pi.ntq = (uint8_t)items[x].size();
+      // boundaries whose own blocks the item's mask-slot rows need (none if it holds spine rows only)
+      int jb_first = 1 << 30, jb_last = -1;
+      for (int t = 0; t < pi.ntq; ++t) {
+        const int blk = items[x][t].blk, ji_t = 128 >> plan.hb_log2[blk], ji0 = items[x][t].idx * ji_t;
+        pi.ji0[t] = (int16_t)ji0;
+        pi.blk[t] = (uint8_t)blk; pi.hs[t] = (uint8_t)plan.hb_log2[blk]; pi.h0[t] = (uint8_t)plan.h0[blk];
+        const int ji_last = std::min(ji0 + ji_t, plan.n_ji) - 1;
+        if (ji_last >= ji0) { jb_first = std::min(jb_first, ji0 / A.Bq); jb_last = std::max(jb_last, ji_last / A.Bq); }
+      }
+      pi.jb0_rel = (int16_t)(jb_last >= 0 ? jb_first : 0);
+      pi.n_tail = (uint8_t)tail_tiles(P.has_tail, P.has_blk, jb_last >= 0 ? jb_last - jb_first + 1 : 0, plan.cap0, plan.cap);
+    }
   }
 
   P.c_log2 = A.scale * 1.4426950408889634f;

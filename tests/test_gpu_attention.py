@@ -80,6 +80,7 @@ def test_shapes(shape):
     W.AttnShape((200, 130, 77, 300, 64, 1, 257, 129), 16, 8, 128, 4, 8),      # one query tile per item: the second tile is absent
     W.AttnShape((520, 129, 64, 300, 1, 257, 128, 0), 40, 8, 128, 6, 8),       # group size 5, ragged, an empty context
     W.AttnShape((150,) * 8, 32, 8, 128, 16, 16, 1, 16),                       # 16 boundaries x 16 slots: the widest tail tile
+    W.AttnShape((200, 130, 77, 300, 64, 1, 257, 129), 40, 8, 128, 9, 8),      # group size 5, 72 rows: three 4-head tiles and one 1-head tile -- the two odd tiles share an item
 ])
 def test_large_batch_shapes(shape):
     """Batches with at least 64 work items at head_dim 128: the persistent kernel without a KV split, every CTA busy."""
