@@ -352,7 +352,49 @@ __global__ void __launch_bounds__(kVsThreads) verify_sampling_kernel(const Verif
   __threadfence();
   __shared__ unsigned long long s_T, s_basepref;
   __shared__ int s_chunk, s_which, s_tok;
-  if (tid == 0) {
+  if (P.nchunks <= kVsThreads) {
+    // thread k holds chunk k's two sums: totals by a block reduction, the crossing chunk by a block scan (one L2 round trip
+    // for all the sums; a single thread walking the chunks paid one round trip per chunk, ~0.7 us each)
+    unsigned long long c0 = 0, c1 = 0;
+    if (tid < P.nchunks) {
+      c0 = __ldcg(P.ws64 + ((size_t)n * P.nchunks + tid) * 2);
+      c1 = __ldcg(P.ws64 + ((size_t)n * P.nchunks + tid) * 2 + 1);
+    }
+    unsigned long long r0 = warp_sum_u64(c0), r1 = warp_sum_u64(c1);
+    if ((tid & 31) == 0) { s_w[0][tid >> 5] = r0; s_w[1][tid >> 5] = r1; }
+    if (tid == 0) { s_tok = 0; s_chunk = 0; }
+    __syncthreads();
+    unsigned long long W0 = 0, W1 = 0;
+#pragma unroll
+    for (int w = 0; w < kVsThreads / 32; ++w) { W0 += s_w[0][w]; W1 += s_w[1][w]; }
+    const int which = W0 ? 0 : (W1 ? 1 : 2);
+    __syncthreads();   // s_w is reused by the scan
+    if (tid == 0) s_which = which;
+    if (which < 2) {
+      const unsigned long long Wt = which ? W1 : W0;
+      // a uniform is m * 2^-24 with m < 2^24; anything at or above 1 is taken as the largest uniform, so the
+      // threshold stays below the total weight and the draw inside the vocabulary
+      unsigned int m = __float2uint_rn(fminf(P.uniforms[(size_t)n * P.J + g], 1.0f) * 16777216.0f);
+      m = m > 16777215u ? 16777215u : m;
+      const unsigned long long lo = (unsigned long long)m * Wt;  // low 64 bits
+      const unsigned long long hi = __umul64hi((unsigned long long)m, Wt);
+      const unsigned long long T = (hi << 40) | (lo >> 24);  // (m * W) >> 24, m < 2^24 so it fits
+      const unsigned long long sel = which ? c1 : c0;
+      unsigned long long inc = sel;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const unsigned long long t = __shfl_up_sync(0xffffffffu, inc, o);
+        if ((tid & 31) >= o) inc += t;
+      }
+      if ((tid & 31) == 31) s_w[0][tid >> 5] = inc;
+      __syncthreads();
+      unsigned long long before = 0;
+      for (int w = 0; w < (tid >> 5); ++w) before += s_w[0][w];
+      inc += before;
+      // the first chunk whose inclusive sum exceeds the threshold (T < total: there is exactly one such first chunk)
+      if (tid < P.nchunks && inc > T && inc - sel <= T) { s_chunk = tid; s_T = T; s_basepref = inc - sel; }
+    }
+  } else if (tid == 0) {
     unsigned long long W0 = 0, W1 = 0;
     for (int k = 0; k < P.nchunks; ++k) {
       W0 += __ldcg(P.ws64 + ((size_t)n * P.nchunks + k) * 2);
