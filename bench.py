@@ -141,6 +141,10 @@ class StepRunner:
                                   prefix_base=a.prefix_base, n_spine=a.spine, boundary_lo=a.n_boundaries - 1)
         self.vplan = dp.VerifyPlan(batch=v.batch, n_boundaries=v.n_boundaries, vocab=v.vocab, block=v.block,
                                    hidden=v.hidden, mode=0)
+        # the same call allowed to start while the attention kernel in front of it is still running (it waits for it only
+        # before it gathers the selected branch): the case where verification has resolved before the precompute ends
+        self.vplan_early = dp.VerifyPlan(batch=v.batch, n_boundaries=v.n_boundaries, vocab=v.vocab, block=v.block,
+                                         hidden=v.hidden, mode=0, early_start=True)
         self.reps = self.out.view(a.batch, a.n_boundaries, a.block, a.hidden)
         self.flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device="cuda")
         self.pinned = None
@@ -157,6 +161,26 @@ class StepRunner:
     def step(self):
         self.attention()
         self.verify()
+
+    def step_early(self):
+        d = self.dev
+        self.attention()
+        self.vplan_early(target=d["target"], draft_tokens=d["draft_tokens"], reps=self.reps)
+
+    def timed_early_steps(self, k: int):
+        """k steps with the early-start verify/select (ms each), and a check that it selects what the plain call selects."""
+        torch = self.torch
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(k)]
+        for s in range(k):
+            self.flush.zero_()
+            ev[s][0].record()
+            self.step_early()
+            ev[s][1].record()
+        torch.cuda.synchronize()
+        self.step()
+        torch.cuda.synchronize()
+        same = all(bool(torch.equal(getattr(self.vplan, f), getattr(self.vplan_early, f))) for f in ("accept_len", "bonus", "out_tokens", "selected"))
+        return [e[0].elapsed_time(e[1]) for e in ev], same
 
     def timed_steps(self, k: int, single_boundary: bool = False, parts: bool = True):
         """k steps, each bracketed by CUDA events on the launching stream, L2 flushed in between.
@@ -418,7 +442,7 @@ def graph_timed_b1(r: "StepRunner", k: int = 20):
                 ts.append(e0.elapsed_time(e1) * 1e3 / k)
         return statistics.median(ts)
     base = timed(lambda: None)
-    return {"graph_replay": {"step_us": timed(r.step) - base, "attention_us": timed(r.attention) - base,
+    return {"graph_replay": {"step_us": timed(r.step) - base, "early_start_step_us": timed(r.step_early) - base, "attention_us": timed(r.attention) - base,
                              "verify_select_us": timed(r.verify) - base, "single_boundary_attention_us": timed(lambda: r.attention(r.plan1)) - base,
                              "note": "k x (flush, calls) replayed from one CUDA graph, minus k x flush"}}
 
@@ -884,11 +908,14 @@ def main():
                                   "unit": "GB/s", "frac": verify_bytes(wl.verify) / (ver_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
                                   "us": ver_ms * 1e3, "bytes": verify_bytes(wl.verify)}}
 
+    te16, same16 = run.timed_early_steps(args.steps)
+    early16 = {"step_us": statistics.median(te16) * 1e3, "same_selection_as_plain_call": same16}
     out = {"metric": METRIC, "value": step_us, "unit": "us", "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
            "ms_per_step": step_us / 1e3, "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
            "data": "synthetic", "config": cfg, "clocks": clocks, "gpu_launches": int(launches),
            "e2e": {"value": e2e_us, "unit": "us", "h2d_bytes_per_step": run.h2d_bytes, "d2h_bytes_per_step": run.d2h_bytes},
-           "roofline": roofline, "steps_per_s_all_gpus": world * 1e6 / step_us}
+           "roofline": roofline, "steps_per_s_all_gpus": world * 1e6 / step_us,
+           "early_start_verify": early16}
 
     if rank == 0 and world == 1:
         # the b = 1 step (cfg2) and the single-boundary (conventional) draft step beside it
@@ -904,6 +931,10 @@ def main():
                      "single_boundary_attention_us": statistics.median(p[1] for p in s2) * 1e3,
                      "all_over_single": a2 / (statistics.median(p[1] for p in s2) * 1e3), "allowance": w2.attn.n_boundaries,
                      "attention_gbs": attention_bytes(w2.attn) / (a2 * 1e-6) / 1e9, "attention_tflops": attention_flops(w2.attn) / (a2 * 1e-6) / 1e12}
+        te, same = r2.timed_early_steps(max(args.steps, 20))
+        out["b1"]["early_start"] = {"step_us": statistics.median(te) * 1e3, "same_selection_as_plain_call": same,
+                                    "note": "verify/select with DPARA_VERIFY_EARLY_START: it reads the (already resident) target logits while the "
+                                            "attention kernel before it is still running and waits for it only before the branch gather"}
         out["b1"].update(graph_timed_b1(r2))
         del r2
         if not args.no_layer:

@@ -200,7 +200,17 @@ typedef struct {
   void *selected;              /* [b][Bq][hidden] bf16 = reps[n][r] (required when reps != NULL) */
   int32_t rep_req_rows;        /* rows of `hidden` elements from one request's representations to the next request's;
                                   0 = J * Bq (packed).  J * Bq + S for the output of a call with spine query rows */
+  int32_t flags;               /* 0, or DPARA_VERIFY_EARLY_START */
 } dpara_verify_io;
+
+/* dpara_verify_io.flags.  EARLY_START: the call may begin before the work enqueued immediately before it on the stream
+ * has finished -- it reads target / draft_probs / draft_tokens / uniforms and uses its workspace and its small outputs
+ * straight away, and waits for that work only before it reads `reps` (and before it completes).  The caller promises that
+ * the immediately preceding work writes none of those inputs and touches neither this call's workspace nor its outputs:
+ * the case of Alg. 1 when verification has resolved while the drafter's precompute (the producer of `reps`) is still
+ * running on the same stream.  Only work that releases its dependents early is affected (this library's own kernels do);
+ * behind anything else the flag changes nothing. */
+#define DPARA_VERIFY_EARLY_START 1
 
 /* Bytes of scratch dpara_verify_select needs; only the sizes and mode of `io` are read. 0 on bad sizes. */
 size_t dpara_verify_workspace_bytes(const dpara_verify_io *io);

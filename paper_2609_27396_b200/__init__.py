@@ -54,7 +54,7 @@ class VerifyIO(C.Structure):
                 ("hidden", C.c_int32), ("mode", C.c_int32), ("target", C.c_void_p), ("draft_probs", C.c_void_p),
                 ("draft_tokens", C.c_void_p), ("uniforms", C.c_void_p), ("reps", C.c_void_p), ("accept_len", C.c_void_p),
                 ("bonus", C.c_void_p), ("gather_idx", C.c_void_p), ("out_tokens", C.c_void_p), ("selected", C.c_void_p),
-                ("rep_req_rows", C.c_int32)]
+                ("rep_req_rows", C.c_int32), ("flags", C.c_int32)]
 
 
 lib.dpara_draft_workspace_bytes.restype = C.c_size_t
@@ -262,13 +262,20 @@ def draft_with_spine_queries(q_rows, n_boundaries: int, block: int, k_ctx, v_ctx
     return (out, lse, plan.status) if want_lse else (out, plan.status)
 
 
+VERIFY_EARLY_START = 1
+
+
 class VerifyPlan:
     """Fixed-address outputs and workspace for repeated verify/select calls on one shape."""
 
     def __init__(self, *, batch: int, n_boundaries: int, vocab: int, block: int, hidden: int, mode: int, rep_req_rows: int = 0,
-                 device="cuda"):
+                 early_start: bool = False, device="cuda"):
+        """early_start: DPARA_VERIFY_EARLY_START -- the call may begin while the work enqueued right before it is still
+        running and waits for it only before it reads `reps` (the caller promises that work writes none of the other
+        inputs and touches neither the workspace nor the outputs)."""
         self.io = VerifyIO(batch, n_boundaries, vocab, block, hidden, mode)
         self.io.rep_req_rows = rep_req_rows
+        self.io.flags = VERIFY_EARLY_START if early_start else 0
         self.accept_len = torch.zeros(batch, dtype=torch.int32, device=device)
         self.bonus = torch.zeros(batch, dtype=torch.int32, device=device)
         self.gather_idx = torch.zeros(batch, dtype=torch.int32, device=device)

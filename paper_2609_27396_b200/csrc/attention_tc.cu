@@ -339,8 +339,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
   const int q_begin = P.use_seg ? (team < P.seg_teams ? (int)P.team_first[team] : 0) : (P.use_sched ? (int)P.cta_first[blockIdx.x] : (int)blockIdx.x);
   const int q_end = P.use_seg ? (team < P.seg_teams ? (int)P.team_first[team + 1] : 0) : (P.use_sched ? (int)P.cta_first[blockIdx.x + 1] : P.n_items);
   const int q_step = (P.use_seg || P.use_sched) ? 1 : (int)gridDim.x;
-  pdl_launch_dependents();
   pdl_wait();  // nothing above touches global memory
+  pdl_launch_dependents();
   // (a CTA of a cluster must not leave early: its peers meet it at the cluster barriers below)
   if (P.nsplit == 1 && A.status_word && (*reinterpret_cast<volatile int32_t *>(A.status_word) & (int32_t)DPARA_STATUS_TIMEOUT)) return;
 

@@ -38,8 +38,8 @@ struct AppendParams {
 __global__ void __launch_bounds__(128) append_rows_kernel(const AppendParams P) {
   extern __shared__ float s_cs[];  // cos[D/2], sin[D/2]
   const int n = blockIdx.x / P.J, i = blockIdx.x % P.J, tid = threadIdx.x, g = blockIdx.y;
-  pdl_launch_dependents();
   pdl_wait();
+  pdl_launch_dependents();
   const uint16_t *knorm_w = P.knorm_w[g];
   const float *kv_parts = P.kv_parts + (size_t)g * P.n_parts * P.part_stride;
   const int r = P.accept_len[n];
@@ -121,8 +121,8 @@ __global__ void __launch_bounds__(128) append_rows_kernel(const AppendParams P) 
 
 // After every layer has read the old lengths: L_n += r_n + 1 for the requests that fitted.
 __global__ void append_commit_kernel(int64_t *ctx_len, const int64_t *capacity, const int32_t *accept_len, int b, int J) {
-  pdl_launch_dependents();
   pdl_wait();
+  pdl_launch_dependents();
   for (int n = blockIdx.x * blockDim.x + threadIdx.x; n < b; n += gridDim.x * blockDim.x) {
     const int r = accept_len[n];
     const long long L = ctx_len[n];

@@ -31,11 +31,13 @@ inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 
     if (e_ != cudaSuccess) return DPARA_ERR_CUDA;              \
   } while (0)
 
-// Programmatic dependent launch.  Every kernel of this library starts with pdl_launch_dependents() (the next kernel on the
-// stream may be set up and its CTAs made resident as SMs free up) followed by pdl_wait() (blocks until the kernels before it
-// have completed and their writes are visible) BEFORE it reads or writes any global memory; launched through launch_pdl
-// the kernel's launch latency and prologue then overlap the tail of its predecessor.  Without the launch attribute both
-// instructions do nothing.
+// Programmatic dependent launch.  Every kernel of this library runs pdl_wait() (blocks until the kernels before it have
+// completed and their writes are visible) BEFORE it reads or writes any global memory, then pdl_launch_dependents() (the
+// next kernel on the stream may be set up and its CTAs made resident as SMs free up); launched through launch_pdl the
+// kernel's launch latency and set-up then overlap its predecessor.  Wait first, trigger second: a dependent is only ever
+// released by a kernel whose own predecessors are complete, so a dependent that reads some of its inputs before its own
+// wait (the early-start form of verify/select) can race with nothing older than its immediate predecessor.  Without the
+// launch attribute both instructions do nothing.
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 

@@ -148,7 +148,6 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
     *abort_flag = 0;
     fence_barrier_init();
   }
-  pdl_launch_dependents();
   if (warp == 5) {
     tmem_alloc(tmem_slot, 512);
     tmem_relinquish();
@@ -158,6 +157,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
   pdl_wait();  // nothing above touches global memory: the set-up overlaps the tail of the kernel before
+  pdl_launch_dependents();
 
   // Persistent: CTA c computes tiles c, c + gridDim.x, ...; tile id = n_tile * m_tiles + m_tile, so the CTAs
   // running together cover all M rows of a few weight tiles (A stays in L2, each weight tile is read once).
@@ -288,7 +288,6 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1) gemm_tc
     *abort_flag = 0;
     fence_barrier_init();
   }
-  pdl_launch_dependents();
   if (warp == 5) {
     tmem_alloc_pair(tmem_slot, 512);
     tmem_relinquish_pair();
@@ -299,6 +298,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1) gemm_tc
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
   pdl_wait();  // nothing above touches global memory: the set-up overlaps the tail of the kernel before
+  pdl_launch_dependents();
 
   if (warp == 4) {
     if (lane == 0) {

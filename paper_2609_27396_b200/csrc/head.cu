@@ -88,13 +88,13 @@ __global__ void __launch_bounds__(kThreads, 1) ar_head_kernel(const __grid_const
     *abort_flag = 0;
     fence_barrier_init();
   }
-  pdl_launch_dependents();
   if (warp == kMmaWarp) { tmem_alloc(tmem_slot, 64); tmem_relinquish(); }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
   pdl_wait();  // nothing above touches global memory
+  pdl_launch_dependents();
   // this CTA's tiles: blockIdx.x, blockIdx.x + gridDim.x, ... (the same in every step)
   const int my_tiles = (P.n_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
   const int step_begin = kSample ? P.step0 : 0, step_end = kSample ? P.step0 + 1 : P.block;
@@ -349,8 +349,8 @@ __global__ void __launch_bounds__(kPickThreads) head_sample_kernel(const float *
                                                                    int step, int chunk) {
   const int n = blockIdx.y, c = blockIdx.x, n_chunks = gridDim.x, tid = threadIdx.x;
   const float *row = z + (size_t)n * vocab;
-  pdl_launch_dependents();
   pdl_wait();
+  pdl_launch_dependents();
   __shared__ float s_max[kPickThreads / 32];
   __shared__ double s_warp[kPickThreads / 32];
   __shared__ int s_flag;

@@ -20,8 +20,8 @@ template <bool kF32In>
 __global__ void __launch_bounds__(128) rmsnorm_kernel(const void *__restrict__ x, const uint16_t *__restrict__ gain,
                                                       uint16_t *__restrict__ out, int H, float eps) {
   const int row = blockIdx.x, tid = threadIdx.x;
-  pdl_launch_dependents();
   pdl_wait();
+  pdl_launch_dependents();
   float ss = 0.f;
   for (int c = tid * 8; c < H; c += 128 * 8) {
     float v[8];
@@ -94,8 +94,8 @@ __global__ void __launch_bounds__(128) qk_norm_rope_kernel(const QkParams P) {
   const int row = blockIdx.x, tid = threadIdx.x;
   const int half = P.D / 2;
   const int R = P.Bq * P.J + P.Sq;
-  pdl_launch_dependents();
   pdl_wait();
+  pdl_launch_dependents();
   const int n = row / R, rr = row % R;
   if (P.use_rope) {
     const int rel = rr < P.Bq * P.J ? rr / P.Bq + 2 + rr % P.Bq : rr - P.Bq * P.J;  // mask slot (j, i): j + 2 + i; spine row s: s

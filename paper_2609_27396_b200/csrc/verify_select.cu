@@ -76,6 +76,7 @@ struct VerifyParams {
   unsigned int *counters;    // greedy: [b*J] row counters, then one "rows finished" counter; sampling: [b]
   unsigned long long *masks; // greedy: [b] completed-row masks
   int b, J, V, nchunks, vec_ok;
+  int early;         // early start: no wait for the preceding kernel until `reps` is read / the workspace is handed back
   size_t rep_bytes;  // Bq * hidden * 2
   size_t req_bytes;  // from one request's representations to the next request's (J * rep_bytes when packed)
 };
@@ -97,8 +98,10 @@ template <int kGreedyLoads>
 __global__ void __launch_bounds__(kVsThreads, kGreedyLoads >= 16 ? 3 : (kGreedyLoads >= 8 ? 4 : 6)) verify_greedy_kernel(const VerifyParams P) {
   constexpr int kGreedyChunk = kGreedyLoads * 1024;  // floats per CTA
   const int tid = threadIdx.x;
-  pdl_launch_dependents();
-  pdl_wait();
+  if (!P.early) {
+    pdl_wait();
+    pdl_launch_dependents();
+  }
   // rows are handed out position-major (every request's row 0 first, then every row 1, ...): the early rows,
   // which decide the accepted length, finish early for ALL requests
   const int n = blockIdx.y % P.b;
@@ -222,6 +225,7 @@ __global__ void __launch_bounds__(kVsThreads, kGreedyLoads >= 16 ? 3 : (kGreedyL
   }
   __syncthreads();
   if (s_act) {
+    if (P.early) pdl_wait();   // the selected branch comes from the kernel before
     const int r = s_r;
     if (tid == 0) {
       P.accept_len[n] = r;
@@ -242,6 +246,7 @@ __global__ void __launch_bounds__(kVsThreads, kGreedyLoads >= 16 ? 3 : (kGreedyL
   }
   __syncthreads();
   if (!s_last) return;
+  if (P.early) pdl_wait();     // (the call does not complete before the work in front of it has)
   for (int i = tid; i < P.b * P.J; i += kVsThreads) { P.ws64[i] = 0ull; P.counters[i] = 0u; }
   for (int i = tid; i < P.b; i += kVsThreads) P.masks[i] = 0ull;
   if (tid == 0) P.counters[(size_t)P.b * P.J] = 0u;
@@ -261,8 +266,10 @@ __device__ __forceinline__ void weights_of(float p, float q, bool residual, unsi
 
 __global__ void __launch_bounds__(kVsThreads) verify_sampling_kernel(const VerifyParams P) {
   const int tid = threadIdx.x;
-  pdl_launch_dependents();
-  pdl_wait();
+  if (!P.early) {
+    pdl_wait();
+    pdl_launch_dependents();
+  }
   const int n = blockIdx.y;
   const int c = blockIdx.x;
   const int g = P.J - 1;
@@ -349,6 +356,7 @@ __global__ void __launch_bounds__(kVsThreads) verify_sampling_kernel(const Verif
   if (!s_flag) return;
 
   // ---- last CTA of request n: total weight, threshold, locate the crossing
+  if (P.early) pdl_wait();     // before the branch is read and before the request's part of the call completes
   __threadfence();
   __shared__ unsigned long long s_T, s_basepref;
   __shared__ int s_chunk, s_which, s_tok;
@@ -524,6 +532,7 @@ static dpara_status validate_verify(const dpara_verify_io *io) {
   dpara_status s = validate_dims(io);
   if (s != DPARA_OK) return s;
   if (!io->target || !io->accept_len || !io->bonus || !io->gather_idx) return DPARA_ERR_INVALID_ARG;
+  if (io->flags & ~DPARA_VERIFY_EARLY_START) return DPARA_ERR_INVALID_ARG;
   if (io->n_boundaries > 1 && !io->draft_tokens) return DPARA_ERR_INVALID_ARG;
   if (io->mode == 1 && (!io->uniforms || (io->n_boundaries > 1 && !io->draft_probs))) return DPARA_ERR_INVALID_ARG;
   if (io->reps) {
@@ -563,6 +572,7 @@ dpara_status launch_verify(const dpara_verify_io *io, void *ws, int32_t *status_
   P.V = io->vocab;
   P.nchunks = chunks_of(io);
   P.rep_bytes = (size_t)io->block * io->hidden * 2;
+  P.early = (io->flags & DPARA_VERIFY_EARLY_START) ? 1 : 0;
   P.req_bytes = io->rep_req_rows > 0 ? (size_t)io->rep_req_rows * io->hidden * 2 : (size_t)io->n_boundaries * P.rep_bytes;
   size_t n64 = ws64_count(io);
   const size_t mask_off = align_up(n64 * 8, 256);
@@ -579,7 +589,10 @@ dpara_status launch_verify(const dpara_verify_io *io, void *ws, int32_t *status_
     // kernel it measured 5 us SLOWER than a plain launch, so only the small-grid forms ask for the early launch
     // (b = 1: 152 CTAs, 3 us faster).
     switch (greedy_loads_of(io)) {
-      case 16: verify_greedy_kernel<16><<<grid, kVsThreads, 0, st>>>(P); break;
+      case 16:
+        if (P.early) launch_pdl(verify_greedy_kernel<16>, dim3(grid), dim3(kVsThreads), 0, st, P);
+        else verify_greedy_kernel<16><<<grid, kVsThreads, 0, st>>>(P);
+        break;
       case 8: launch_pdl(verify_greedy_kernel<8>, dim3(grid), dim3(kVsThreads), 0, st, P); break;
       case 4: launch_pdl(verify_greedy_kernel<4>, dim3(grid), dim3(kVsThreads), 0, st, P); break;
       case 2: launch_pdl(verify_greedy_kernel<2>, dim3(grid), dim3(kVsThreads), 0, st, P); break;

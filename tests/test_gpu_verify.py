@@ -165,3 +165,36 @@ def test_sampling_uniform_of_one_is_clamped():
     v = W.VerifyInputs(W.VerifyShape(1, J, V, 2, 64, "sampling"), p, toks, None, q, u)
     ref = _check(v, 1)
     assert ref["accept_len"][0] == 0 and ref["bonus"][0] == 4100
+
+
+@pytest.mark.parametrize("mode", [0, 1])
+def test_early_start_behind_the_attention_kernel(mode):
+    """DPARA_VERIFY_EARLY_START: queued right behind the attention call that produces `reps`, the call starts on its other
+    inputs at once and waits for the attention only before the gather -- same outputs as the plain call, bit for bit,
+    every time (eight rounds with fresh attention inputs, so a gather that ran ahead would read the round before)."""
+    import paper_2609_27396_b200 as dp
+    from gpu_util import dev_bf16
+    w = W.workload(2)
+    a, v = w.attn, w.verify
+    plain = dp.VerifyPlan(batch=v.batch, n_boundaries=v.n_boundaries, vocab=v.vocab, block=v.block, hidden=v.hidden, mode=mode)
+    early = dp.VerifyPlan(batch=v.batch, n_boundaries=v.n_boundaries, vocab=v.vocab, block=v.block, hidden=v.hidden, mode=mode, early_start=True)
+    out = torch.zeros((a.batch, a.n_boundaries, a.block, a.n_q_heads, a.head_dim), dtype=torch.bfloat16, device="cuda")
+    reps = out.view(a.batch, a.n_boundaries, a.block, a.n_q_heads * a.head_dim)
+    for rnd in range(8):
+        inp = W.make_attn_inputs(a, 100 + rnd)
+        t = {k: dev_bf16(getattr(inp, k)) for k in ("q", "k_ctx", "v_ctx", "k_spine", "v_spine", "k_blk", "v_blk")}
+        plan = dp.DraftPlan(ctx_offsets=[int(x) for x in inp.ctx_offsets], n_boundaries=a.n_boundaries, block=a.block, n_q_heads=a.n_q_heads,
+                            n_kv_heads=a.n_kv_heads, head_dim=a.head_dim, prefix_base=a.prefix_base, n_spine=a.spine)
+        ver = W.make_verify_inputs(W.VerifyShape(v.batch, v.n_boundaries, v.vocab, v.block, v.hidden, "greedy" if mode == 0 else "sampling", v.agreement,
+                                                 v.logit_sigma), 200 + rnd)
+        kw = dict(target=torch.from_numpy(ver.target).cuda(), draft_tokens=torch.from_numpy(ver.draft_tokens).cuda())
+        if mode == 1:
+            kw.update(draft_probs=torch.from_numpy(ver.draft_probs).cuda(), uniforms=torch.from_numpy(ver.uniforms).cuda())
+        plan(**t, out=out)
+        early(reps=reps, **kw)
+        torch.cuda.synchronize()
+        plain(reps=reps, **kw)
+        torch.cuda.synchronize()
+        for f in ("accept_len", "bonus", "gather_idx", "out_tokens", "selected"):
+            assert torch.equal(getattr(plain, f), getattr(early, f)), (rnd, f)
+        assert plain.status.item() == early.status.item() == 0
