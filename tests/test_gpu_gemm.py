@@ -20,7 +20,9 @@ def _dev(bits):
     return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda().view(torch.bfloat16)
 
 
-@pytest.mark.parametrize("M,N,K", [(128, 256, 64), (128, 256, 256), (256, 512, 512), (200, 264, 192), (1024, 768, 1024), (40, 8, 64)])
+@pytest.mark.parametrize("M,N,K", [(128, 256, 64), (128, 256, 256), (256, 512, 512), (200, 264, 192), (1024, 768, 1024), (40, 8, 64),
+                                   (1024, 6144, 256),     # 192-column tiles, exact multiple (the QKV shape's tiling)
+                                   (300, 1000, 128)])     # ragged rows and a part-filled last 192-column tile
 def test_gemm_bf16_store(M, N, K):
     import paper_2609_27396_b200 as dp
     rng = np.random.default_rng(M + N + K)
